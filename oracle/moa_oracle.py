@@ -1,0 +1,412 @@
+"""CPU oracle for the Mixture-of-Attentions drafter forward step (arXiv 2410.03804).
+
+TEST INFRASTRUCTURE ONLY. Nothing on the product path may import this file;
+only the tests, the smoke check and the CPU-baseline leg of the benchmark do.
+It shares no code with the CUDA path and is deliberately plain and slow:
+numpy in fp64, one step of the paper's method per function, in the paper's
+order. numpy's matmul / sort serve as library primitives for single steps.
+
+What the paper fixes and what is a reading of it
+------------------------------------------------
+The paper (Section 3.1, Algorithm 1, Section 2.2, hyper-parameter table in
+Appendix A.1) fixes: LSA = bidirectional self-attention over the layer axis,
+tokens independent, followed by a mean over layers; SA = causal self-attention
+over token embeddings (tree-masked while drafting a tree); CA = unmasked
+cross-attention from SA outputs into keys/values derived from the LSA output;
+LM head + softmax; an EAGLE-2-style tree: expand the B most probable, rank the
+B*B children by joint probability, keep B per level, D levels, finally keep the
+m best of the B + (D-1)*B*B pool. Attention softmax is done in higher
+precision than the storage type (Section 4, last paragraph before 4.1).
+
+The paper is silent on normalisation, biases, activation, positional encoding
+and block wiring. This oracle takes the Llama-style reading: pre-RMSNorm with a
+learnable gain before every attention and MLP, no biases, SwiGLU MLP, residual
+connections; rotary position embedding (half-split pairing) in SA only; none in
+LSA or CA; the LLM's final RMSNorm gain precedes the LM head; the MLP listed
+"after LSA" is applied per (token, layer) row before the mean. Joint
+probabilities are sums of fp32 log-probabilities. Ties break towards the
+smaller index everywhere.
+
+Parity status: every function below is pinned by tests/test_oracle_pins.py
+against closed forms, library routines, brute force or invariants. The model's
+outputs are NOT pinned against the authors' trained system (no worked example,
+weights or code exist here): "parity unpinned" in that sense only.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# elementary steps
+# --------------------------------------------------------------------------
+def rmsnorm(x, g, eps):
+    """n(x; g) = x * g / sqrt(mean(x^2) + eps), over the last axis."""
+    x = np.asarray(x, F64)
+    g = np.asarray(g, F64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x * g / np.sqrt(ms + eps)
+
+
+def softmax(a):
+    """Softmax over the last axis: subtract the max, exponentiate, divide by the sum."""
+    a = np.asarray(a, F64)
+    e = np.exp(a - np.max(a, axis=-1, keepdims=True))
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def silu(x):
+    x = np.asarray(x, F64)
+    return x / (1.0 + np.exp(-x))
+
+
+def linear(x, w):
+    """y = W x for a row-major weight W[out, in]; x may carry leading row axes."""
+    return np.matmul(np.asarray(x, F64), np.asarray(w, F64).T)
+
+
+def swiglu_mlp(u, w_gate, w_up, w_down):
+    """W_down (silu(W_gate u) * (W_up u))."""
+    return linear(silu(linear(u, w_gate)) * linear(u, w_up), w_down)
+
+
+def attend(q, K, V):
+    """Attention core for ONE query vector: softmax(q.K^T / sqrt(dh)) V.
+
+    q [dh], K [n, dh], V [n, dh] -> [dh]."""
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    a = K @ q / np.sqrt(q.shape[-1])
+    p = softmax(a)
+    return p @ V
+
+
+def kv_head_of(h, hq, hkv):
+    """Grouped-query attention: query head h reads kv head h // (hq // hkv)."""
+    return h // (hq // hkv)
+
+
+def rope(x, pos, theta):
+    """Rotary embedding of x [..., dh] at integer position pos.
+
+    Element i (< dh/2) is paired with element i + dh/2 and the pair is rotated
+    by the angle pos * theta^(-2i/dh). theta == 0 disables the rotation."""
+    x = np.asarray(x, F64)
+    if theta == 0:
+        return x.copy()
+    dh = x.shape[-1]
+    half = dh // 2
+    i = np.arange(half, dtype=F64)
+    ang = float(pos) * theta ** (-2.0 * i / dh)
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def lm_head_topk(o_hat, final_norm, w_lm, eps, B):
+    """LM head, log-softmax and the B most probable tokens (Eq. 1; Section 2.2).
+
+    z = W_lm n(o_hat; g_final); logp = z - logsumexp(z).
+    Order: log-probability descending, token id ascending on equality.
+    Returns (ids [B] int64, logp [B] float64, z [V] float64)."""
+    z = linear(rmsnorm(o_hat, final_norm, eps), w_lm)
+    zmax = np.max(z)
+    lse = zmax + np.log(np.sum(np.exp(z - zmax)))
+    logp = z - lse
+    order = np.lexsort((np.arange(z.shape[0]), -logp))[:B]
+    return order.astype(np.int64), logp[order], z
+
+
+# --------------------------------------------------------------------------
+# the drafter
+# --------------------------------------------------------------------------
+class Drafter:
+    """The drafter's layers, one method per step of Algorithm 1.
+
+    cfg: mapping with d_model, n_stack, d_stack, vocab, head_dim, lsa_hq,
+    lsa_hkv, sa_hq, sa_hkv, ca_hq, ca_hkv, rms_eps, rope_theta.
+    weights: mapping name -> array [out, in] (any float dtype; widened to fp64
+    where used)."""
+
+    def __init__(self, cfg, weights, cache_f64=True):
+        self.c = dict(cfg)
+        self.w_raw = weights
+        self._cache = {} if cache_f64 else None
+
+    def w(self, name):
+        if self._cache is None:
+            return np.asarray(self.w_raw[name], F64)
+        if name not in self._cache:
+            self._cache[name] = np.asarray(self.w_raw[name], F64)
+        return self._cache[name]
+
+    # ---- Layer Self-Attention (Section 3.1.1, "Layer Self-Attention") -----
+    def lsa_rows(self, X):
+        """LSA block for ONE token, before the mean. X [S, D_in] -> Z [S, D_in].
+
+        Rows of X are the S stacked layer activations; attention runs over
+        these S rows with a full (bidirectional) mask and no positional term."""
+        c = self.c
+        S = X.shape[0]
+        dh, hq, hkv = c["head_dim"], c["lsa_hq"], c["lsa_hkv"]
+        X = np.asarray(X, F64)
+        U = rmsnorm(X, self.w("lsa_norm1"), c["rms_eps"])
+        Q = linear(U, self.w("lsa_wq")).reshape(S, hq, dh)
+        K = linear(U, self.w("lsa_wk")).reshape(S, hkv, dh)
+        V = linear(U, self.w("lsa_wv")).reshape(S, hkv, dh)
+        O = np.zeros((S, hq, dh), F64)
+        for h in range(hq):
+            g = kv_head_of(h, hq, hkv)
+            for s in range(S):
+                O[s, h] = attend(Q[s, h], K[:, g], V[:, g])
+        Y = X + linear(O.reshape(S, hq * dh), self.w("lsa_wo"))
+        Z = Y + swiglu_mlp(rmsnorm(Y, self.w("lsa_norm2"), c["rms_eps"]),
+                           self.w("lsa_wgate"), self.w("lsa_wup"), self.w("lsa_wdown"))
+        return Z
+
+    def lsa_token(self, X):
+        """LSA followed by the mean aggregation over the layer axis: [S, D_in] -> [D_in]."""
+        return np.mean(self.lsa_rows(X), axis=0)
+
+    def lsa_forward(self, h_stack):
+        """kv = LSA_layer_with_mean(h) (Algorithm 1, both LSA_layer_with_mean steps): every
+        token independently. h_stack [n_tok, S, D_in] -> [n_tok, D_in]."""
+        return np.stack([self.lsa_token(h_stack[t]) for t in range(h_stack.shape[0])]) \
+            if h_stack.shape[0] else np.zeros((0, self.c["d_stack"]), F64)
+
+    # ---- Cross-attention keys / values (Section 3.1.2, "Cross-Attention") -
+    def ca_kv(self, kv):
+        """K_c = W_k n(kv), V_c = W_v n(kv): one row per context position.
+        kv [n, D_in] -> K_c, V_c [n, Hkv, dh]."""
+        c = self.c
+        u = rmsnorm(kv, self.w("ca_normkv"), c["rms_eps"])
+        n = u.shape[0]
+        return (linear(u, self.w("ca_wk")).reshape(n, c["ca_hkv"], c["head_dim"]),
+                linear(u, self.w("ca_wv")).reshape(n, c["ca_hkv"], c["head_dim"]))
+
+    # ---- Self-attention (Section 3.1.2, "Self-Attention") -----------------
+    def sa_qkv(self, tok, pos):
+        """Embedding, pre-norm, q/k/v projections and rotation for one token
+        at absolute position pos. Returns e [E], q [Hq,dh], k [Hkv,dh], v [Hkv,dh]."""
+        c = self.c
+        dh = c["head_dim"]
+        e = np.asarray(self.w_raw["embed"][int(tok)], F64)
+        u = rmsnorm(e, self.w("sa_norm1"), c["rms_eps"])
+        q = rope(linear(u, self.w("sa_wq")).reshape(c["sa_hq"], dh), pos, c["rope_theta"])
+        k = rope(linear(u, self.w("sa_wk")).reshape(c["sa_hkv"], dh), pos, c["rope_theta"])
+        v = linear(u, self.w("sa_wv")).reshape(c["sa_hkv"], dh)
+        return e, q, k, v
+
+    def sa_block(self, e, q, K, V):
+        """SA block for one row, given its embedding e, rotated queries q
+        [Hq,dh] and the key/value set it may see, K, V [n, Hkv, dh] (the row's
+        own key and value included by the caller). Returns x [E]."""
+        c = self.c
+        hq, hkv, dh = c["sa_hq"], c["sa_hkv"], c["head_dim"]
+        o = np.zeros((hq, dh), F64)
+        for h in range(hq):
+            g = kv_head_of(h, hq, hkv)
+            o[h] = attend(q[h], K[:, g], V[:, g])
+        a = e + linear(o.reshape(hq * dh), self.w("sa_wo"))
+        return a + swiglu_mlp(rmsnorm(a, self.w("sa_norm2"), c["rms_eps"]),
+                              self.w("sa_wgate"), self.w("sa_wup"), self.w("sa_wdown"))
+
+    # ---- Cross-attention block (Section 3.1.2; Algorithm 1, CA_layer step) -------
+    def ca_block(self, x, K_c, V_c):
+        """CA block for one row: queries from x, keys/values = ALL cached
+        K_c, V_c [n, Hkv, dh]; no mask at generation time, no positional term."""
+        c = self.c
+        hq, hkv, dh = c["ca_hq"], c["ca_hkv"], c["head_dim"]
+        qc = linear(rmsnorm(x, self.w("ca_normq"), c["rms_eps"]), self.w("ca_wq")).reshape(hq, dh)
+        o = np.zeros((hq, dh), F64)
+        for h in range(hq):
+            g = kv_head_of(h, hq, hkv)
+            o[h] = attend(qc[h], K_c[:, g], V_c[:, g])
+        cc = x + linear(o.reshape(hq * dh), self.w("ca_wo"))
+        return cc + swiglu_mlp(rmsnorm(cc, self.w("ca_norm2"), c["rms_eps"]),
+                               self.w("ca_wgate"), self.w("ca_wup"), self.w("ca_wdown"))
+
+    def head(self, o_hat, B):
+        return lm_head_topk(o_hat, self.w("final_norm"), self.w("lm_head"), self.c["rms_eps"], B)
+
+    # ---- prefix of the self-attention cache -------------------------------
+    def sa_prefix(self, toks, start=0):
+        """Rotated keys and values of prompt / accepted tokens at positions
+        start, start+1, ... -> K, V [n, Hkv, dh]."""
+        c = self.c
+        ks, vs = [], []
+        for i, t in enumerate(toks):
+            _, _, k, v = self.sa_qkv(t, start + i)
+            ks.append(k)
+            vs.append(v)
+        shape = (0, c["sa_hkv"], c["head_dim"])
+        return (np.stack(ks) if ks else np.zeros(shape, F64),
+                np.stack(vs) if vs else np.zeros(shape, F64))
+
+    # ---- one drafter forward for one row ----------------------------------
+    def forward_row(self, tok, pos, saK, saV, caK, caV, B):
+        """SA -> CA -> LM head for a token at position pos whose visible
+        self-attention keys/values (excluding itself) are saK, saV.
+        Returns dict(x, o_hat, ids, logp, k, v, z)."""
+        e, q, k, v = self.sa_qkv(tok, pos)
+        K = np.concatenate([np.asarray(saK, F64), k[None]], axis=0)
+        V = np.concatenate([np.asarray(saV, F64), v[None]], axis=0)
+        x = self.sa_block(e, q, K, V)
+        o_hat = self.ca_block(x, caK, caV)
+        ids, logp, z = self.head(o_hat, B)
+        return dict(x=x, o_hat=o_hat, ids=ids, logp=logp, k=k, v=v, z=z)
+
+
+# --------------------------------------------------------------------------
+# the dynamic draft tree (Section 2.2, last paragraph)
+# --------------------------------------------------------------------------
+class TreeState:
+    """Node pool of one sequence. Scores are fp32 sums of fp32 log-probs."""
+
+    def __init__(self, root_tok, B, D, m):
+        self.B, self.D, self.m = B, D, m
+        self.root_tok = int(root_tok)
+        self.tok, self.parent, self.depth = [], [], []   # parent: pool index or -1 (root)
+        self.score = []                                  # np.float32
+        self.step = 0
+        self.frontier = [-1]                             # pool indices; -1 = root
+
+    def frontier_tokens(self):
+        return [self.root_tok if f < 0 else self.tok[f] for f in self.frontier]
+
+    def path_to(self, node):
+        """Pool indices from the depth-1 ancestor down to node (root excluded)."""
+        path = []
+        while node >= 0:
+            path.append(node)
+            node = self.parent[node]
+        return path[::-1]
+
+
+def tree_expand(ts: TreeState, ids, logp):
+    """Append the children of the current frontier and choose the next one.
+
+    ids, logp: [len(frontier), B], each row sorted as lm_head_topk sorts. A
+    child's score is its parent's score plus its log-probability (fp32 add).
+    Children are appended in (frontier row, rank) order; the next frontier is
+    the top B of the new children by (score desc, pool index asc)."""
+    B = ts.B
+    logp = np.asarray(logp, np.float32)
+    first = len(ts.tok)
+    for r, f in enumerate(ts.frontier):
+        base = np.float32(0.0) if f < 0 else ts.score[f]
+        for j in range(B):
+            ts.tok.append(int(ids[r][j]))
+            ts.parent.append(f)
+            ts.depth.append(ts.step + 1)
+            ts.score.append(np.float32(base + logp[r][j]))
+    new = list(range(first, len(ts.tok)))
+    new.sort(key=lambda i: (-float(ts.score[i]), i))
+    ts.frontier = new[:B]
+    ts.step += 1
+
+
+def tree_finalize(ts: TreeState):
+    """Keep the min(m, pool) best nodes by (score desc, pool index asc), list
+    them by pool index, put the root in slot 0 and rewrite parents as slots.
+    Returns tok, parent, depth (int64 [n]) and score (float32 [n])."""
+    n_pool = len(ts.tok)
+    order = sorted(range(n_pool), key=lambda i: (-float(ts.score[i]), i))
+    kept = sorted(order[:min(ts.m, n_pool)])
+    slot = {-1: 0}
+    for s, i in enumerate(kept):
+        slot[i] = s + 1
+    tok = [ts.root_tok] + [ts.tok[i] for i in kept]
+    parent = [-1] + [slot[ts.parent[i]] for i in kept]
+    depth = [0] + [ts.depth[i] for i in kept]
+    score = [np.float32(0.0)] + [ts.score[i] for i in kept]
+    return (np.array(tok, np.int64), np.array(parent, np.int64),
+            np.array(depth, np.int64), np.array(score, np.float32))
+
+
+def tree_mask(parent):
+    """mask[i][j] = 1 iff j == i or j is an ancestor of i. parent[0] = -1."""
+    n = len(parent)
+    mask = np.zeros((n, n), np.uint8)
+    for i in range(n):
+        j = i
+        while j >= 0:
+            mask[i, j] = 1
+            j = int(parent[j])
+    return mask
+
+
+def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None):
+    """Grow one sequence's draft tree with D drafter forwards.
+
+    saK, saV [ctx, Hkv, dh]: self-attention prefix cache (positions 0..ctx-1);
+    the root sits at position ctx, a node of depth d at ctx + d, and sees the
+    prefix, its ancestors (root included) and itself.
+    forced: optional list of per-step (ids, logp) to expand with instead of
+    the oracle's own top-B (used to follow another implementation's choices).
+    Returns (TreeState, steps) with steps[s] = list of forward_row dicts."""
+    ctx = saK.shape[0]
+    ts = TreeState(root_tok, B, D, m)
+    node_kv = {}      # pool index (or -1) -> (k, v) of nodes that were forwarded
+    steps = []
+    for s in range(D):
+        rows = []
+        for f in ts.frontier:
+            # the root sees only the prefix; a node sees the root and its proper ancestors
+            anc = [] if f < 0 else [-1] + ts.path_to(f)[:-1]
+            Ks = [saK] + [node_kv[a][0][None] for a in anc]
+            Vs = [saV] + [node_kv[a][1][None] for a in anc]
+            tok = ts.root_tok if f < 0 else ts.tok[f]
+            out = dr.forward_row(tok, ctx + s, np.concatenate(Ks, 0), np.concatenate(Vs, 0), caK, caV, B)
+            rows.append(out)
+        for f, out in zip(ts.frontier, rows):
+            node_kv[f] = (out["k"], out["v"])
+        steps.append(rows)
+        if forced is not None:
+            ids, logp = forced[s]
+        else:
+            ids = [r["ids"] for r in rows]
+            logp = [r["logp"] for r in rows]
+        tree_expand(ts, ids, logp)
+    return ts, steps
+
+
+# --------------------------------------------------------------------------
+# independent loop-based paths used to pin the tree code by brute force
+# --------------------------------------------------------------------------
+def sequential_decode(dr: Drafter, prefix_toks, path_toks, caK, caV, B):
+    """Plain causal decoding, token by token (Algorithm 1, the inner drafting loop with the
+    tokens given): the self-attention cache grows by one entry per token and
+    every token sees all earlier ones. Returns the forward_row dict of each
+    token of path_toks."""
+    c = dr.c
+    K = np.zeros((0, c["sa_hkv"], c["head_dim"]), F64)
+    V = np.zeros((0, c["sa_hkv"], c["head_dim"]), F64)
+    pos = 0
+    for t in prefix_toks:
+        _, _, k, v = dr.sa_qkv(t, pos)
+        K = np.concatenate([K, k[None]], 0)
+        V = np.concatenate([V, v[None]], 0)
+        pos += 1
+    outs = []
+    for t in path_toks:
+        out = dr.forward_row(t, pos, K, V, caK, caV, B)
+        K = np.concatenate([K, out["k"][None]], 0)
+        V = np.concatenate([V, out["v"][None]], 0)
+        outs.append(out)
+        pos += 1
+    return outs
+
+
+def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft):
+    """Chain drafting (Algorithm 1, inner loop) with greedy choice: K_draft
+    tokens, each the most probable continuation. Returns (tokens, logps)."""
+    toks, lps = [int(root_tok)], []
+    for _ in range(K_draft):
+        out = sequential_decode(dr, prefix_toks, toks, caK, caV, 1)[-1]
+        toks.append(int(out["ids"][0]))
+        lps.append(float(out["logp"][0]))
+    return toks[1:], lps
