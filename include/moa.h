@@ -1,0 +1,165 @@
+/*
+ * moa.h -- C ABI of the Mixture-of-Attentions drafter hot path for one NVIDIA B200 (sm_100a).
+ *
+ * The library computes the drafter's forward step of "Mixture of Attentions for
+ * Speculative Decoding" (arXiv 2410.03804): Layer Self-Attention over each token's
+ * stack of per-layer LLM activations followed by a mean over layers (Section 3.1.1),
+ * causal / tree-masked self-attention over token embeddings and cross-attention into
+ * keys and values derived from the LSA output (Section 3.1.2, Algorithm 1), the LM head
+ * with log-softmax and the B most probable tokens (Eq. 1), and the EAGLE-2-style dynamic
+ * draft tree with its ancestor mask (Section 2.2). Target Layer Inference is fixed at
+ * TLI = 0 (Section 3.2): the drafter predicts the last decoder layer's activation.
+ *
+ * Conventions
+ *  - Every pointer is DEVICE memory owned by the caller unless its name ends in _host or
+ *    the comment says "host". The library allocates and frees no device memory.
+ *  - Matrices are row-major [out, in]; there are no biases. "T" below is the storage type
+ *    selected by moa_config.dtype (float or bfloat16); accumulation is always fp32.
+ *  - Every call enqueues work on `stream` (a cudaStream_t passed as void*) and returns
+ *    without synchronising. Results are valid once the caller has synchronised the stream.
+ *  - Arguments are validated on the host before anything is launched; on error a status is
+ *    returned and nothing is enqueued. No call throws, aborts or exits.
+ *  - All device base pointers must be 16-byte aligned.
+ *  - One moa_ctx may be used by one host thread at a time.
+ */
+#ifndef MOA_H_
+#define MOA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOA_MAX_BATCH 64      /* sequences per call */
+#define MOA_MAX_TOPK 16       /* tree breadth B */
+#define MOA_MAX_DEPTH 16      /* tree depth D */
+
+typedef struct moa_ctx moa_ctx; /* opaque, host side */
+
+typedef enum {
+  MOA_OK = 0,
+  MOA_ERR_NULL = 1,       /* a required pointer is NULL */
+  MOA_ERR_SHAPE = 2,      /* a dimension is out of range or inconsistent */
+  MOA_ERR_DTYPE = 3,
+  MOA_ERR_ALIGN = 4,      /* a device pointer is not 16-byte aligned */
+  MOA_ERR_WORKSPACE = 5,  /* workspace smaller than moa_state_bytes() reports */
+  MOA_ERR_CAPACITY = 6,   /* a cache or the node pool would overflow */
+  MOA_ERR_STATE = 7,      /* calls out of order (e.g. draft step before moa_tree_begin) */
+  MOA_ERR_ARCH = 8,       /* the current device is not compute capability 10.x */
+  MOA_ERR_CUDA = 9,       /* a CUDA runtime call failed; see moa_last_cuda_error() */
+  MOA_ERR_TIMEOUT = 10    /* a bounded device-side wait expired */
+} moa_status;
+
+typedef enum { MOA_F32 = 0, MOA_BF16 = 1 } moa_dtype;
+
+typedef struct {
+  int32_t d_model;   /* E: token embedding width = SA and CA width                         */
+  int32_t n_stack;   /* S: activations stacked per token (the LLM's layers) fed to LSA     */
+  int32_t d_stack;   /* D_in: width of one stacked activation = LSA width                  */
+  int32_t vocab;     /* V                                                                  */
+  int32_t head_dim;  /* dh, 64 or 128, shared by the three attentions                      */
+  int32_t lsa_hq, lsa_hkv, lsa_mlp; /* heads (query / key-value) and MLP width, LSA block  */
+  int32_t sa_hq, sa_hkv, sa_mlp;    /* ... self-attention block                            */
+  int32_t ca_hq, ca_hkv, ca_mlp;    /* ... cross-attention block                           */
+  int32_t max_batch; /* <= MOA_MAX_BATCH                                                   */
+  int32_t max_ctx;   /* capacity of the caches, in positions per sequence                  */
+  int32_t tree_topk; /* B <= MOA_MAX_TOPK                                                  */
+  int32_t tree_depth;/* D <= MOA_MAX_DEPTH: number of drafter forwards per tree            */
+  int32_t tree_keep; /* m: nodes kept for verification (the root is one more)              */
+  float rms_eps;       /* RMSNorm epsilon, added to the mean square                        */
+  float sa_rope_theta; /* rotary base of the self-attention; 0 disables the rotation       */
+  int32_t dtype;       /* moa_dtype of weights, activations and caches                     */
+} moa_config;
+
+typedef struct { /* device pointers of type T */
+  const void *embed, *lm_head, *final_norm;                 /* [V,E] [V,E] [E] */
+  const void *lsa_norm1, *lsa_wq, *lsa_wk, *lsa_wv, *lsa_wo; /* [D_in] [Hq*dh,D_in] [Hkv*dh,D_in] x2 [D_in,Hq*dh] */
+  const void *lsa_norm2, *lsa_wgate, *lsa_wup, *lsa_wdown;  /* [D_in] [F,D_in] [F,D_in] [D_in,F] */
+  const void *sa_norm1, *sa_wq, *sa_wk, *sa_wv, *sa_wo;     /* as above with E in place of D_in */
+  const void *sa_norm2, *sa_wgate, *sa_wup, *sa_wdown;
+  const void *ca_normq, *ca_normkv;                         /* [E] [D_in] */
+  const void *ca_wq, *ca_wk, *ca_wv, *ca_wo;                /* [Hq*dh,E] [Hkv*dh,D_in] x2 [E,Hq*dh] */
+  const void *ca_norm2, *ca_wgate, *ca_wup, *ca_wdown;
+} moa_weights;
+
+typedef struct {
+  void *ca_k, *ca_v;        /* T [max_batch, max_ctx, ca_hkv, head_dim]: cross-attention keys / values   */
+  void *sa_k, *sa_v;        /* T [max_batch, max_ctx, sa_hkv, head_dim]: rotated self-attention prefix   */
+  int32_t *ca_len, *sa_len; /* device int32 [max_batch]: valid positions; written only by the library    */
+  void *tree;               /* device blob of moa_state_bytes().tree_bytes: node pool, frontier, tree K/V */
+  int32_t *ca_len_host, *sa_len_host; /* HOST int32 [max_batch]: mirrors kept by the library             */
+  int32_t step;             /* HOST: draft steps done since moa_tree_begin, -1 before it; library-owned  */
+} moa_state;
+
+/* Creates a context for the CURRENT device. Copies config and weight pointers (not the weights).
+ * MOA_ERR_ARCH if the device is not compute capability 10.x: there is no fallback path. */
+moa_status moa_create(const moa_config *cfg, const moa_weights *w, moa_ctx **out);
+void moa_destroy(moa_ctx *ctx);
+
+/* Sizes in bytes of moa_state.tree and of the workspace every compute call needs.
+ * lsa_chunk_tokens (>= 1) is the number of tokens moa_lsa_forward processes per internal
+ * pass; a larger value needs a larger workspace. */
+moa_status moa_state_bytes(const moa_ctx *ctx, int32_t lsa_chunk_tokens, size_t *tree_bytes, size_t *workspace_bytes);
+
+const char *moa_status_str(moa_status s);
+const char *moa_last_cuda_error(void); /* text of the last CUDA error seen by this thread's calls */
+
+/* Sets the valid length of the caches of sequences 0..batch-1 (device and host copies), e.g. after
+ * the caller filled a cache itself or dropped rejected positions. which: 0 = ca, 1 = sa. */
+moa_status moa_state_set_len(moa_ctx *ctx, moa_state *st, int32_t which, const int32_t *len_host, int32_t batch, void *stream);
+
+/* Layer Self-Attention with mean, then the cross-attention key/value projection
+ * (Section 3.1.1; Algorithm 1: kv <- LSA_layer_with_mean(h), kv <- (kv, kv')).
+ *   h_stack    T [sum n_tok, S, D_in], sequences back to back
+ *   n_tok_host HOST int32 [batch], tokens of each sequence (may be 0)
+ *   kv_out     T [sum n_tok, D_in] or NULL: the LSA output rows
+ * Appends n_tok[b] rows W_k n(kv), W_v n(kv) to ca_k / ca_v of sequence b at position ca_len[b]
+ * and advances ca_len. MOA_ERR_CAPACITY if ca_len[b] + n_tok[b] > max_ctx. */
+moa_status moa_lsa_forward(moa_ctx *ctx, moa_state *st, const void *h_stack, const int32_t *n_tok_host, int32_t batch,
+                           void *kv_out, void *ws, size_t ws_bytes, void *stream);
+
+/* Self-attention prefix for prompt / accepted tokens (Section 3.1.2 "Self-Attention"): embeds the
+ * tokens, projects keys and values, rotates keys at positions sa_len[b], sa_len[b]+1, ... and
+ * appends them to sa_k / sa_v.   tok: device int32 [sum n], n_host: HOST int32 [batch]. */
+moa_status moa_sa_append(moa_ctx *ctx, moa_state *st, const int32_t *tok, const int32_t *n_host, int32_t batch,
+                         void *ws, size_t ws_bytes, void *stream);
+
+/* Starts a draft tree per sequence (Section 2.2). root_tok: device int32 [batch], the last verified
+ * token; it sits at position sa_len[b]. Sets st->step = 0. */
+moa_status moa_tree_begin(moa_ctx *ctx, moa_state *st, const int32_t *root_tok, int32_t batch, void *stream);
+
+/* One drafter forward for the current frontier (Algorithm 1, the SA_layer, CA_layer and LM_head
+ * steps of the inner loop; Eq. 1): R = batch rows at step 0 (the roots), batch*B afterwards, row
+ * b*B + r = r-th frontier node of sequence b. A row at depth d sits at position sa_len[b] + d and
+ * sees the prefix, its ancestors and itself.
+ *   topk_id    int32 [R, B]  token ids, by (log-probability descending, id ascending)
+ *   topk_logp  float [R, B]  their log-probabilities (logit - logsumexp over the vocabulary)
+ *   hidden_out T [R, E] or NULL: the drafter's output activation (input of the LM head) */
+moa_status moa_draft_step(moa_ctx *ctx, moa_state *st, int32_t batch, int32_t *topk_id, float *topk_logp,
+                          void *hidden_out, void *ws, size_t ws_bytes, void *stream);
+
+/* Expands the tree with the rows' top-B lists (Section 2.2): child score = parent score + logp
+ * (fp32), children appended in (row, rank) order, next frontier = top B children by (score
+ * descending, pool index ascending). Advances st->step. After the D-th expansion it also selects
+ * the m best pool nodes (same order), lists them by pool index behind the root (slot 0) and, if the
+ * out_* pointers are non-NULL, writes int32 / float [batch, m+1] arrays (parent = slot number,
+ * root's parent = -1; unused tail slots hold -1 / 0) and out_n [batch] = 1 + nodes kept. */
+moa_status moa_tree_expand(moa_ctx *ctx, moa_state *st, int32_t batch, const int32_t *topk_id, const float *topk_logp,
+                           int32_t *out_tok, int32_t *out_parent, int32_t *out_depth, float *out_score, int32_t *out_n,
+                           void *stream);
+
+/* Tree Attention mask (Section 2.2, verification with Tree Attention): mask[b][i][j] = 1 iff j == i or
+ * j is an ancestor of i. parent: device int32 [batch, n] with parent[0] = -1 and parent[i] < i; an
+ * entry < 0 at i > 0 marks an unused slot (its row is zero).
+ * packed = 0: uint8 [batch, n, n]; packed = 1: uint64 [batch, n, ceil(n/64)], bit j%64 of word j/64. */
+moa_status moa_tree_attn_mask(const int32_t *parent, int32_t batch, int32_t n, void *mask_out, int32_t packed, void *stream);
+
+/* Reads back the device status word kept in st->tree (0 = no device-side problem seen). Synchronises the stream. */
+moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOA_H_ */

@@ -1,0 +1,366 @@
+// Generic kernels of the drafter forward: normalisation, an FMA GEMM for the fp32 path and for
+// shapes the tensor-core kernels do not take, rotary embedding + cache writes, a plain attention
+// row kernel, SwiGLU glue, layer mean, and a row-wise logsumexp + top-B over stored logits.
+#pragma once
+#include "moa_common.cuh"
+
+namespace moa {
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm (pre-norm of every attention / MLP): y = x * g / sqrt(mean(x^2) + eps).
+// One block per row. Input either gathered from the embedding table (tok != nullptr) or read from
+// x[row]. Optionally also writes the un-normalised row in fp32 (the residual stream).
+// ---------------------------------------------------------------------------------------------
+template <typename TIN, typename T>
+__global__ void rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok, int vocab,
+                                    const T* __restrict__ gain, int K, float eps,
+                                    float* __restrict__ res_out, T* __restrict__ y) {
+  __shared__ float red[33];
+  const int r = blockIdx.x;
+  const TIN* xr;
+  if (tok != nullptr) {
+    int t = tok[r];
+    t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+    xr = x + (size_t)t * K;
+  } else {
+    xr = x + (size_t)r * K;
+  }
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    float v = to_f<TIN>(xr[k]);
+    ss += v * v;
+  }
+  ss = block_sum(ss, red);
+  const float rinv = rsqrtf(ss / (float)K + eps);
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    float v = to_f<TIN>(xr[k]);
+    if (res_out) res_out[(size_t)r * K + k] = v;
+    y[(size_t)r * K + k] = from_f<T>(v * rinv * to_f<T>(gain[k]));
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// C[R, N] (fp32, leading dimension ldc) = A[R, K] * W[N, K]^T (+ res[R, N] with leading dim ldr).
+// Classic 64x64x16 shared-memory tiling, 256 threads, 4x4 outputs per thread, fp32 FMA.
+// K must be a multiple of 16.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_fma_kernel(const T* __restrict__ A, const T* __restrict__ W,
+                                                       int R, int N, int K, const float* res, int ldr,
+                                                       float* C, int ldc) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Ws[16][64 + 4];
+  const int tid = threadIdx.x;
+  const int n0 = blockIdx.x * 64, r0 = blockIdx.y * 64;
+  const int lrow = tid >> 2, lk = (tid & 3) * 4;   // loader: 64 rows x 4 groups of 4 k
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    {
+      const int ar = r0 + lrow;
+      const int wn = n0 + lrow;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        As[lk + j][lrow] = ar < R ? to_f<T>(A[(size_t)ar * K + k0 + lk + j]) : 0.f;
+        Ws[lk + j][lrow] = wn < N ? to_f<T>(W[(size_t)wn * K + k0 + lk + j]) : 0.f;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float a[4], w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[j] = Ws[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + ty * 4 + i;
+    if (r >= R) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= N) continue;
+      float v = acc[i][j];
+      if (res) v += res[(size_t)r * ldr + n];
+      C[(size_t)r * ldc + n] = v;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// fp32 -> T, flat.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void cast_flat_kernel(const float* __restrict__ x, T* __restrict__ y, size_t total) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) y[i] = from_f<T>(x[i]);
+}
+
+// h = silu(gate) * up, fp32 in (two column blocks of one buffer), T out.
+template <typename T>
+__global__ void silu_mul_kernel(const float* __restrict__ gate, const float* __restrict__ up, int ld, int F,
+                                T* __restrict__ h, size_t total) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  size_t r = i / F;
+  int c = (int)(i - r * F);
+  float g = gate[r * ld + c], u = up[r * ld + c];
+  h[i] = from_f<T>(g / (1.f + __expf(-g)) * u);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rotary embedding + stores. One block per row.
+//   q (optional): fp32 [R, hq*dh] at qkv + q_off (leading dim ld) -> rotated, T [R, hq*dh]
+//   k, v: fp32 [R, hkv*dh] -> k rotated; written as T to  kdst/vdst + dst_index(row) * hkv*dh
+// Row r sits at position pos_base[seq(r)] + pos_add(r). Angles are formed in double:
+// angle = pos * theta^(-2i/dh), element i paired with i + dh/2. theta == 0: no rotation.
+// mode 0 (draft rows): seq = step0 ? r : r / B; pos_add = step; dst = seq * slots + self_slot
+// mode 1 (prefix append): seq from split; i = r - off[seq]; pos_add = i; dst = seq * max_ctx + len + i
+// ---------------------------------------------------------------------------------------------
+struct RopeRows {
+  int mode;
+  int step, B, slots;      // mode 0
+  int max_ctx;             // mode 1
+  SeqSplit split;          // mode 1 (rows are relative to row0)
+  int row0;
+};
+
+template <typename T>
+__global__ void rope_store_kernel(const float* __restrict__ qkv, int ld, int q_off, int k_off, int v_off,
+                                  int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
+                                  RopeRows rr, T* __restrict__ qdst, T* __restrict__ kdst, T* __restrict__ vdst) {
+  __shared__ float cs[64], sn[64];
+  const int r = blockIdx.x;
+  int seq, pos_add;
+  size_t dst;
+  if (rr.mode == 0) {
+    seq = rr.step == 0 ? r : r / rr.B;
+    pos_add = rr.step;
+    const int slot = rr.step == 0 ? 0 : 1 + (rr.step - 1) * rr.B + (r % rr.B);
+    dst = (size_t)seq * rr.slots + slot;
+  } else {
+    const int t = rr.row0 + r;
+    seq = rr.split.seq_of(t);
+    pos_add = t - rr.split.off[seq];
+    dst = (size_t)seq * rr.max_ctx + pos_base[seq] + pos_add;
+  }
+  const int pos = pos_base[seq] + pos_add;
+  const int half = dh >> 1;
+  if (threadIdx.x < half) {
+    if (theta == 0.f) {
+      cs[threadIdx.x] = 1.f;
+      sn[threadIdx.x] = 0.f;
+    } else {
+      const double inv = exp2(-2.0 * (double)threadIdx.x / (double)dh * log2((double)theta));
+      double s, c;
+      sincos((double)pos * inv, &s, &c);
+      cs[threadIdx.x] = (float)c;
+      sn[threadIdx.x] = (float)s;
+    }
+  }
+  __syncthreads();
+  const float* row = qkv + (size_t)r * ld;
+  if (qdst) {
+    for (int i = threadIdx.x; i < hq * half; i += blockDim.x) {
+      const int h = i / half, j = i - h * half;
+      const float x1 = row[q_off + h * dh + j], x2 = row[q_off + h * dh + half + j];
+      qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
+      qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+    }
+  }
+  for (int i = threadIdx.x; i < hkv * half; i += blockDim.x) {
+    const int h = i / half, j = i - h * half;
+    const float x1 = row[k_off + h * dh + j], x2 = row[k_off + h * dh + half + j];
+    kdst[dst * hkv * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
+    kdst[dst * hkv * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+  }
+  for (int i = threadIdx.x; i < hkv * dh; i += blockDim.x) vdst[dst * hkv * dh + i] = from_f<T>(row[v_off + i]);
+}
+
+// Cross-attention cache append: fp32 [n, hkv*dh] k and v rows -> T cache rows at (seq, ca_len[seq] + i).
+template <typename T>
+__global__ void cache_append_kernel(const float* __restrict__ kv, int ld, int k_off, int v_off, int width,
+                                    const int* __restrict__ len, int max_ctx, SeqSplit split, int row0,
+                                    T* __restrict__ kdst, T* __restrict__ vdst) {
+  const int r = blockIdx.x;
+  const int t = row0 + r;
+  const int seq = split.seq_of(t);
+  const int i = t - split.off[seq];
+  const size_t dst = ((size_t)seq * max_ctx + len[seq] + i) * width;
+  for (int c = threadIdx.x; c < width; c += blockDim.x) {
+    kdst[dst + c] = from_f<T>(kv[(size_t)r * ld + k_off + c]);
+    vdst[dst + c] = from_f<T>(kv[(size_t)r * ld + v_off + c]);
+  }
+}
+
+__global__ void add_len_kernel(int* len, SeqSplit split) {
+  const int b = threadIdx.x;
+  if (b < split.n_seq) len[b] += split.off[b + 1] - split.off[b];
+}
+struct LenVals { int n; int v[64]; };
+__global__ void set_len_kernel(int* len, LenVals lv) {
+  const int b = threadIdx.x;
+  if (b < lv.n) len[b] = lv.v[b];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention, one block (4 warps) per (query row, query head): softmax(q K^T / sqrt(dh)) V in fp32.
+// Key set = segment A: keys 0..nA-1 of sequence `seq` in a cache [n_seq, capA, hkv, dh]
+//         + segment B: nB listed slots of a second cache [n_seq, capB, hkv, dh] (tree nodes).
+// Row -> sequence: seq = r / rows_per_seq. nA = lenA ? lenA[seq] : nA_fixed.
+// Each warp walks keys warp, warp+4, ...; a lane owns dh/32 consecutive elements.
+// ---------------------------------------------------------------------------------------------
+template <typename T, int DH>
+__global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q, int hq, int hkv,
+                                                        const T* __restrict__ kA, const T* __restrict__ vA, int capA,
+                                                        const int* __restrict__ lenA, int nA_fixed,
+                                                        const T* __restrict__ kB, const T* __restrict__ vB, int capB,
+                                                        const int* __restrict__ slotsB, int slots_ld, int nB,
+                                                        int rows_per_seq, T* __restrict__ out) {
+  constexpr int VEC = DH / 32;
+  __shared__ float s_m[4], s_l[4], s_acc[4][DH];
+  const int r = blockIdx.x, h = blockIdx.y;
+  const int g = h / (hq / hkv);
+  const int seq = r / rows_per_seq;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nA = lenA ? lenA[seq] : nA_fixed;
+  const float scale = rsqrtf((float)DH);
+  float qv[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) qv[e] = to_f<T>(q[((size_t)r * hq + h) * DH + lane * VEC + e]) * scale;
+  float m = -INFINITY, l = 0.f, acc[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+  const int n = nA + nB;
+  for (int j = warp; j < n; j += 4) {
+    const T *kp, *vp;
+    if (j < nA) {
+      const size_t o = (((size_t)seq * capA + j) * hkv + g) * DH + lane * VEC;
+      kp = kA + o;
+      vp = vA + o;
+    } else {
+      const int slot = slotsB[(size_t)r * slots_ld + (j - nA)];
+      const size_t o = (((size_t)seq * capB + slot) * hkv + g) * DH + lane * VEC;
+      kp = kB + o;
+      vp = vB + o;
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) s = fmaf(qv[e], to_f<T>(kp[e]), s);
+    s = warp_sum(s);
+    const float mn = fmaxf(m, s);
+    const float corr = __expf(m - mn);     // m = -inf at the first key: exp(-inf) = 0
+    const float p = __expf(s - mn);
+    l = l * corr + p;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = acc[e] * corr + p * to_f<T>(vp[e]);
+    m = mn;
+  }
+  if (lane == 0) { s_m[warp] = m; s_l[warp] = l; }
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) s_acc[warp][lane * VEC + e] = acc[e];
+  __syncthreads();
+  if (warp == 0) {
+    float M = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+    float L = 0.f, o[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) o[e] = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float c = s_m[w] == -INFINITY ? 0.f : __expf(s_m[w] - M);
+      L += s_l[w] * c;
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) o[e] += s_acc[w][lane * VEC + e] * c;
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) out[((size_t)r * hq + h) * DH + lane * VEC + e] = from_f<T>(o[e] * inv);
+  }
+}
+
+// kv[t, :] = mean over the S layer rows of Z[t, s, :] (fp32 in; fp32 and optional T out).
+template <typename T>
+__global__ void mean_layers_kernel(const float* __restrict__ Z, int S, int D, float* __restrict__ kvf,
+                                   T* __restrict__ kv_out) {
+  const int t = blockIdx.x;
+  for (int c = threadIdx.x; c < D; c += blockDim.x) {
+    float s = 0.f;
+    for (int l = 0; l < S; ++l) s += Z[((size_t)t * S + l) * D + c];
+    s *= 1.f / (float)S;
+    kvf[(size_t)t * D + c] = s;
+    if (kv_out) kv_out[(size_t)t * D + c] = from_f<T>(s);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row-wise log-softmax top-B over stored logits z[R, V] (fp32): lse = max + log(sum exp(z - max)),
+// then B rounds of block arg-max in the order (value descending, id ascending).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {   // (va, ia) ranks before (vb, ib)
+  return va > vb || (va == vb && ia < ib);
+}
+
+__global__ void __launch_bounds__(256) lse_topk_rows_kernel(const float* __restrict__ z, int V, int B,
+                                                            int* __restrict__ ids, float* __restrict__ logp) {
+  __shared__ float red[33];
+  __shared__ float s_v[8];
+  __shared__ int s_i[8];
+  __shared__ float pick_v;
+  __shared__ int pick_i;
+  const int r = blockIdx.x;
+  const float* zr = z + (size_t)r * V;
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) mx = fmaxf(mx, zr[i]);
+  mx = block_max(mx, red);
+  float se = 0.f;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) se += expf(zr[i] - mx);
+  se = block_sum(se, red);
+  const float lse = mx + logf(se);
+  float pv = INFINITY;
+  int pi = -1;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (int b = 0; b < B; ++b) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+      const float v = zr[i];
+      if (better(pv, pi, v, i) && better(v, i, bv, bi)) { bv = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) { s_v[wid] = bv; s_i[wid] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float fv = s_v[0];
+      int fi = s_i[0];
+      for (int w = 1; w < 8; ++w)
+        if (better(s_v[w], s_i[w], fv, fi)) { fv = s_v[w]; fi = s_i[w]; }
+      pick_v = fv;
+      pick_i = fi;
+      ids[(size_t)r * B + b] = fi == 0x7fffffff ? -1 : fi;
+      logp[(size_t)r * B + b] = fv - lse;
+    }
+    __syncthreads();
+    pv = pick_v;
+    pi = pick_i;
+  }
+}
+
+}  // namespace moa
