@@ -27,6 +27,16 @@ LSA or CA; the LLM's final RMSNorm gain precedes the LM head; the MLP listed
 probabilities are sums of fp32 log-probabilities. Ties break towards the
 smaller index everywhere.
 
+Storage precision: with store="bf16" every tensor that the method keeps in
+the 16-bit storage type between two matrix products is rounded to bfloat16
+(round to nearest even) at that point -- normalised activations entering a
+projection, projected q / k / v, attention outputs, the gated MLP hidden
+vector, cache entries and the reported LSA / drafter outputs; the residual
+stream and all sums stay in full precision, as "16-bit storage, softmax and
+accumulation in higher precision" (Section 4) implies. Top-B decisions are
+compared in this mode, so that both sides decide in the same precision;
+values are compared against the unrounded mode (store=None).
+
 Parity status: every function below is pinned by tests/test_oracle_pins.py
 against closed forms, library routines, brute force or invariants. The model's
 outputs are NOT pinned against the authors' trained system (no worked example,
@@ -67,9 +77,9 @@ def linear(x, w):
     return np.matmul(np.asarray(x, F64), np.asarray(w, F64).T)
 
 
-def swiglu_mlp(u, w_gate, w_up, w_down):
-    """W_down (silu(W_gate u) * (W_up u))."""
-    return linear(silu(linear(u, w_gate)) * linear(u, w_up), w_down)
+def swiglu_mlp(u, w_gate, w_up, w_down, rnd=lambda t: t):
+    """W_down (silu(W_gate u) * (W_up u)); rnd rounds the gated hidden vector (a stored tensor)."""
+    return linear(rnd(silu(linear(u, w_gate)) * linear(u, w_up)), w_down)
 
 
 def attend(q, K, V):
@@ -106,13 +116,22 @@ def rope(x, pos, theta):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
-def lm_head_topk(o_hat, final_norm, w_lm, eps, B):
+def round_bf16(x):
+    """Round to the nearest bfloat16 (ties to even), returned as float64."""
+    x32 = np.ascontiguousarray(np.asarray(x, np.float32))
+    bits = x32.view(np.uint32)
+    lsb = (bits >> np.uint32(16)) & np.uint32(1)
+    rounded = (bits + np.uint32(0x7FFF) + lsb) & np.uint32(0xFFFF0000)
+    return rounded.view(np.float32).astype(F64).reshape(np.shape(x))
+
+
+def lm_head_topk(o_hat, final_norm, w_lm, eps, B, rnd=lambda t: t):
     """LM head, log-softmax and the B most probable tokens (Eq. 1; Section 2.2).
 
     z = W_lm n(o_hat; g_final); logp = z - logsumexp(z).
     Order: log-probability descending, token id ascending on equality.
     Returns (ids [B] int64, logp [B] float64, z [V] float64)."""
-    z = linear(rmsnorm(o_hat, final_norm, eps), w_lm)
+    z = linear(rnd(rmsnorm(o_hat, final_norm, eps)), w_lm)
     zmax = np.max(z)
     lse = zmax + np.log(np.sum(np.exp(z - zmax)))
     logp = z - lse
@@ -131,10 +150,12 @@ class Drafter:
     weights: mapping name -> array [out, in] (any float dtype; widened to fp64
     where used)."""
 
-    def __init__(self, cfg, weights, cache_f64=True):
+    def __init__(self, cfg, weights, cache_f64=True, store=None):
         self.c = dict(cfg)
         self.w_raw = weights
         self._cache = {} if cache_f64 else None
+        assert store in (None, "bf16")
+        self.rnd = round_bf16 if store == "bf16" else (lambda t: t)
 
     def w(self, name):
         if self._cache is None:
@@ -153,19 +174,23 @@ class Drafter:
         S = X.shape[0]
         dh, hq, hkv = c["head_dim"], c["lsa_hq"], c["lsa_hkv"]
         X = np.asarray(X, F64)
-        U = rmsnorm(X, self.w("lsa_norm1"), c["rms_eps"])
-        Q = linear(U, self.w("lsa_wq")).reshape(S, hq, dh)
-        K = linear(U, self.w("lsa_wk")).reshape(S, hkv, dh)
-        V = linear(U, self.w("lsa_wv")).reshape(S, hkv, dh)
+        rnd = self.rnd
+        U = rnd(rmsnorm(X, self.w("lsa_norm1"), c["rms_eps"]))
+        Q = rnd(linear(U, self.w("lsa_wq"))).reshape(S, hq, dh)
+        K = rnd(linear(U, self.w("lsa_wk"))).reshape(S, hkv, dh)
+        V = rnd(linear(U, self.w("lsa_wv"))).reshape(S, hkv, dh)
         O = np.zeros((S, hq, dh), F64)
         for h in range(hq):
             g = kv_head_of(h, hq, hkv)
             for s in range(S):
                 O[s, h] = attend(Q[s, h], K[:, g], V[:, g])
-        Y = X + linear(O.reshape(S, hq * dh), self.w("lsa_wo"))
-        Z = Y + swiglu_mlp(rmsnorm(Y, self.w("lsa_norm2"), c["rms_eps"]),
-                           self.w("lsa_wgate"), self.w("lsa_wup"), self.w("lsa_wdown"))
+        Y = X + linear(rnd(O).reshape(S, hq * dh), self.w("lsa_wo"))
+        Z = Y + self.mlp(rnd(rmsnorm(Y, self.w("lsa_norm2"), c["rms_eps"])), "lsa")
         return Z
+
+    def mlp(self, u, block):
+        """SwiGLU MLP of one block; the gated hidden vector is a stored tensor."""
+        return swiglu_mlp(u, self.w(block + "_wgate"), self.w(block + "_wup"), self.w(block + "_wdown"), self.rnd)
 
     def lsa_token(self, X):
         """LSA followed by the mean aggregation over the layer axis: [S, D_in] -> [D_in]."""
@@ -182,10 +207,10 @@ class Drafter:
         """K_c = W_k n(kv), V_c = W_v n(kv): one row per context position.
         kv [n, D_in] -> K_c, V_c [n, Hkv, dh]."""
         c = self.c
-        u = rmsnorm(kv, self.w("ca_normkv"), c["rms_eps"])
+        u = self.rnd(rmsnorm(kv, self.w("ca_normkv"), c["rms_eps"]))
         n = u.shape[0]
-        return (linear(u, self.w("ca_wk")).reshape(n, c["ca_hkv"], c["head_dim"]),
-                linear(u, self.w("ca_wv")).reshape(n, c["ca_hkv"], c["head_dim"]))
+        return (self.rnd(linear(u, self.w("ca_wk"))).reshape(n, c["ca_hkv"], c["head_dim"]),
+                self.rnd(linear(u, self.w("ca_wv"))).reshape(n, c["ca_hkv"], c["head_dim"]))
 
     # ---- Self-attention (Section 3.1.2, "Self-Attention") -----------------
     def sa_qkv(self, tok, pos):
@@ -194,10 +219,10 @@ class Drafter:
         c = self.c
         dh = c["head_dim"]
         e = np.asarray(self.w_raw["embed"][int(tok)], F64)
-        u = rmsnorm(e, self.w("sa_norm1"), c["rms_eps"])
-        q = rope(linear(u, self.w("sa_wq")).reshape(c["sa_hq"], dh), pos, c["rope_theta"])
-        k = rope(linear(u, self.w("sa_wk")).reshape(c["sa_hkv"], dh), pos, c["rope_theta"])
-        v = linear(u, self.w("sa_wv")).reshape(c["sa_hkv"], dh)
+        u = self.rnd(rmsnorm(e, self.w("sa_norm1"), c["rms_eps"]))
+        q = self.rnd(rope(linear(u, self.w("sa_wq")).reshape(c["sa_hq"], dh), pos, c["rope_theta"]))
+        k = self.rnd(rope(linear(u, self.w("sa_wk")).reshape(c["sa_hkv"], dh), pos, c["rope_theta"]))
+        v = self.rnd(linear(u, self.w("sa_wv")).reshape(c["sa_hkv"], dh))
         return e, q, k, v
 
     def sa_block(self, e, q, K, V):
@@ -210,9 +235,8 @@ class Drafter:
         for h in range(hq):
             g = kv_head_of(h, hq, hkv)
             o[h] = attend(q[h], K[:, g], V[:, g])
-        a = e + linear(o.reshape(hq * dh), self.w("sa_wo"))
-        return a + swiglu_mlp(rmsnorm(a, self.w("sa_norm2"), c["rms_eps"]),
-                              self.w("sa_wgate"), self.w("sa_wup"), self.w("sa_wdown"))
+        a = e + linear(self.rnd(o).reshape(hq * dh), self.w("sa_wo"))
+        return a + self.mlp(self.rnd(rmsnorm(a, self.w("sa_norm2"), c["rms_eps"])), "sa")
 
     # ---- Cross-attention block (Section 3.1.2; Algorithm 1, CA_layer step) -------
     def ca_block(self, x, K_c, V_c):
@@ -220,17 +244,16 @@ class Drafter:
         K_c, V_c [n, Hkv, dh]; no mask at generation time, no positional term."""
         c = self.c
         hq, hkv, dh = c["ca_hq"], c["ca_hkv"], c["head_dim"]
-        qc = linear(rmsnorm(x, self.w("ca_normq"), c["rms_eps"]), self.w("ca_wq")).reshape(hq, dh)
+        qc = self.rnd(linear(self.rnd(rmsnorm(x, self.w("ca_normq"), c["rms_eps"])), self.w("ca_wq"))).reshape(hq, dh)
         o = np.zeros((hq, dh), F64)
         for h in range(hq):
             g = kv_head_of(h, hq, hkv)
             o[h] = attend(qc[h], K_c[:, g], V_c[:, g])
-        cc = x + linear(o.reshape(hq * dh), self.w("ca_wo"))
-        return cc + swiglu_mlp(rmsnorm(cc, self.w("ca_norm2"), c["rms_eps"]),
-                               self.w("ca_wgate"), self.w("ca_wup"), self.w("ca_wdown"))
+        cc = x + linear(self.rnd(o).reshape(hq * dh), self.w("ca_wo"))
+        return cc + self.mlp(self.rnd(rmsnorm(cc, self.w("ca_norm2"), c["rms_eps"])), "ca")
 
     def head(self, o_hat, B):
-        return lm_head_topk(o_hat, self.w("final_norm"), self.w("lm_head"), self.c["rms_eps"], B)
+        return lm_head_topk(o_hat, self.w("final_norm"), self.w("lm_head"), self.c["rms_eps"], B, self.rnd)
 
     # ---- prefix of the self-attention cache -------------------------------
     def sa_prefix(self, toks, start=0):

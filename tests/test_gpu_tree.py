@@ -28,7 +28,7 @@ def test_tree_expand_and_finalize_bit_exact(B, D, m, batch):
     for s in range(D):
         R = batch * (1 if s == 0 else B)
         lp = -np.sort(rng.exponential(1.0, (R, B)), axis=-1).astype(np.float32)
-        if s == 2:
+        if s == 2 and B > 1:
             lp[:, 1] = lp[:, 0]                    # exact ties inside a row
             lp[-1] = lp[0]                         # and across rows
         ids = rng.integers(0, 1024, (R, B)).astype(np.int32)

@@ -93,6 +93,29 @@ def test_silu_and_mlp_special_cases():
     assert np.allclose(out, [0, 0, 0, want], atol=1e-15)
 
 
+def test_round_bf16_against_library_and_by_hand():
+    x = np.concatenate([RNG.standard_normal(4000) * 10.0 ** RNG.integers(-6, 6, 4000), [0.0, -0.0, 1.0, 65504.0]])
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(O.round_bf16(x), want)
+    assert O.round_bf16(1 + 2.0 ** -8) == 1.0                    # tie -> even mantissa
+    assert O.round_bf16(1 + 3 * 2.0 ** -8) == 1 + 2.0 ** -6      # tie -> even mantissa, upwards
+    assert O.round_bf16(1 + 2.0 ** -8 + 2.0 ** -20) == 1 + 2.0 ** -7
+    assert O.round_bf16(np.ones((2, 3))).shape == (2, 3)
+
+
+def test_bf16_storage_mode_is_a_small_perturbation():
+    c = tiny_cfg()
+    w = {k: O.round_bf16(v) for k, v in tiny_weights(c).items()}
+    H = O.round_bf16(RNG.standard_normal((2, c["n_stack"], c["d_stack"])))
+    a = O.Drafter(c, w).lsa_forward(H)
+    b = O.Drafter(c, w, store="bf16").lsa_forward(H)
+    rel = np.max(np.abs(a - b)) / np.max(np.abs(a))
+    assert 0 < rel < 2e-2
+    # stored tensors are exactly representable in bfloat16
+    Kc, Vc = O.Drafter(c, w, store="bf16").ca_kv(b)
+    assert np.array_equal(O.round_bf16(Kc), Kc) and np.array_equal(O.round_bf16(Vc), Vc)
+
+
 def test_linear_orientation():
     # W[n, k] with a single one routes x[k] to y[n]: catches a transposed operand
     w = np.zeros((3, 5)); w[2, 4] = 1.0
