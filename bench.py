@@ -1,0 +1,319 @@
+#!/usr/bin/env python
+"""Benchmark of the Mixture-of-Attentions drafter hot path on B200.
+
+One "step" of this benchmark is one drafting cycle over one batch of synthetic input: LSA on the newly
+accepted tokens + self-attention prefix append + D drafter forwards with tree expansion + the final
+top-m cut + the tree-attention mask. The headline metric is draft-tree steps per second (D drafter
+forwards per cycle); drafted tokens per second (m kept nodes per cycle) rides along.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload c2|c4|c5|c1]
+
+Prints ONE JSON line. With --impl reference it times the CPU oracle (a deliberately plain program) on a
+bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+CFG_KEYS = ("d_model", "n_stack", "d_stack", "vocab", "head_dim", "lsa_hq", "lsa_hkv", "lsa_mlp", "sa_hq", "sa_hkv",
+            "sa_mlp", "ca_hq", "ca_hkv", "ca_mlp", "tree_topk", "tree_depth", "tree_keep", "rms_eps", "rope_theta",
+            "dtype")
+
+
+def algorithmic_bytes(p) -> dict:
+    """Bytes one steady-state draft step must move: every weight once, every cache entry once per sequence."""
+    e = 4 if p.dtype == "f32" else 2
+    dh, E = p.head_dim, p.d_model
+    sa_w = (p.sa_hq + 2 * p.sa_hkv) * dh * E + E * p.sa_hq * dh + 3 * E * p.sa_mlp
+    ca_w = p.ca_hq * dh * E + E * p.ca_hq * dh + 3 * E * p.ca_mlp
+    lm = p.vocab * E
+    caches = p.batch * p.ctx * 2 * (p.sa_hkv + p.ca_hkv) * dh
+    lsa_w = ((p.lsa_hq + 2 * p.lsa_hkv) * dh * p.d_stack + p.d_stack * p.lsa_hq * dh + 3 * p.d_stack * p.lsa_mlp
+             + 2 * p.ca_hkv * dh * p.d_stack)
+    lsa_in = p.batch * p.lsa_tokens * p.n_stack * p.d_stack
+    return dict(step=(sa_w + ca_w + lm + caches) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms",
+                                          "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CPU oracle, timed on a bounded sample (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------------
+def oracle_sample(p, rows: int = 2, lsa_tok: int = 1):
+    """Times `lsa_tok` LSA tokens and `rows` drafter forward rows of the workload on the host cores and
+    scales them to one drafting cycle. Returns (cycle_seconds_estimate, cores, description)."""
+    import numpy as np
+    import torch
+    from oracle import moa_oracle as O
+    from paper_2410_03804_b200 import synth
+
+    cores = torch.get_num_threads()
+    w = synth.make_weights(p)
+    cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
+    dr = O.Drafter(cfg, {k: v.float().numpy() for k, v in w.items()})
+    for name in w:                       # widen the weights once: set-up, like loading a checkpoint
+        dr.w(name)
+    ctx = min(p.ctx, 2048)
+    caK, caV = synth.make_cache(synth.scaled(p, batch=1), "ca", ctx)
+    saK, saV = synth.make_cache(synth.scaled(p, batch=1), "sa", ctx)
+    caK, caV, saK, saV = [t[0].float().numpy().astype(np.float64) for t in (caK, caV, saK, saV)]
+    h = synth.make_h_stack(p, lsa_tok).float().numpy()
+    t0 = time.perf_counter()
+    dr.lsa_forward(h)
+    t_lsa = (time.perf_counter() - t0) / lsa_tok
+    toks = synth.make_root(synth.scaled(p, batch=rows)).tolist()
+    t0 = time.perf_counter()
+    for t in toks:
+        dr.forward_row(t, ctx, saK, saV, caK, caV, p.tree_topk)
+    t_row = (time.perf_counter() - t0) / rows
+    n_rows = p.batch * (1 + p.tree_topk * (p.tree_depth - 1))
+    cycle = p.batch * p.lsa_tokens * t_lsa + n_rows * t_row
+    what = (f"{lsa_tok} LSA token(s) ({t_lsa:.2f} s each) + {rows} drafter forward rows ({t_row:.2f} s each) of {p.name}"
+            f" with {ctx}-entry caches, scaled to one cycle = {p.batch * p.lsa_tokens} LSA tokens + {n_rows} rows;"
+            f" weights widened to fp64 beforehand")
+    return cycle, cores, what
+
+
+def run_reference(args, p):
+    t_all = []
+    for _ in range(args.warmup + args.steps):
+        cycle, cores, what = oracle_sample(p, rows=1, lsa_tok=1)
+        t_all.append(cycle)
+    t = statistics.mean(t_all[args.warmup:]) if len(t_all) > args.warmup else t_all[-1]
+    D, m = p.tree_depth, p.tree_keep
+    val = D / t
+    line = {"impl": "reference", "metric": "draft_tree_steps_per_sec", "value": val, "unit": "steps/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(p),
+            "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "drafted_tokens_per_sec": p.batch * m / t}
+    print(json.dumps(line))
+
+
+def workload_config(p):
+    return {"workload": f"{p.name}: Llama-3-shaped MoA drafter, one drafting cycle = LSA on {p.lsa_tokens} tokens/seq + "
+                        f"SA append + {p.tree_depth} drafter forwards (tree top-{p.tree_topk}, keep {p.tree_keep}) + mask",
+            "batch": p.batch, "context": p.ctx, "d_model": p.d_model, "vocab": p.vocab, "n_stack": p.n_stack,
+            "l2": "inputs larger than L2 (weights streamed per step exceed 126 MB)" if p.name != "c1" else "L2-resident"}
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CUDA path
+# ---------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
+
+    from paper_2410_03804_b200 import synth
+    p = synth.PRESETS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, p)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_03804_b200 import moa
+
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local)
+    # Replicas only: the path does not shard (one sequence batch per GPU, no data-path collective).
+    w = {k: v.to(dev) for k, v in synth.make_weights(p).items()}
+    cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
+    max_ctx = p.ctx + 64
+    g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens)
+    caK, caV = synth.make_cache(p, "ca")
+    saK, saV = synth.make_cache(p, "sa")
+    g.fill_cache("ca", caK.to(dev), caV.to(dev))
+    g.fill_cache("sa", saK.to(dev), saV.to(dev))
+    del caK, caV, saK, saV
+    nb, A, D, B, m = p.batch, p.lsa_tokens, p.tree_depth, p.tree_topk, p.tree_keep
+    h_host = synth.make_h_stack(p, nb * A).pin_memory()
+    tok_host = synth.make_tokens(p, A).reshape(-1).contiguous().pin_memory()
+    root_host = synth.make_root(p).pin_memory()
+    h_dev, tok_dev, root_dev = h_host.to(dev), tok_host.to(dev), root_host.to(dev)
+    h_stage, tok_stage, root_stage = torch.empty_like(h_dev), torch.empty_like(tok_dev), torch.empty_like(root_dev)
+    W = m + 1
+    ids_buf = torch.empty((nb * B, B), dtype=torch.int32, device=dev)
+    lp_buf = torch.empty((nb * B, B), dtype=torch.float32, device=dev)
+    outs = (torch.empty((nb, W), dtype=torch.int32, device=dev), torch.empty((nb, W), dtype=torch.int32, device=dev),
+            torch.empty((nb, W), dtype=torch.int32, device=dev), torch.empty((nb, W), dtype=torch.float32, device=dev),
+            torch.empty((nb,), dtype=torch.int32, device=dev))
+    host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in outs]
+    mask_host = torch.empty((nb, W, W), dtype=torch.uint8).pin_memory()
+    lens = [p.ctx] * nb
+
+    def cycle(h, tok, root):
+        g.moa_state_set_len("ca", lens)
+        g.moa_state_set_len("sa", lens)
+        g.moa_lsa_forward(h, [A] * nb, want_kv=False)
+        g.moa_sa_append(tok, [A] * nb)
+        g.moa_tree_begin(root)
+        res = None
+        for s in range(D):
+            R = nb if s == 0 else nb * B
+            ids, lp, _ = g.moa_draft_step(out=(ids_buf[:R], lp_buf[:R], None))
+            res = g.moa_tree_expand(ids, lp, out=outs)
+        return moa.moa_tree_attn_mask(res[1])
+
+    def cycle_e2e():
+        h_stage.copy_(h_host, non_blocking=True)
+        tok_stage.copy_(tok_host, non_blocking=True)
+        root_stage.copy_(root_host, non_blocking=True)
+        mask = cycle(h_stage, tok_stage, root_stage)
+        for hst, d in zip(host_out, outs):
+            hst.copy_(d, non_blocking=True)
+        mask_host.copy_(mask, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, k):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        start.record()
+        for _ in range(k):
+            fn()
+        stop.record()
+        barrier()
+        ms = start.elapsed_time(stop)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        cycle(h_dev, tok_dev, root_dev)
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    n0 = g.moa_launch_count()
+    g.moa_profile_begin()
+    ms = timed(lambda: cycle(h_dev, tok_dev, root_dev), args.steps)
+    lm_ms, lm_n = g.moa_profile_end()
+    launches = g.moa_launch_count() - n0
+    clocks = sampler.stop()
+    for _ in range(2):
+        cycle_e2e()
+    ms_e2e = timed(cycle_e2e, args.steps)
+    assert g.moa_state_status() == 0
+
+    t_cycle = ms / args.steps / 1e3
+    t_e2e = ms_e2e / args.steps / 1e3
+    ab = algorithmic_bytes(p)
+    peak, peak_kind = measured_peaks()
+    lm_avg_s = lm_ms / max(lm_n, 1) / 1e3
+    achieved = ab["lm_head"] / lm_avg_s / 1e9 if lm_n else None
+    h2d = h_host.numel() * h_host.element_size() + tok_host.numel() * 4 + root_host.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in host_out) + mask_host.numel()
+    line = {
+        "metric": "draft_tree_steps_per_sec", "value": world * D / t_cycle, "unit": "steps/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_cycle * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": p.dtype, "data": "synthetic",
+        "config": workload_config(p),
+        "drafted_tokens_per_sec": world * nb * m / t_cycle,
+        "e2e": {"value": world * D / t_e2e, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "lm_head", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "launches_timed": lm_n, "avg_launch_us": lm_avg_s * 1e6},
+        "cycle_roofline": {"algorithmic_bytes_per_cycle": D * ab["step"] + ab["lsa"],
+                           "achieved_gbs": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9,
+                           "frac_of_measured": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9 / peak,
+                           "frac_of_8tbs": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9 / 8000.0},
+        "replicas": "replicas only: no data-path collective" if world > 1 else None,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cyc, cores, what = oracle_sample(p)
+        line["cpu_baseline"] = {"value": D / cyc, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -159,6 +159,16 @@ moa_status moa_tree_attn_mask(const int32_t *parent, int32_t batch, int32_t n, v
 /* Reads back the device status word kept in st->tree (0 = no device-side problem seen). Synchronises the stream. */
 moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
 
+/* Measurement hooks (no counterpart in the paper). Between moa_profile_begin and moa_profile_end every
+ * launch of the LM-head kernel (the step's dominant HBM stream, Eq. 1) is bracketed by CUDA events on the
+ * caller's stream; moa_profile_end synchronises those events and returns their summed duration in
+ * milliseconds and the number of launches timed (at most 512 per begin/end pair; later ones are skipped).
+ * Do not use inside a stream capture. */
+moa_status moa_profile_begin(moa_ctx *ctx);
+moa_status moa_profile_end(moa_ctx *ctx, double *ms_total, int32_t *launches);
+/* Kernels launched so far by this host thread through the library. */
+int64_t moa_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -12,6 +12,9 @@
 using namespace moa;
 
 static thread_local char g_cuda_err[256] = "";
+static thread_local long long g_launches = 0;
+
+enum { PROF_MAX = 512 };
 
 struct moa_ctx {
   moa_config c;
@@ -19,6 +22,11 @@ struct moa_ctx {
   int sm_count;
   size_t elt;          // bytes per T
   TreeLayout tl;
+  // measurement hooks: event pairs around the LM-head launches
+  bool prof_on;
+  int prof_n;
+  cudaEvent_t prof_ev[2 * PROF_MAX];
+  bool prof_made;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -76,6 +84,7 @@ static int chunk_from_bytes(const moa_config& c, size_t elt, size_t ws_bytes) {
 // ---------------------------------------------------------------------------------------------
 #define MOA_CHECK_LAUNCH()                                                                               \
   do {                                                                                                   \
+    ++g_launches;                                                                                        \
     cudaError_t e__ = cudaGetLastError();                                                                \
     if (e__ != cudaSuccess) {                                                                            \
       snprintf(g_cuda_err, sizeof(g_cuda_err), "%s:%d %s", __FILE__, __LINE__, cudaGetErrorString(e__)); \
@@ -307,7 +316,10 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   if (hidden_out) MOA_TRY(cast_flat<T>(s, xres, (T*)hidden_out, (size_t)R * E));
   rmsnorm_rows_kernel<float, T><<<R, 256, 0, s>>>(xres, nullptr, 0, (const T*)w.final_norm, E, c.rms_eps, nullptr, xn);
   MOA_CHECK_LAUNCH();
+  const bool timed = ctx->prof_on && ctx->prof_n < PROF_MAX;
+  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
   MOA_TRY(gemm<T>(s, xn, w.lm_head, R, V, E, nullptr, 0, logits, V));
+  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
   lse_topk_rows_kernel<<<R, 256, 0, s>>>(logits, V, B, topk_id, topk_logp);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
@@ -381,11 +393,59 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
   ctx->sm_count = prop.multiProcessorCount;
   ctx->elt = cfg->dtype == MOA_F32 ? 4 : 2;
   ctx->tl = make_tree_layout(cfg->max_batch, cfg->tree_topk, cfg->tree_depth, cfg->sa_hkv, cfg->head_dim, ctx->elt);
+  ctx->prof_on = false;
+  ctx->prof_n = 0;
+  ctx->prof_made = false;
   *out = ctx;
   return MOA_OK;
 }
 
-void moa_destroy(moa_ctx* ctx) { delete ctx; }
+void moa_destroy(moa_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->prof_made)
+    for (int i = 0; i < 2 * PROF_MAX; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+  delete ctx;
+}
+
+moa_status moa_profile_begin(moa_ctx* ctx) {
+  if (!ctx) return MOA_ERR_NULL;
+  if (!ctx->prof_made) {
+    for (int i = 0; i < 2 * PROF_MAX; ++i) {
+      cudaError_t e = cudaEventCreate(&ctx->prof_ev[i]);
+      if (e != cudaSuccess) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_profile_begin: %s", cudaGetErrorString(e));
+        for (int j = 0; j < i; ++j) cudaEventDestroy(ctx->prof_ev[j]);
+        return MOA_ERR_CUDA;
+      }
+    }
+    ctx->prof_made = true;
+  }
+  ctx->prof_n = 0;
+  ctx->prof_on = true;
+  return MOA_OK;
+}
+
+moa_status moa_profile_end(moa_ctx* ctx, double* ms_total, int32_t* launches) {
+  if (!ctx || !ms_total || !launches) return MOA_ERR_NULL;
+  if (!ctx->prof_on) return MOA_ERR_STATE;
+  ctx->prof_on = false;
+  double total = 0.0;
+  for (int i = 0; i < ctx->prof_n; ++i) {
+    cudaError_t e = cudaEventSynchronize(ctx->prof_ev[2 * i + 1]);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]);
+    if (e != cudaSuccess) {
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_profile_end: %s", cudaGetErrorString(e));
+      return MOA_ERR_CUDA;
+    }
+    total += ms;
+  }
+  *ms_total = total;
+  *launches = ctx->prof_n;
+  return MOA_OK;
+}
+
+int64_t moa_launch_count(void) { return g_launches; }
 
 moa_status moa_state_bytes(const moa_ctx* ctx, int32_t lsa_chunk_tokens, size_t* tree_bytes, size_t* workspace_bytes) {
   if (!ctx) return MOA_ERR_NULL;

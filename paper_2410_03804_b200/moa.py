@@ -21,7 +21,8 @@ MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_tree_begin", "moa_draft_step",
-           "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status"]
+           "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end",
+           "moa_launch_count"]
 
 
 class MoaConfig(C.Structure):
@@ -91,9 +92,13 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_tree_expand.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moa_tree_attn_mask.argtypes = [vp, i32, i32, vp, i32, vp]
     lib.moa_state_status.argtypes = [vp, C.POINTER(MoaState), vp]
+    lib.moa_profile_begin.argtypes = [vp]
+    lib.moa_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
+    lib.moa_launch_count.argtypes = []
     for n in EXPORTS:
-        if n not in ("moa_destroy", "moa_status_str", "moa_last_cuda_error"):
+        if n not in ("moa_destroy", "moa_status_str", "moa_last_cuda_error", "moa_launch_count"):
             getattr(lib, n).restype = i32
+    lib.moa_launch_count.restype = C.c_int64
     _lib = lib
     return lib
 
@@ -262,6 +267,18 @@ class MoA:
 
     def moa_state_status(self, stream=None) -> int:
         return int(self.lib.moa_state_status(self.h, C.byref(self.st), _stream(stream)))
+
+    def moa_profile_begin(self):
+        _check(self.lib.moa_profile_begin(self.h), "moa_profile_begin")
+
+    def moa_profile_end(self):
+        """Returns (summed LM-head kernel milliseconds, launches timed)."""
+        ms, n = C.c_double(), C.c_int32()
+        _check(self.lib.moa_profile_end(self.h, C.byref(ms), C.byref(n)), "moa_profile_end")
+        return ms.value, n.value
+
+    def moa_launch_count(self) -> int:
+        return int(self.lib.moa_launch_count())
 
     # ---- convenience for tests / bench: raw views of the tree blob ---------------------------
     def fill_cache(self, which: str, k: torch.Tensor, v: torch.Tensor):
