@@ -8,13 +8,24 @@
 
 #include "moa_basic.cuh"
 #include "moa_tree.cuh"
+#include "moa_wstream.cuh"
 
 using namespace moa;
 
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512 };
+enum { PROF_MAX = 512, WMAP_MAX = 32 };
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct WeightMap {
+  const void* ptr;
+  int n, k;
+  CUtensorMap tm;
+};
 
 struct moa_ctx {
   moa_config c;
@@ -22,6 +33,11 @@ struct moa_ctx {
   int sm_count;
   size_t elt;          // bytes per T
   TreeLayout tl;
+  // tensor-core path (bf16 only)
+  EncodeTiledFn encode;
+  WeightMap wmap[WMAP_MAX];
+  int n_wmap;
+  bool fast;           // weight-streaming tcgen05 GEMMs usable
   // measurement hooks: event pairs around the LM-head launches
   bool prof_on;
   int prof_n;
@@ -33,35 +49,42 @@ struct moa_ctx {
 // workspace carving (same arithmetic in moa_state_bytes and in the calls)
 // ---------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t xres, xn, wide, narrow, obuf, logits, kvf, kvn, total;
-  int rows_cap, draft_rows, chunk_tok;
+  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, total;
+  int rows_cap, draft_rows, chunk_tok, part_rows, wide;
 };
 
 static inline int imax(int a, int b) { return a > b ? a : b; }
+static inline int imin(int a, int b) { return a < b ? a : b; }
 
 static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) {
   Workspace p;
   p.chunk_tok = chunk_tok;
   p.draft_rows = c.max_batch * c.tree_topk;
   p.rows_cap = imax(p.draft_rows, chunk_tok * c.n_stack);
+  p.part_rows = imax(640, p.rows_cap);      // room for several K-split planes when there are few rows
   const int dmax = imax(c.d_model, c.d_stack);
   const int qkv_lsa = (c.lsa_hq + 2 * c.lsa_hkv) * c.head_dim;
   const int qkv_sa = (c.sa_hq + 2 * c.sa_hkv) * c.head_dim;
   const int q_ca = imax(c.ca_hq * c.head_dim, 2 * c.ca_hkv * c.head_dim);
   const int fmax = imax(c.lsa_mlp, imax(c.sa_mlp, c.ca_mlp));
-  const int wide = imax(imax(qkv_lsa, qkv_sa), imax(q_ca, 2 * fmax));
+  p.wide = imax(imax(imax(qkv_lsa, qkv_sa), imax(q_ca, 2 * fmax)), dmax);
   const int narrow = imax(imax(qkv_lsa, qkv_sa), imax(q_ca, fmax));
   const int omax = imax(c.lsa_hq, imax(c.sa_hq, c.ca_hq)) * c.head_dim;
+  const size_t n_sub = (size_t)4 * ((c.vocab + WS_BM - 1) / WS_BM);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
-  p.xres = take((size_t)p.rows_cap * dmax * sizeof(float));     // residual stream, fp32
-  p.xn = take((size_t)p.rows_cap * dmax * elt);                 // normalised GEMM operand, T
-  p.wide = take((size_t)p.rows_cap * wide * sizeof(float));     // q, k, v or gate, up: fp32
-  p.narrow = take((size_t)p.rows_cap * narrow * elt);           // q, k, v or silu(gate)*up: T
-  p.obuf = take((size_t)p.rows_cap * omax * elt);               // attention output, T
-  p.logits = take((size_t)p.draft_rows * c.vocab * sizeof(float));
-  p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));  // LSA output rows, fp32
-  p.kvn = take((size_t)chunk_tok * c.d_stack * elt);            // their normalised copy, T
+  p.xres = take((size_t)p.rows_cap * dmax * sizeof(float));      // residual stream, fp32
+  p.xn = take((size_t)p.rows_cap * dmax * elt);                  // normalised GEMM operand, T
+  p.part = take((size_t)p.part_rows * p.wide * sizeof(float));   // GEMM outputs: K-split partial planes, fp32
+  p.narrow = take((size_t)p.rows_cap * narrow * elt);            // q|k|v or silu(gate)*up, T
+  p.obuf = take((size_t)p.rows_cap * omax * elt);                // attention output, T
+  p.logits = take(elt == 4 ? (size_t)p.draft_rows * c.vocab * sizeof(float) : 256);   // fp32 path only
+  p.pmax = take(n_sub * p.draft_rows * sizeof(float));           // LM-head partials per 32-row vocabulary slice
+  p.psum = take(n_sub * p.draft_rows * sizeof(float));
+  p.cval = take(n_sub * p.draft_rows * c.tree_topk * sizeof(float));
+  p.cid = take(n_sub * p.draft_rows * c.tree_topk * sizeof(int));
+  p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));   // LSA output rows, fp32
+  p.kvn = take((size_t)chunk_tok * c.d_stack * elt);             // their normalised copy, T
   p.total = o;
   return p;
 }
@@ -98,58 +121,186 @@ static int chunk_from_bytes(const moa_config& c, size_t elt, size_t ws_bytes) {
   } while (0)
 
 static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+static inline unsigned blocks_for(size_t total, int threads) { return (unsigned)((total + threads - 1) / threads); }
 
-template <typename T>
-static moa_status gemm(cudaStream_t s, const T* A, const void* W, int R, int N, int K, const float* res, int ldr,
-                       float* C, int ldc) {
-  if (R <= 0 || N <= 0) return MOA_OK;
-  dim3 grid((N + 63) / 64, (R + 63) / 64);
-  gemm_fma_kernel<T><<<grid, 256, 0, s>>>(A, (const T*)W, R, N, K, res, ldr, C, ldc);
+// 2-D bf16 tensor map: global [rows, k] row-major, box 64 x box_rows, 128-byte swizzle, zero fill outside.
+static bool encode_map(const moa_ctx* ctx, CUtensorMap* tm, const void* ptr, int rows, int k, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)k * 2};
+  cuuint32_t box[2] = {(cuuint32_t)WS_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return r == CUDA_SUCCESS;
+}
+
+static const WeightMap* find_wmap(const moa_ctx* ctx, const void* w) {
+  for (int i = 0; i < ctx->n_wmap; ++i)
+    if (ctx->wmap[i].ptr == w) return &ctx->wmap[i];
+  return nullptr;
+}
+
+// K-split count: best use of the SMs' waves, fewest splits among near-equal choices.
+static int pick_splits(int tiles, int kb_total, int R, int part_rows, int sms) {
+  const int smax = imax(1, imin(imin(16, kb_total), part_rows / imax(R, 1)));
+  int best = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= smax; ++s) {
+    const int units = tiles * s;
+    const int waves = (units + sms - 1) / sms;
+    const double eff = (double)units / ((double)waves * sms);
+    if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+  }
+  return best;
+}
+
+struct LinOut {          // where a linear layer left its result: `splits` fp32 planes of [R, ld]
+  const float* part;
+  int splits;
+  size_t plane;
+  int ld;
+};
+
+template <int NPAD>
+static moa_status launch_ws(cudaStream_t s, const WsParams& P, int grid) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(wstream_gemm_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ws_smem_bytes(NPAD));
+    if (e != cudaSuccess) {
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+      return MOA_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  wstream_gemm_kernel<NPAD><<<grid, WS_THREADS, ws_smem_bytes(NPAD), s>>>(P);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
 
+static moa_status launch_ws_any(cudaStream_t s, const WsParams& P, int npad, int grid) {
+  switch (npad) {
+    case 16: return launch_ws<16>(s, P, grid);
+    case 32: return launch_ws<32>(s, P, grid);
+    case 64: return launch_ws<64>(s, P, grid);
+    case 128: return launch_ws<128>(s, P, grid);
+    default: return launch_ws<256>(s, P, grid);
+  }
+}
+
+static inline int npad_for(int R) { return R <= 16 ? 16 : R <= 32 ? 32 : R <= 64 ? 64 : R <= 128 ? 128 : 256; }
+
+static bool fast_shape(const moa_ctx* ctx, int K, int nseg, const void* const* W) {
+  if (!ctx->fast || K % WS_BK != 0) return false;
+  for (int i = 0; i < nseg; ++i)
+    if (!find_wmap(ctx, W[i])) return false;
+  return true;
+}
+
+// Linear layer(s) sharing one input: Y[:, col_i : col_i + N_i] = X W_i^T for up to three weight matrices.
+// Result: fp32 partial planes in the workspace's `part` buffer (see LinOut).
 template <typename T>
-static moa_status attention(cudaStream_t s, int dh, const T* q, int R, int hq, int hkv, const T* kA, const T* vA,
-                            int capA, const int* lenA, int nA_fixed, const T* kB, const T* vB, int capB,
-                            const int* slotsB, int slots_ld, int nB, int rows_per_seq, T* out) {
+static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K, int nseg, const void* const* W,
+                         const int* N, char* ws, const Workspace& p, LinOut* out, void* status_word) {
+  float* part = (float*)(ws + p.part);
+  int ntot = 0;
+  for (int i = 0; i < nseg; ++i) ntot += N[i];
+  out->part = part;
+  out->ld = ntot;
+  out->plane = (size_t)R * ntot;
+  out->splits = 1;
+  if (R <= 0) return MOA_OK;
+  if (sizeof(T) == 2 && fast_shape(ctx, K, nseg, W)) {
+    WsParams P;
+    memset(&P, 0, sizeof(P));
+    P.n_seg = nseg;
+    int tiles = 0, col = 0;
+    for (int i = 0; i < nseg; ++i) {
+      P.tmW[i] = find_wmap(ctx, W[i])->tm;
+      P.seg_n[i] = N[i];
+      P.seg_tile0[i] = tiles;
+      P.seg_col[i] = col;
+      tiles += (N[i] + WS_BM - 1) / WS_BM;
+      col += N[i];
+    }
+    P.tiles_total = tiles;
+    P.kb_total = K / WS_BK;
+    P.mode = 0;
+    P.ldo = ntot;
+    P.plane = out->plane;
+    P.status = (int*)status_word;
+    const int nblk = (R + 255) / 256;
+    P.splits = pick_splits(tiles * nblk, P.kb_total, R, p.part_rows, ctx->sm_count);
+    out->splits = P.splits;
+    for (int r0 = 0; r0 < R; r0 += 256) {
+      const int rows = imin(256, R - r0);
+      const int npad = npad_for(rows);
+      if (!encode_map(ctx, &P.tmX, (const bf16*)X + (size_t)r0 * K, rows, K, npad)) return MOA_ERR_CUDA;
+      P.R = rows;
+      P.out = part + (size_t)r0 * ntot;
+      const int units = tiles * P.splits;
+      MOA_TRY(launch_ws_any(s, P, npad, imin(units, ctx->sm_count)));
+    }
+    return MOA_OK;
+  }
+  int col = 0;
+  for (int i = 0; i < nseg; ++i) {
+    dim3 grid((N[i] + 63) / 64, (R + 63) / 64);
+    gemm_fma_kernel<T><<<grid, 256, 0, s>>>(X, (const T*)W[i], R, N[i], K, nullptr, 0, part + col, ntot);
+    MOA_CHECK_LAUNCH();
+    col += N[i];
+  }
+  return MOA_OK;
+}
+
+template <typename T>
+static moa_status attention(cudaStream_t s, int dh, const T* q, int q_ld, int R, int hq, int hkv, const T* kA,
+                            const T* vA, int capA, int posA_ld, const int* lenA, int nA_fixed, const T* kB, const T* vB,
+                            int capB, const int* slotsB, int slots_ld, int nB, int rows_per_seq, T* out) {
   if (R <= 0) return MOA_OK;
   dim3 grid(R, hq);
   if (dh == 128)
-    attn_rows_kernel<T, 128><<<grid, 128, 0, s>>>(q, hq, hkv, kA, vA, capA, lenA, nA_fixed, kB, vB, capB, slotsB,
-                                                  slots_ld, nB, rows_per_seq, out);
+    attn_rows_kernel<T, 128><<<grid, 128, 0, s>>>(q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
+                                                  slotsB, slots_ld, nB, rows_per_seq, out);
   else
-    attn_rows_kernel<T, 64><<<grid, 128, 0, s>>>(q, hq, hkv, kA, vA, capA, lenA, nA_fixed, kB, vB, capB, slotsB,
-                                                 slots_ld, nB, rows_per_seq, out);
+    attn_rows_kernel<T, 64><<<grid, 128, 0, s>>>(q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
+                                                 slotsB, slots_ld, nB, rows_per_seq, out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
 
+// xres += previous linear's result; xn = RMSNorm(xres; gain) (skipped when gain == nullptr)
 template <typename T>
-static moa_status cast_flat(cudaStream_t s, const float* x, T* y, size_t total) {
-  if (total == 0) return MOA_OK;
-  cast_flat_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, s>>>(x, y, total);
+static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, const Workspace& p, int R, int K,
+                                const LinOut* lo, const void* gain, void* hidden_out) {
+  if (R <= 0) return MOA_OK;
+  residual_norm_kernel<T><<<R, 256, 0, s>>>((float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0,
+                                            lo ? lo->plane : 0, K, (const T*)gain, ctx->c.rms_eps, (T*)(ws + p.xn),
+                                            (T*)hidden_out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
 
-// MLP with residual: xres += W_down (silu(W_gate n) * (W_up n)), n = RMSNorm(xres; gain)
+// MLP, given xn = RMSNorm(xres) already in place: leaves the down-projection in `lo`
+// (the caller folds it into the residual stream together with the next normalisation).
 template <typename T>
-static moa_status mlp_block(cudaStream_t s, const moa_ctx* ctx, const Workspace& p, char* ws, int R, int K, int F,
-                            const void* gain, const void* wgate, const void* wup, const void* wdown) {
-  float* xres = (float*)(ws + p.xres);
-  T* xn = (T*)(ws + p.xn);
-  float* gate = (float*)(ws + p.wide);
-  float* up = gate + (size_t)R * F;
+static moa_status mlp_block(cudaStream_t s, moa_ctx* ctx, const Workspace& p, char* ws, int R, int K, int F,
+                            const void* wgate, const void* wup, const void* wdown, LinOut* lo, void* status_word) {
+  const T* xn = (const T*)(ws + p.xn);
   T* h = (T*)(ws + p.narrow);
-  rmsnorm_rows_kernel<float, T><<<R, 256, 0, s>>>(xres, nullptr, 0, (const T*)gain, K, ctx->c.rms_eps, nullptr, xn);
-  MOA_CHECK_LAUNCH();
-  MOA_TRY(gemm<T>(s, xn, wgate, R, F, K, nullptr, 0, gate, F));
-  MOA_TRY(gemm<T>(s, xn, wup, R, F, K, nullptr, 0, up, F));
+  const void* W2[2] = {wgate, wup};
+  const int N2[2] = {F, F};
+  MOA_TRY(linear<T>(ctx, s, xn, R, K, 2, W2, N2, ws, p, lo, status_word));
   const size_t total = (size_t)R * F;
-  silu_mul_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, s>>>(gate, up, F, F, h, total);
-  MOA_CHECK_LAUNCH();
-  return gemm<T>(s, h, wdown, R, K, F, xres, K, xres, K);
+  if (total) {
+    silu_mul_split_kernel<T><<<blocks_for(total, 256), 256, 0, s>>>(lo->part, lo->splits, lo->plane, F, h, total);
+    MOA_CHECK_LAUNCH();
+  }
+  const void* W1[1] = {wdown};
+  const int N1[1] = {K};
+  return linear<T>(ctx, s, h, R, F, 1, W1, N1, ws, p, lo, status_word);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -161,38 +312,41 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
   const moa_config& c = ctx->c;
   const moa_weights& w = ctx->w;
   const int S = c.n_stack, D = c.d_stack, dh = c.head_dim;
-  const int nq = c.lsa_hq * dh, nkv = c.lsa_hkv * dh;
+  const int nq = c.lsa_hq * dh, nkv = c.lsa_hkv * dh, ld = nq + 2 * nkv;
+  void* status_word = (char*)st->tree + ctx->tl.status;
   float* xres = (float*)(ws + p.xres);
   T* xn = (T*)(ws + p.xn);
-  float* wide = (float*)(ws + p.wide);
   T* narrow = (T*)(ws + p.narrow);
   T* obuf = (T*)(ws + p.obuf);
   float* kvf = (float*)(ws + p.kvf);
   T* kvn = (T*)(ws + p.kvn);
   const int total = split.off[split.n_seq];
+  LinOut lo;
   for (int t0 = 0; t0 < total; t0 += p.chunk_tok) {
     const int nt = (total - t0) < p.chunk_tok ? (total - t0) : p.chunk_tok;
     const int R = nt * S;
     const T* x = (const T*)h_stack + (size_t)t0 * S * D;
-    // pre-norm and q, k, v projections of every (token, layer) row; three dense fp32 blocks
+    // pre-norm and q, k, v projections of every (token, layer) row: rows of [q | k | v]
     rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>(x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn);
     MOA_CHECK_LAUNCH();
-    float* qf = wide;
-    float* kf = qf + (size_t)R * nq;
-    float* vf = kf + (size_t)R * nkv;
-    MOA_TRY(gemm<T>(s, xn, w.lsa_wq, R, nq, D, nullptr, 0, qf, nq));
-    MOA_TRY(gemm<T>(s, xn, w.lsa_wk, R, nkv, D, nullptr, 0, kf, nkv));
-    MOA_TRY(gemm<T>(s, xn, w.lsa_wv, R, nkv, D, nullptr, 0, vf, nkv));
-    MOA_TRY(cast_flat<T>(s, wide, narrow, (size_t)R * (nq + 2 * nkv)));
-    const T* qd = narrow;
-    const T* kd = qd + (size_t)R * nq;
-    const T* vd = kd + (size_t)R * nkv;
+    const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
+    const int N3[3] = {nq, nkv, nkv};
+    MOA_TRY(linear<T>(ctx, s, xn, R, D, 3, W3, N3, ws, p, &lo, status_word));
+    {
+      const size_t tot = (size_t)R * ld;
+      sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
+      MOA_CHECK_LAUNCH();
+    }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
-    MOA_TRY(attention<T>(s, dh, qd, R, c.lsa_hq, c.lsa_hkv, kd, vd, S, nullptr, S, nullptr, nullptr, 0, nullptr, 0, 0,
-                         S, obuf));
+    MOA_TRY(attention<T>(s, dh, narrow, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld, nullptr, S,
+                         (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, S, obuf));
     // out-projection + residual, MLP + residual
-    MOA_TRY(gemm<T>(s, obuf, w.lsa_wo, R, D, nq, xres, D, xres, D));
-    MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, D, c.lsa_mlp, w.lsa_norm2, w.lsa_wgate, w.lsa_wup, w.lsa_wdown));
+    const void* W1[1] = {w.lsa_wo};
+    const int N1[1] = {D};
+    MOA_TRY(linear<T>(ctx, s, obuf, R, nq, 1, W1, N1, ws, p, &lo, status_word));
+    MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, D, &lo, w.lsa_norm2, nullptr));
+    MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, D, c.lsa_mlp, w.lsa_wgate, w.lsa_wup, w.lsa_wdown, &lo, status_word));
+    MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, D, &lo, nullptr, nullptr));
     // mean over layers
     T* kvo = kv_out ? (T*)kv_out + (size_t)t0 * D : nullptr;
     mean_layers_kernel<T><<<nt, 256, 0, s>>>(xres, S, D, kvf, kvo);
@@ -201,12 +355,11 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     rmsnorm_rows_kernel<float, T><<<nt, 256, 0, s>>>(kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn);
     MOA_CHECK_LAUNCH();
     const int ckv = c.ca_hkv * dh;
-    float* ckf = wide;
-    float* cvf = ckf + (size_t)nt * ckv;
-    MOA_TRY(gemm<T>(s, kvn, w.ca_wk, nt, ckv, D, nullptr, 0, ckf, ckv));
-    MOA_TRY(gemm<T>(s, kvn, w.ca_wv, nt, ckv, D, nullptr, 0, cvf, ckv));
-    cache_append_kernel<T><<<nt, 256, 0, s>>>(ckf, ckv, 0, nt * ckv, ckv, st->ca_len, c.max_ctx, split, t0,
-                                              (T*)st->ca_k, (T*)st->ca_v);
+    const void* W2[2] = {w.ca_wk, w.ca_wv};
+    const int N2[2] = {ckv, ckv};
+    MOA_TRY(linear<T>(ctx, s, kvn, nt, D, 2, W2, N2, ws, p, &lo, status_word));
+    cache_append_kernel<T><<<nt, 256, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * ckv, 0, ckv, ckv, st->ca_len, c.max_ctx,
+                                              split, t0, (T*)st->ca_k, (T*)st->ca_v);
     MOA_CHECK_LAUNCH();
   }
   add_len_kernel<<<1, 64, 0, s>>>(st->ca_len, split);
@@ -220,30 +373,79 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
   const moa_config& c = ctx->c;
   const moa_weights& w = ctx->w;
   const int E = c.d_model, dh = c.head_dim, nkv = c.sa_hkv * dh;
+  void* status_word = (char*)st->tree + ctx->tl.status;
   T* xn = (T*)(ws + p.xn);
-  float* wide = (float*)(ws + p.wide);
   const int total = split.off[split.n_seq];
+  LinOut lo;
   for (int t0 = 0; t0 < total; t0 += p.rows_cap) {
     const int R = (total - t0) < p.rows_cap ? (total - t0) : p.rows_cap;
     rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>((const T*)w.embed, tok + t0, c.vocab, (const T*)w.sa_norm1, E,
                                                 c.rms_eps, nullptr, xn);
     MOA_CHECK_LAUNCH();
-    float* kf = wide;
-    float* vf = kf + (size_t)R * nkv;
-    MOA_TRY(gemm<T>(s, xn, w.sa_wk, R, nkv, E, nullptr, 0, kf, nkv));
-    MOA_TRY(gemm<T>(s, xn, w.sa_wv, R, nkv, E, nullptr, 0, vf, nkv));
+    const void* W2[2] = {w.sa_wk, w.sa_wv};
+    const int N2[2] = {nkv, nkv};
+    MOA_TRY(linear<T>(ctx, s, xn, R, E, 2, W2, N2, ws, p, &lo, status_word));
     RopeRows rr;
     memset(&rr, 0, sizeof(rr));
     rr.mode = 1;
     rr.max_ctx = c.max_ctx;
     rr.split = split;
     rr.row0 = t0;
-    // k and v rows are dense [R, nkv] blocks: leading dimension nkv, v block R*nkv elements after k
-    rope_store_kernel<T><<<R, 128, 0, s>>>(kf, nkv, 0, 0, R * nkv, 0, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr,
-                                           (T*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
+    rope_store_kernel<T><<<R, 128, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
+                                           c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
     MOA_CHECK_LAUNCH();
   }
   add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+// LM head + log-softmax + top-B on xn = RMSNorm(o_hat; final_norm)
+template <typename T>
+static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int R, int* topk_id,
+                            float* topk_logp, void* status_word) {
+  const moa_config& c = ctx->c;
+  const int E = c.d_model, V = c.vocab, B = c.tree_topk;
+  const T* xn = (const T*)(ws + p.xn);
+  const void* W1[1] = {ctx->w.lm_head};
+  const bool timed = ctx->prof_on && ctx->prof_n < PROF_MAX;
+  if (sizeof(T) == 2) {
+    if (R > 256 || !fast_shape(ctx, E, 1, W1)) return MOA_ERR_SHAPE;   // validated at moa_create
+    WsParams P;
+    memset(&P, 0, sizeof(P));
+    P.n_seg = 1;
+    P.tmW[0] = find_wmap(ctx, ctx->w.lm_head)->tm;
+    P.seg_n[0] = V;
+    P.tiles_total = (V + WS_BM - 1) / WS_BM;
+    P.kb_total = E / WS_BK;
+    P.splits = 1;
+    P.mode = 1;
+    P.R = R;
+    P.B = B;
+    P.p_max = (float*)(ws + p.pmax);
+    P.p_sum = (float*)(ws + p.psum);
+    P.c_val = (float*)(ws + p.cval);
+    P.c_id = (int*)(ws + p.cid);
+    P.status = (int*)status_word;
+    const int npad = npad_for(R);
+    if (!encode_map(ctx, &P.tmX, xn, R, E, npad)) return MOA_ERR_CUDA;
+    if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
+    MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count)));
+    if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
+    lm_merge_kernel<<<R, MERGE_THREADS, 0, s>>>(P.p_max, P.p_sum, P.c_val, P.c_id, 4 * P.tiles_total, R, B, topk_id,
+                                                topk_logp);
+    MOA_CHECK_LAUNCH();
+    return MOA_OK;
+  }
+  float* logits = (float*)(ws + p.logits);
+  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
+  {
+    dim3 grid((V + 63) / 64, (R + 63) / 64);
+    gemm_fma_kernel<T><<<grid, 256, 0, s>>>(xn, (const T*)ctx->w.lm_head, R, V, E, nullptr, 0, logits, V);
+    MOA_CHECK_LAUNCH();
+  }
+  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
+  lse_topk_rows_kernel<<<R, 256, 0, s>>>(logits, V, B, topk_id, topk_logp);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -255,6 +457,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   const moa_weights& w = ctx->w;
   const TreeLayout& L = ctx->tl;
   const TreePtrs tp = tree_ptrs(st->tree, L);
+  void* status_word = (char*)st->tree + L.status;
   const int step = st->step, B = c.tree_topk, D = c.tree_depth;
   const int R = step == 0 ? batch : batch * B;
   const int rows_per_seq = step == 0 ? 1 : B;
@@ -267,62 +470,62 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   T* tv = (T*)((char*)st->tree + L.tv);
   float* xres = (float*)(ws + p.xres);
   T* xn = (T*)(ws + p.xn);
-  float* wide = (float*)(ws + p.wide);
   T* narrow = (T*)(ws + p.narrow);
   T* obuf = (T*)(ws + p.obuf);
-  float* logits = (float*)(ws + p.logits);
+  LinOut lo;
 
   // ---- self-attention block ----
   rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>((const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn);
   MOA_CHECK_LAUNCH();
   const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh;
-  float* qf = wide;
-  float* kf = qf + (size_t)R * nq;
-  float* vf = kf + (size_t)R * nkv;
-  MOA_TRY(gemm<T>(s, xn, w.sa_wq, R, nq, E, nullptr, 0, qf, nq));
-  MOA_TRY(gemm<T>(s, xn, w.sa_wk, R, nkv, E, nullptr, 0, kf, nkv));
-  MOA_TRY(gemm<T>(s, xn, w.sa_wv, R, nkv, E, nullptr, 0, vf, nkv));
+  {
+    const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
+    const int N3[3] = {nq, nkv, nkv};
+    MOA_TRY(linear<T>(ctx, s, xn, R, E, 3, W3, N3, ws, p, &lo, status_word));
+  }
   RopeRows rr;
   memset(&rr, 0, sizeof(rr));
   rr.mode = 0;
   rr.step = step;
   rr.B = B;
   rr.slots = L.NS;
-  // q, k, v blocks have different leading dimensions; the kernel indexes a row as base + r*ld + off, so
-  // it is launched once for q (+ a k/v pass that writes nothing is avoided by giving hkv = 0) and once for k, v.
-  rope_store_kernel<T><<<R, 128, 0, s>>>(qf, nq, 0, 0, 0, c.sa_hq, 0, dh, c.sa_rope_theta, st->sa_len, rr, narrow,
-                                         (T*)nullptr, (T*)nullptr);
+  rope_store_kernel<T><<<R, 128, 0, s>>>(lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
+                                         dh, c.sa_rope_theta, st->sa_len, rr, narrow, tk, tv);
   MOA_CHECK_LAUNCH();
-  rope_store_kernel<T><<<R, 128, 0, s>>>(kf, nkv, 0, 0, R * nkv, 0, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr,
-                                         (T*)nullptr, tk, tv);
-  MOA_CHECK_LAUNCH();
-  MOA_TRY(attention<T>(s, dh, narrow, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v, c.max_ctx,
+  MOA_TRY(attention<T>(s, dh, narrow, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v, c.max_ctx, nkv,
                        st->sa_len, 0, tk, tv, L.NS, row_anc, D, step + 1, rows_per_seq, obuf));
-  MOA_TRY(gemm<T>(s, obuf, w.sa_wo, R, E, nq, xres, E, xres, E));
-  MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.sa_mlp, w.sa_norm2, w.sa_wgate, w.sa_wup, w.sa_wdown));
+  {
+    const void* W1[1] = {w.sa_wo};
+    const int N1[1] = {E};
+    MOA_TRY(linear<T>(ctx, s, obuf, R, nq, 1, W1, N1, ws, p, &lo, status_word));
+  }
+  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.sa_norm2, nullptr));
+  MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.sa_mlp, w.sa_wgate, w.sa_wup, w.sa_wdown, &lo, status_word));
 
   // ---- cross-attention block ----
-  const int cq = c.ca_hq * dh;
-  rmsnorm_rows_kernel<float, T><<<R, 256, 0, s>>>(xres, nullptr, 0, (const T*)w.ca_normq, E, c.rms_eps, nullptr, xn);
-  MOA_CHECK_LAUNCH();
-  MOA_TRY(gemm<T>(s, xn, w.ca_wq, R, cq, E, nullptr, 0, wide, cq));
-  MOA_TRY(cast_flat<T>(s, wide, narrow, (size_t)R * cq));
-  MOA_TRY(attention<T>(s, dh, narrow, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx,
-                       st->ca_len, 0, nullptr, nullptr, 0, nullptr, 0, 0, rows_per_seq, obuf));
-  MOA_TRY(gemm<T>(s, obuf, w.ca_wo, R, E, cq, xres, E, xres, E));
-  MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.ca_mlp, w.ca_norm2, w.ca_wgate, w.ca_wup, w.ca_wdown));
+  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_normq, nullptr));
+  const int cq = c.ca_hq * dh, ckv = c.ca_hkv * dh;
+  {
+    const void* W1[1] = {w.ca_wq};
+    const int N1[1] = {cq};
+    MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
+    const size_t tot = (size_t)R * cq;
+    sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
+    MOA_CHECK_LAUNCH();
+  }
+  MOA_TRY(attention<T>(s, dh, narrow, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx, ckv,
+                       st->ca_len, 0, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, rows_per_seq, obuf));
+  {
+    const void* W1[1] = {w.ca_wo};
+    const int N1[1] = {E};
+    MOA_TRY(linear<T>(ctx, s, obuf, R, cq, 1, W1, N1, ws, p, &lo, status_word));
+  }
+  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_norm2, nullptr));
+  MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.ca_mlp, w.ca_wgate, w.ca_wup, w.ca_wdown, &lo, status_word));
 
   // ---- LM head, log-softmax, top-B ----
-  if (hidden_out) MOA_TRY(cast_flat<T>(s, xres, (T*)hidden_out, (size_t)R * E));
-  rmsnorm_rows_kernel<float, T><<<R, 256, 0, s>>>(xres, nullptr, 0, (const T*)w.final_norm, E, c.rms_eps, nullptr, xn);
-  MOA_CHECK_LAUNCH();
-  const bool timed = ctx->prof_on && ctx->prof_n < PROF_MAX;
-  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
-  MOA_TRY(gemm<T>(s, xn, w.lm_head, R, V, E, nullptr, 0, logits, V));
-  if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
-  lse_topk_rows_kernel<<<R, 256, 0, s>>>(logits, V, B, topk_id, topk_logp);
-  MOA_CHECK_LAUNCH();
-  return MOA_OK;
+  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.final_norm, hidden_out));
+  return lm_head_t<T>(ctx, s, ws, p, R, topk_id, topk_logp, status_word);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -355,6 +558,7 @@ static moa_status validate_config(const moa_config* c) {
   const int dims[] = {c->d_model, c->d_stack, c->lsa_mlp, c->sa_mlp, c->ca_mlp};
   for (int d : dims)
     if (d <= 0 || d % 16 != 0) return MOA_ERR_SHAPE;
+  if (c->dtype == MOA_BF16 && c->d_model % 64 != 0) return MOA_ERR_SHAPE;   // the fused LM head streams 64-wide k blocks
   if (c->n_stack <= 0 || c->vocab <= 0) return MOA_ERR_SHAPE;
   const int hq[] = {c->lsa_hq, c->sa_hq, c->ca_hq}, hkv[] = {c->lsa_hkv, c->sa_hkv, c->ca_hkv};
   for (int i = 0; i < 3; ++i)
@@ -364,6 +568,7 @@ static moa_status validate_config(const moa_config* c) {
   if (c->tree_topk <= 0 || c->tree_topk > MOA_MAX_TOPK || c->tree_topk > c->vocab) return MOA_ERR_SHAPE;
   if (c->tree_depth <= 0 || c->tree_depth > MOA_MAX_DEPTH) return MOA_ERR_SHAPE;
   if (c->tree_keep <= 0) return MOA_ERR_SHAPE;
+  if ((long long)c->max_batch * c->tree_topk > 256) return MOA_ERR_SHAPE;   // rows of one draft step
   if (!(c->rms_eps >= 0.f) || !(c->sa_rope_theta >= 0.f)) return MOA_ERR_SHAPE;
   return MOA_OK;
 }
@@ -396,6 +601,46 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
   ctx->prof_on = false;
   ctx->prof_n = 0;
   ctx->prof_made = false;
+  ctx->encode = nullptr;
+  ctx->n_wmap = 0;
+  ctx->fast = false;
+  if (cfg->dtype == MOA_BF16) {
+    // tensor maps of every weight matrix whose inner dimension the streaming GEMM can take
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_create: cuTensorMapEncodeTiled unavailable");
+      delete ctx;
+      return MOA_ERR_CUDA;
+    }
+    ctx->encode = (EncodeTiledFn)fn;
+    const int dh = cfg->head_dim, E = cfg->d_model, Din = cfg->d_stack;
+    struct { const void* p; int n, k; } mats[] = {
+        {w->lm_head, cfg->vocab, E},
+        {w->lsa_wq, cfg->lsa_hq * dh, Din}, {w->lsa_wk, cfg->lsa_hkv * dh, Din}, {w->lsa_wv, cfg->lsa_hkv * dh, Din},
+        {w->lsa_wo, Din, cfg->lsa_hq * dh}, {w->lsa_wgate, cfg->lsa_mlp, Din}, {w->lsa_wup, cfg->lsa_mlp, Din},
+        {w->lsa_wdown, Din, cfg->lsa_mlp},
+        {w->sa_wq, cfg->sa_hq * dh, E}, {w->sa_wk, cfg->sa_hkv * dh, E}, {w->sa_wv, cfg->sa_hkv * dh, E},
+        {w->sa_wo, E, cfg->sa_hq * dh}, {w->sa_wgate, cfg->sa_mlp, E}, {w->sa_wup, cfg->sa_mlp, E},
+        {w->sa_wdown, E, cfg->sa_mlp},
+        {w->ca_wq, cfg->ca_hq * dh, E}, {w->ca_wk, cfg->ca_hkv * dh, Din}, {w->ca_wv, cfg->ca_hkv * dh, Din},
+        {w->ca_wo, E, cfg->ca_hq * dh}, {w->ca_wgate, cfg->ca_mlp, E}, {w->ca_wup, cfg->ca_mlp, E},
+        {w->ca_wdown, E, cfg->ca_mlp}};
+    for (auto& m : mats) {
+      if (m.k % WS_BK != 0) continue;    // such a matrix takes the generic GEMM
+      WeightMap& wm = ctx->wmap[ctx->n_wmap];
+      wm.ptr = m.p;
+      wm.n = m.n;
+      wm.k = m.k;
+      if (!encode_map(ctx, &wm.tm, m.p, m.n, m.k, WS_BM)) {
+        delete ctx;
+        return MOA_ERR_CUDA;
+      }
+      ++ctx->n_wmap;
+    }
+    ctx->fast = true;
+  }
   *out = ctx;
   return MOA_OK;
 }
@@ -543,7 +788,7 @@ moa_status moa_sa_append(moa_ctx* ctx, moa_state* st, const int32_t* tok, const 
 moa_status moa_tree_begin(moa_ctx* ctx, moa_state* st, const int32_t* root_tok, int32_t batch, void* stream) {
   MOA_TRY(check_state(ctx, st, batch));
   if (!root_tok) return MOA_ERR_NULL;
-  for (int b = 0; b < batch; ++b)   // the deepest forwarded row sits at sa_len + D - 1; positions are not stored
+  for (int b = 0; b < batch; ++b)
     if (st->sa_len_host[b] < 0 || st->sa_len_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
   const TreePtrs tp = tree_ptrs(st->tree, ctx->tl);
   tree_begin_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(tp, root_tok, batch, ctx->c.max_batch * ctx->c.tree_topk,

@@ -101,28 +101,64 @@ __global__ void __launch_bounds__(256) gemm_fma_kernel(const T* __restrict__ A, 
 }
 
 // ---------------------------------------------------------------------------------------------
-// fp32 -> T, flat.
+// Glue between GEMMs. A GEMM leaves `splits` fp32 partial planes (`plane` elements apart, one per
+// K split); every consumer adds them in a fixed order, so results are deterministic.
 // ---------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void cast_flat_kernel(const float* __restrict__ x, T* __restrict__ y, size_t total) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < total) y[i] = from_f<T>(x[i]);
+__device__ __forceinline__ float sum_splits(const float* p, size_t plane, int splits) {
+  float s = 0.f;
+  for (int i = 0; i < splits; ++i) s += p[(size_t)i * plane];
+  return s;
 }
 
-// h = silu(gate) * up, fp32 in (two column blocks of one buffer), T out.
+// xres[r, :] += sum of partial planes [R, K]; then, if gain != nullptr, xn = RMSNorm(xres; gain) as T;
+// optionally also copies the updated xres to hidden_out as T. One block per row.
 template <typename T>
-__global__ void silu_mul_kernel(const float* __restrict__ gate, const float* __restrict__ up, int ld, int F,
-                                T* __restrict__ h, size_t total) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+__global__ void residual_norm_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
+                                     int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
+                                     T* __restrict__ hidden_out) {
+  __shared__ float red[33];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    float v = xres[(size_t)r * K + k];
+    if (part) v += sum_splits(part + (size_t)r * K + k, plane, splits);
+    xres[(size_t)r * K + k] = v;
+    ss += v * v;
+  }
+  if (gain == nullptr && hidden_out == nullptr) return;
+  ss = block_sum(ss, red);
+  const float rinv = rsqrtf(ss / (float)K + eps);
+  for (int k = threadIdx.x; k < K; k += blockDim.x) {
+    const float v = xres[(size_t)r * K + k];
+    if (hidden_out) hidden_out[(size_t)r * K + k] = from_f<T>(v);
+    if (gain) xn[(size_t)r * K + k] = from_f<T>(v * rinv * to_f<T>(gain[k]));
+  }
+}
+
+// h = silu(sum gate) * (sum up): a partial plane row holds [gate | up] (2F columns).
+template <typename T>
+__global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
+                                      T* __restrict__ h, size_t total) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
-  size_t r = i / F;
-  int c = (int)(i - r * F);
-  float g = gate[r * ld + c], u = up[r * ld + c];
+  const size_t r = i / F;
+  const int c = (int)(i - r * F);
+  const float g = sum_splits(part + r * 2 * F + c, plane, splits);
+  const float u = sum_splits(part + r * 2 * F + F + c, plane, splits);
   h[i] = from_f<T>(g / (1.f + __expf(-g)) * u);
 }
 
+// y = T(sum of planes), flat.
+template <typename T>
+__global__ void sum_cast_kernel(const float* __restrict__ part, int splits, size_t plane, size_t total,
+                                T* __restrict__ y) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < total) y[i] = from_f<T>(sum_splits(part + i, plane, splits));
+}
+
 // ---------------------------------------------------------------------------------------------
-// Rotary embedding + stores. One block per row.
+// Rotary embedding + stores. One block per row. The input may be `splits` partial planes (plane
+// elements apart) that are summed on the fly.
 //   q (optional): fp32 [R, hq*dh] at qkv + q_off (leading dim ld) -> rotated, T [R, hq*dh]
 //   k, v: fp32 [R, hkv*dh] -> k rotated; written as T to  kdst/vdst + dst_index(row) * hkv*dh
 // Row r sits at position pos_base[seq(r)] + pos_add(r). Angles are formed in double:
@@ -139,7 +175,8 @@ struct RopeRows {
 };
 
 template <typename T>
-__global__ void rope_store_kernel(const float* __restrict__ qkv, int ld, int q_off, int k_off, int v_off,
+__global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, size_t plane, int ld, int q_off, int k_off,
+                                  int v_off,
                                   int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
                                   RopeRows rr, T* __restrict__ qdst, T* __restrict__ kdst, T* __restrict__ vdst) {
   __shared__ float cs[64], sn[64];
@@ -172,27 +209,33 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int ld, int q_o
     }
   }
   __syncthreads();
-  const float* row = qkv + (size_t)r * ld;
+  const float* row0 = qkv + (size_t)r * ld;
+  auto row = [&](int c) {                 // the K-split partial planes are added in a fixed order
+    float a = 0.f;
+    for (int sp = 0; sp < splits; ++sp) a += row0[(size_t)sp * plane + c];
+    return a;
+  };
   if (qdst) {
     for (int i = threadIdx.x; i < hq * half; i += blockDim.x) {
       const int h = i / half, j = i - h * half;
-      const float x1 = row[q_off + h * dh + j], x2 = row[q_off + h * dh + half + j];
+      const float x1 = row(q_off + h * dh + j), x2 = row(q_off + h * dh + half + j);
       qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
       qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
     }
   }
   for (int i = threadIdx.x; i < hkv * half; i += blockDim.x) {
     const int h = i / half, j = i - h * half;
-    const float x1 = row[k_off + h * dh + j], x2 = row[k_off + h * dh + half + j];
+    const float x1 = row(k_off + h * dh + j), x2 = row(k_off + h * dh + half + j);
     kdst[dst * hkv * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
     kdst[dst * hkv * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
   }
-  for (int i = threadIdx.x; i < hkv * dh; i += blockDim.x) vdst[dst * hkv * dh + i] = from_f<T>(row[v_off + i]);
+  for (int i = threadIdx.x; i < hkv * dh; i += blockDim.x) vdst[dst * hkv * dh + i] = from_f<T>(row(v_off + i));
 }
 
 // Cross-attention cache append: fp32 [n, hkv*dh] k and v rows -> T cache rows at (seq, ca_len[seq] + i).
 template <typename T>
-__global__ void cache_append_kernel(const float* __restrict__ kv, int ld, int k_off, int v_off, int width,
+__global__ void cache_append_kernel(const float* __restrict__ kv, int splits, size_t plane, int ld, int k_off, int v_off,
+                                    int width,
                                     const int* __restrict__ len, int max_ctx, SeqSplit split, int row0,
                                     T* __restrict__ kdst, T* __restrict__ vdst) {
   const int r = blockIdx.x;
@@ -201,8 +244,13 @@ __global__ void cache_append_kernel(const float* __restrict__ kv, int ld, int k_
   const int i = t - split.off[seq];
   const size_t dst = ((size_t)seq * max_ctx + len[seq] + i) * width;
   for (int c = threadIdx.x; c < width; c += blockDim.x) {
-    kdst[dst + c] = from_f<T>(kv[(size_t)r * ld + k_off + c]);
-    vdst[dst + c] = from_f<T>(kv[(size_t)r * ld + v_off + c]);
+    float a = 0.f, b = 0.f;
+    for (int sp = 0; sp < splits; ++sp) {
+      a += kv[(size_t)sp * plane + (size_t)r * ld + k_off + c];
+      b += kv[(size_t)sp * plane + (size_t)r * ld + v_off + c];
+    }
+    kdst[dst + c] = from_f<T>(a);
+    vdst[dst + c] = from_f<T>(b);
   }
 }
 
@@ -221,11 +269,14 @@ __global__ void set_len_kernel(int* len, LenVals lv) {
 // Key set = segment A: keys 0..nA-1 of sequence `seq` in a cache [n_seq, capA, hkv, dh]
 //         + segment B: nB listed slots of a second cache [n_seq, capB, hkv, dh] (tree nodes).
 // Row -> sequence: seq = r / rows_per_seq. nA = lenA ? lenA[seq] : nA_fixed.
+// q_ld: elements between query rows; posA_ld: elements between consecutive positions of segment A
+// (hkv*dh for a dense cache; larger when k and v sit inside wider rows).
 // Each warp walks keys warp, warp+4, ...; a lane owns dh/32 consecutive elements.
 // ---------------------------------------------------------------------------------------------
 template <typename T, int DH>
-__global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q, int hq, int hkv,
+__global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q, int q_ld, int hq, int hkv,
                                                         const T* __restrict__ kA, const T* __restrict__ vA, int capA,
+                                                        int posA_ld,
                                                         const int* __restrict__ lenA, int nA_fixed,
                                                         const T* __restrict__ kB, const T* __restrict__ vB, int capB,
                                                         const int* __restrict__ slotsB, int slots_ld, int nB,
@@ -240,7 +291,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
   const float scale = rsqrtf((float)DH);
   float qv[VEC];
 #pragma unroll
-  for (int e = 0; e < VEC; ++e) qv[e] = to_f<T>(q[((size_t)r * hq + h) * DH + lane * VEC + e]) * scale;
+  for (int e = 0; e < VEC; ++e) qv[e] = to_f<T>(q[(size_t)r * q_ld + h * DH + lane * VEC + e]) * scale;
   float m = -INFINITY, l = 0.f, acc[VEC];
 #pragma unroll
   for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
@@ -248,7 +299,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
   for (int j = warp; j < n; j += 4) {
     const T *kp, *vp;
     if (j < nA) {
-      const size_t o = (((size_t)seq * capA + j) * hkv + g) * DH + lane * VEC;
+      const size_t o = ((size_t)seq * capA + j) * posA_ld + g * DH + lane * VEC;
       kp = kA + o;
       vp = vA + o;
     } else {

@@ -1,0 +1,453 @@
+// Weight-streaming GEMM for sm_100a:  Y^T[n, r] = sum_k W[n, k] * X[r, k]   (bf16 in, fp32 accumulate)
+//
+// The weight matrix is the big operand: it is streamed from HBM exactly once per call, 128 rows x 64
+// columns (16 KB) per pipeline stage, by TMA into 128B-swizzled shared memory, and fed to the 5th-gen
+// tensor cores as the A operand (M = 128) of tcgen05.mma. The R activation rows (R <= 256 per call) are
+// the B operand (N = R padded to 16/32/64/128/256), re-fetched from L2 next to each weight tile.
+// Accumulators live in TMEM, double-buffered so that the epilogue of one tile overlaps the MMAs of the
+// next. One CTA per SM, persistent over work units (weight tile x K split), 6 warps:
+//   warp 0     : TMA producer (one lane)
+//   warp 1     : TMEM allocation + MMA issue (one lane)
+//   warps 2..5 : epilogue, one TMEM lane quadrant each
+// Epilogues:
+//   mode 0: fp32 partial sums, out[split][r][col0 + n]  (the consumer adds the splits in a fixed order,
+//           so results are deterministic and need no atomics or zero-filled buffers)
+//   mode 1: LM head -- per 32 vocabulary rows and per activation row: max, sum of exponentials and
+//           the B largest logits with their ids, sorted; the logits never go to HBM (Eq. 1 + top-B).
+// Every mbarrier wait is bounded: on expiry the CTA raises an abort flag, drains, frees TMEM, writes
+// DEV_ERR_TIMEOUT to the status word and returns.
+#pragma once
+#include <cuda.h>
+
+#include "moa_common.cuh"
+
+namespace moa {
+
+constexpr int WS_BM = 128;         // weight rows per tile (MMA M)
+constexpr int WS_BK = 64;          // k elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int WS_THREADS = 192;
+constexpr int WS_W_BYTES = WS_BM * WS_BK * 2;
+constexpr int WS_SMEM_BUDGET = 200 * 1024;
+constexpr long long WS_WAIT_CYCLES = 4000000000ll;   // ~2 s at boost clock
+
+struct WsParams {
+  CUtensorMap tmW[3];      // weight matrices [n_i, K], box 64 x 128, swizzle 128B
+  CUtensorMap tmX;         // activations [R, K], box 64 x NPAD, swizzle 128B, rows >= R read as zero
+  int n_seg;
+  int seg_n[3];            // rows of each weight matrix
+  int seg_tile0[3];        // first tile index of each segment
+  int seg_col[3];          // first output column of each segment
+  int tiles_total;
+  int R;                   // valid activation rows
+  int kb_total;            // K / 64
+  int splits;              // K splits per tile
+  int mode;                // 0: fp32 partials, 1: LM-head partial top-B
+  int ldo;                 // mode 0: columns of one partial plane
+  float* out;              // mode 0: plane `split` starts at out + split * plane; row r, column c at [r * ldo + c]
+  size_t plane;            // mode 0: elements between two partial planes
+  int B;                   // mode 1
+  float* p_max;            // mode 1: [4*tiles][R]
+  float* p_sum;            //         [4*tiles][R]
+  float* c_val;            //         [4*tiles][R][B]
+  int* c_id;               //         [4*tiles][R][B]
+  int* status;             // device status word (may be nullptr)
+};
+
+__host__ __device__ constexpr int ws_stage_bytes(int npad) { return WS_W_BYTES + npad * WS_BK * 2; }
+__host__ __device__ constexpr int ws_stages(int npad) {
+  return (WS_SMEM_BUDGET / ws_stage_bytes(npad)) > 12 ? 12 : (WS_SMEM_BUDGET / ws_stage_bytes(npad));
+}
+__host__ __device__ constexpr int ws_smem_bytes(int npad) { return ws_stages(npad) * ws_stage_bytes(npad) + 1024 + 256; }
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false when the abort flag is up or the time limit passed (and raises the flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if ((spin & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WS_WAIT_CYCLES) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as 128-byte rows with the 128B swizzle:
+// 8-row groups lie 1024 bytes apart (stride byte offset), the leading byte offset is unused.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: D = fp32, A = B = bf16, both K-major, M = 128, N = npad.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ bool ranks_before(float va, int ia, float vb, int ib) {
+  return va > vb || (va == vb && ia < ib);
+}
+
+// ---------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------
+template <int NPAD>
+__global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __grid_constant__ WsParams P) {
+  constexpr int STAGES = ws_stages(NPAD);
+  constexpr int STAGE_BYTES = ws_stage_bytes(NPAD);
+  constexpr uint32_t TMEM_COLS = (2 * NPAD) < 32 ? 32 : (2 * NPAD);
+  constexpr uint32_t IDESC = umma_idesc_bf16(WS_BM, NPAD);
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzled tiles need 1024-byte alignment
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = (uint64_t*)(base_ptr + STAGES * STAGE_BYTES);      // full[STAGES], empty[STAGES], tfull[2], tempty[2]
+  const uint32_t bar0 = base + STAGES * STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int units = P.tiles_total * P.splits;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // unit -> (tile, split) -> (segment, first weight row, k-block range)
+  auto decode = [&](int u, int& seg, int& n0, int& kb0, int& kb1, int& split, int& tile) {
+    tile = u / P.splits;
+    split = u - tile * P.splits;
+    seg = 0;
+    if (P.n_seg > 1 && tile >= P.seg_tile0[1]) seg = 1;
+    if (P.n_seg > 2 && tile >= P.seg_tile0[2]) seg = 2;
+    n0 = (tile - P.seg_tile0[seg]) * WS_BM;
+    kb0 = (int)(((long long)split * P.kb_total) / P.splits);
+    kb1 = (int)(((long long)(split + 1) * P.kb_total) / P.splits);
+  };
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int seg, n0, kb0, kb1, split, tile;
+        decode(u, seg, n0, kb0, kb1, split, tile);
+        const CUtensorMap* tw = &P.tmW[seg];
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          const uint32_t dst = base + s * STAGE_BYTES;
+          tma_load_2d(dst, tw, kb * WS_BK, n0, full_bar(s));
+          tma_load_2d(dst + WS_W_BYTES, &P.tmX, kb * WS_BK, 0, full_bar(s));
+        }
+      }
+      if (!ok) {
+        // give the copies already issued a bounded time to land before the CTA tears down
+        const uint32_t pending = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+        for (uint32_t j = 0; j < pending; ++j) {
+          const uint32_t i2 = it - 1 - j;
+          const long long t0 = clock64();
+          while (!mbar_try(full_bar(i2 % STAGES), (i2 / STAGES) & 1u) && clock64() - t0 < 20000000ll) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      int j = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++j) {
+        int seg, n0, kb0, kb1, split, tile;
+        decode(u, seg, n0, kb0, kb1, split, tile);
+        const int buf = j & 1;
+        const uint32_t bph = (uint32_t)(j >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NPAD);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t wa = base + s * STAGE_BYTES;
+          const uint64_t adesc = umma_desc_sw128(wa);
+          const uint64_t bdesc = umma_desc_sw128(wa + WS_W_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < WS_BK / 16; ++kk) {
+            // advancing 16 k-elements = 32 bytes inside the swizzled row: +2 in the descriptor's 16-byte units
+            tc_mma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, IDESC, (kb > kb0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));       // frees the stage once these MMAs have read it
+        }
+        if (ok) tc_commit(tfull_bar(buf));
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    int j = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++j) {
+      int seg, n0, kb0, kb1, split, tile;
+      decode(u, seg, n0, kb0, kb1, split, tile);
+      const int buf = j & 1;
+      const uint32_t bph = (uint32_t)(j >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(buf), bph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int nrow = n0 + q * 32 + lane;                  // weight row inside the segment
+      const bool valid = nrow < P.seg_n[seg];
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * NPAD);
+      if (P.mode == 0) {
+        float* plane = P.out + (size_t)split * P.plane + P.seg_col[seg] + nrow;
+#pragma unroll 1
+        for (int c0 = 0; c0 < NPAD; c0 += 16) {
+          if (c0 >= P.R) break;
+          float v[16];
+          tc_ld16(taddr + c0, v);
+          if (valid) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (c0 + i < P.R) plane[(size_t)(c0 + i) * P.ldo] = v[i];
+          }
+        }
+      } else {
+        const int sub = tile * 4 + q;                         // 32-row vocabulary slice
+        const int B = P.B;
+#pragma unroll 1
+        for (int c0 = 0; c0 < NPAD; c0 += 16) {
+          if (c0 >= P.R) break;
+          float v[16];
+          tc_ld16(taddr + c0, v);
+#pragma unroll 1
+          for (int i = 0; i < 16; ++i) {
+            const int r = c0 + i;
+            if (r >= P.R) break;
+            float val = valid ? v[i] : -INFINITY;
+            int id = nrow;
+            const float wmax = warp_max(val);
+            const float e = (valid && wmax > -INFINITY) ? __expf(val - wmax) : 0.f;
+            const float wsum = warp_sum(e);
+            // bitonic sort of the 32 (value, id) pairs: best (largest value, then smallest id) ends in lane 0
+#pragma unroll
+            for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+              for (int jj = k >> 1; jj > 0; jj >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, val, jj);
+                const int oi = __shfl_xor_sync(0xffffffffu, id, jj);
+                const bool lower = (lane & jj) == 0;
+                const bool up = (lane & k) == 0;
+                const bool want_better = lower == up;
+                const bool other_better = ranks_before(ov, oi, val, id);
+                if (want_better == other_better) { val = ov; id = oi; }
+              }
+            }
+            if (lane < B) {
+              P.c_val[((size_t)sub * P.R + r) * B + lane] = val;
+              P.c_id[((size_t)sub * P.R + r) * B + lane] = id;
+            }
+            if (lane == 0) {
+              P.p_max[(size_t)sub * P.R + r] = wmax;
+              P.p_sum[(size_t)sub * P.R + r] = wsum;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(buf));
+    }
+  }
+
+  // ------------------------------ teardown ------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && P.status) atomicMax(P.status, DEV_ERR_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------------------------
+// LM-head merge: one block per activation row combines the per-slice partials into
+// logsumexp and the global top-B, ordered by (log-probability descending, id ascending).
+// ---------------------------------------------------------------------------------------------
+constexpr int MERGE_THREADS = 1024;
+constexpr int MERGE_MAXB = 16;
+
+__global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __restrict__ p_max,
+                                                                 const float* __restrict__ p_sum,
+                                                                 const float* __restrict__ c_val,
+                                                                 const int* __restrict__ c_id, int n_sub, int R, int B,
+                                                                 int* __restrict__ ids, float* __restrict__ logp) {
+  __shared__ float red[33];
+  __shared__ float w_val[32][MERGE_MAXB];
+  __shared__ int w_id[32][MERGE_MAXB];
+  const int r = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // logsumexp over all slices
+  float m = -INFINITY;
+  for (int s = tid; s < n_sub; s += MERGE_THREADS) m = fmaxf(m, p_max[(size_t)s * R + r]);
+  m = block_max(m, red);
+  float se = 0.f;
+  for (int s = tid; s < n_sub; s += MERGE_THREADS) {
+    const float pm = p_max[(size_t)s * R + r];
+    if (pm > -INFINITY) se += p_sum[(size_t)s * R + r] * __expf(pm - m);
+  }
+  se = block_sum(se, red);
+  const float lse = m + logf(se);
+  // thread-local top-B over this thread's slices (each slice list is already sorted)
+  float tv[MERGE_MAXB];
+  int ti[MERGE_MAXB];
+#pragma unroll
+  for (int i = 0; i < MERGE_MAXB; ++i) { tv[i] = -INFINITY; ti[i] = 0x7fffffff; }
+  for (int s = tid; s < n_sub; s += MERGE_THREADS) {
+    const float* cv = c_val + ((size_t)s * R + r) * B;
+    const int* ci = c_id + ((size_t)s * R + r) * B;
+    for (int c = 0; c < B; ++c) {
+      const float v = cv[c];
+      const int id = ci[c];
+      if (!ranks_before(v, id, tv[B - 1], ti[B - 1])) break;   // sorted list: the rest ranks lower still
+      // insert into the sorted local list
+      float nv = v;
+      int ni = id;
+#pragma unroll
+      for (int i = 0; i < MERGE_MAXB; ++i) {
+        if (i < B && ranks_before(nv, ni, tv[i], ti[i])) {
+          const float sv = tv[i]; const int si = ti[i];
+          tv[i] = nv; ti[i] = ni;
+          nv = sv; ni = si;
+        }
+      }
+    }
+  }
+  // warp level: B rounds of arg-best over the 32 thread heads
+  int head = 0;
+  for (int round = 0; round < B; ++round) {
+    float hv = -INFINITY;
+    int hi = 0x7fffffff;
+#pragma unroll
+    for (int i = 0; i < MERGE_MAXB; ++i)
+      if (i == head) { hv = tv[i]; hi = ti[i]; }
+    float bv = hv;
+    int bi = hi;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ranks_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    }
+    if (hi == bi && hv == bv && bi != 0x7fffffff) ++head;
+    if (lane == 0) { w_val[wid][round] = bv; w_id[wid][round] = bi; }
+  }
+  __syncthreads();
+  // block level: warp 0 merges the 32 sorted warp lists the same way
+  if (wid == 0) {
+    int h2 = 0;
+    for (int round = 0; round < B; ++round) {
+      const float hv = h2 < B ? w_val[lane][h2] : -INFINITY;
+      const int hi = h2 < B ? w_id[lane][h2] : 0x7fffffff;
+      float bv = hv;
+      int bi = hi;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ranks_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      if (hi == bi && hv == bv && bi != 0x7fffffff) ++h2;
+      if (lane == 0) {
+        ids[(size_t)r * B + round] = bi == 0x7fffffff ? -1 : bi;
+        logp[(size_t)r * B + round] = bv - lse;
+      }
+    }
+  }
+}
+
+}  // namespace moa
