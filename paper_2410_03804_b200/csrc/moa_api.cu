@@ -6,6 +6,7 @@
 #include <string.h>
 #include <new>
 
+#include "moa_attn.cuh"
 #include "moa_basic.cuh"
 #include "moa_tree.cuh"
 #include "moa_wstream.cuh"
@@ -49,8 +50,9 @@ struct moa_ctx {
 // workspace carving (same arithmetic in moa_state_bytes and in the calls)
 // ---------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, total;
+  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, total;
   int rows_cap, draft_rows, chunk_tok, part_rows, wide;
+  long long att_units;   // (row, head, part) triples the split-attention partial buffers hold
 };
 
 static inline int imax(int a, int b) { return a > b ? a : b; }
@@ -85,6 +87,10 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   p.cid = take(n_sub * p.draft_rows * c.tree_topk * sizeof(int));
   p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));   // LSA output rows, fp32
   p.kvn = take((size_t)chunk_tok * c.d_stack * elt);             // their normalised copy, T
+  const int gmax = imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), hqmax = imax(c.sa_hq, c.ca_hq);
+  p.att_units = (long long)c.tree_topk * gmax * 2 * 160 + 2ll * p.draft_rows * hqmax;
+  p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
+  p.att_ml = take(elt == 2 ? (size_t)p.att_units * 2 * sizeof(float) : 256);           // their (max, sum)
   p.total = o;
   return p;
 }
@@ -255,11 +261,65 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
   return MOA_OK;
 }
 
+template <int DH>
+static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nseq, int nwarps) {
+  static bool attr_set = false;
+  const int smem = nwarps * 16 * DH * 2 + 4 * AT_KB * DH * 2;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         8 * 16 * DH * 2 + 4 * AT_KB * DH * 2);
+    if (e != cudaSuccess) {
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+      return MOA_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  dim3 grid(P.n_parts, P.hkv * P.q_tiles, nseq);
+  attn_split_kernel<DH><<<grid, nwarps * 32, smem, s>>>(P);
+  MOA_CHECK_LAUNCH();
+  if (P.n_parts > 1) {
+    attn_combine_kernel<DH><<<nseq * P.rows_per_seq * P.hq, DH, 0, s>>>(P.part_o, P.part_ml, P.n_parts, P.out);
+    MOA_CHECK_LAUNCH();
+  }
+  return MOA_OK;
+}
+
+// softmax(q K^T / sqrt(dh)) V for R = nseq * rows_per_seq query rows. Segment A: a cache (or the LSA rows
+// themselves) with max_len positions at most on the host's count; segment B: tree slots masked per row.
 template <typename T>
-static moa_status attention(cudaStream_t s, int dh, const T* q, int q_ld, int R, int hq, int hkv, const T* kA,
-                            const T* vA, int capA, int posA_ld, const int* lenA, int nA_fixed, const T* kB, const T* vB,
-                            int capB, const int* slotsB, int slots_ld, int nB, int rows_per_seq, T* out) {
+static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int dh, const T* q, int q_ld,
+                            int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
+                            int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
+                            int slots_ld, int nB, int n_slots, int rows_per_seq, T* out) {
   if (R <= 0) return MOA_OK;
+  if (sizeof(T) == 2) {
+    AttnParams P;
+    memset(&P, 0, sizeof(P));
+    const int nseq = R / rows_per_seq;
+    P.q = (const bf16*)q; P.q_ld = q_ld;
+    P.hq = hq; P.hkv = hkv; P.group = hq / hkv;
+    P.rows_per_seq = rows_per_seq;
+    P.kA = (const bf16*)kA; P.vA = (const bf16*)vA; P.capA = capA; P.posA_ld = posA_ld;
+    P.lenA = lenA; P.nA_fixed = nA_fixed;
+    P.kB = (const bf16*)kB; P.vB = (const bf16*)vB; P.capB = capB;
+    P.slotsB = slotsB; P.slots_ld = slots_ld; P.nB = nB; P.n_slots = n_slots;
+    const int Qn = rows_per_seq * P.group;
+    const int nwarps = imin(8, (Qn + 15) / 16);
+    P.q_tiles = (Qn + nwarps * 16 - 1) / (nwarps * 16);
+    const int has_tree = (kB != nullptr && nB > 0) ? 1 : 0;
+    const int blocks = imax(1, (max_len + AT_KB - 1) / AT_KB);
+    int n_split = imax(1, imin(blocks, (2 * ctx->sm_count) / imax(1, nseq * hkv * P.q_tiles)));
+    const long long per_part = (long long)R * hq;
+    while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
+    if (per_part * (n_split + has_tree) > p.att_units && n_split + has_tree > 1) return MOA_ERR_WORKSPACE;
+    P.n_split = n_split;
+    P.n_parts = n_split + has_tree;
+    P.part_o = (float*)(ws + p.att_o);
+    P.part_ml = (float*)(ws + p.att_ml);
+    P.out = (bf16*)out;
+    P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    return dh == 128 ? launch_attn_split<128>(s, P, nseq, nwarps) : launch_attn_split<64>(s, P, nseq, nwarps);
+  }
   dim3 grid(R, hq);
   if (dh == 128)
     attn_rows_kernel<T, 128><<<grid, 128, 0, s>>>(q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
@@ -276,6 +336,13 @@ template <typename T>
 static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, const Workspace& p, int R, int K,
                                 const LinOut* lo, const void* gain, void* hidden_out) {
   if (R <= 0) return MOA_OK;
+  if (K % RN_CLUSTER == 0 && K / RN_CLUSTER <= 256 * RN_MAX_PER_THREAD) {
+    residual_norm_cluster_kernel<T><<<dim3(RN_CLUSTER, R), 256, 0, s>>>(
+        (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0, lo ? lo->plane : 0, K, (const T*)gain,
+        ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out);
+    MOA_CHECK_LAUNCH();
+    return MOA_OK;
+  }
   residual_norm_kernel<T><<<R, 256, 0, s>>>((float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0,
                                             lo ? lo->plane : 0, K, (const T*)gain, ctx->c.rms_eps, (T*)(ws + p.xn),
                                             (T*)hidden_out);
@@ -338,8 +405,8 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
       MOA_CHECK_LAUNCH();
     }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
-    MOA_TRY(attention<T>(s, dh, narrow, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld, nullptr, S,
-                         (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, S, obuf));
+    MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld,
+                         nullptr, S, S, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0, S, obuf));
     // out-projection + residual, MLP + residual
     const void* W1[1] = {w.lsa_wo};
     const int N1[1] = {D};
@@ -349,7 +416,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, D, &lo, nullptr, nullptr));
     // mean over layers
     T* kvo = kv_out ? (T*)kv_out + (size_t)t0 * D : nullptr;
-    mean_layers_kernel<T><<<nt, 256, 0, s>>>(xres, S, D, kvf, kvo);
+    mean_layers_kernel<T><<<dim3(nt, (D + 255) / 256), 256, 0, s>>>(xres, S, D, kvf, kvo);
     MOA_CHECK_LAUNCH();
     // cross-attention keys / values of the new positions, appended to the cache
     rmsnorm_rows_kernel<float, T><<<nt, 256, 0, s>>>(kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn);
@@ -391,7 +458,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
     rr.max_ctx = c.max_ctx;
     rr.split = split;
     rr.row0 = t0;
-    rope_store_kernel<T><<<R, 128, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
+    rope_store_kernel<T><<<dim3(R, 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
                                            c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
     MOA_CHECK_LAUNCH();
   }
@@ -489,11 +556,17 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   rr.step = step;
   rr.B = B;
   rr.slots = L.NS;
-  rope_store_kernel<T><<<R, 128, 0, s>>>(lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
+  rope_store_kernel<T><<<dim3(R, c.sa_hq + 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
                                          dh, c.sa_rope_theta, st->sa_len, rr, narrow, tk, tv);
   MOA_CHECK_LAUNCH();
-  MOA_TRY(attention<T>(s, dh, narrow, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v, c.max_ctx, nkv,
-                       st->sa_len, 0, tk, tv, L.NS, row_anc, D, step + 1, rows_per_seq, obuf));
+  int max_sa = 0, max_ca = 0;
+  for (int b = 0; b < batch; ++b) {
+    max_sa = imax(max_sa, st->sa_len_host[b]);
+    max_ca = imax(max_ca, st->ca_len_host[b]);
+  }
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
+                       c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
+                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
   {
     const void* W1[1] = {w.sa_wo};
     const int N1[1] = {E};
@@ -513,8 +586,9 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
     MOA_CHECK_LAUNCH();
   }
-  MOA_TRY(attention<T>(s, dh, narrow, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx, ckv,
-                       st->ca_len, 0, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, rows_per_seq, obuf));
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,
+                       c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0,
+                       rows_per_seq, obuf));
   {
     const void* W1[1] = {w.ca_wo};
     const int N1[1] = {E};

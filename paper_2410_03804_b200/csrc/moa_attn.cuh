@@ -1,0 +1,295 @@
+// Split-KV attention for the drafter's three attentions on the bf16 path (sm_100a).
+//
+// One CTA = one (sequence, kv head, query tile, key split). All query vectors that share a kv head --
+// (rows of the sequence) x (query heads of the group) -- are stacked into the M dimension of
+// mma.sync.m16n8k16 (16 queries per warp), so every cached key / value byte is read from HBM once per
+// sequence and kv head whatever the number of tree rows or grouped heads. Keys and values stream
+// through shared memory in blocks of 64 positions (cp.async, two stages, XOR-swizzled 16-byte chunks,
+// ldmatrix); scores, softmax statistics and the output accumulate in fp32 (flash-style online softmax,
+// probabilities rounded to bf16 for the P.V product).
+//
+// Key set of a row = segment A: positions 0..len-1 of a cache  [seq, capA, (posA_ld)]  (unmasked)
+//                  + segment B: the sequence's tree slots, masked per row by its ancestor list.
+// Splits 0..n_split-1 cover segment A; one more part (index n_split) covers segment B when present.
+// With a single part the normalised output is written directly; otherwise each part leaves
+// (max, sum, unnormalised output) and attn_combine_kernel merges them.
+#pragma once
+#include "moa_common.cuh"
+
+namespace moa {
+
+constexpr int AT_KB = 64;        // keys per block
+
+struct AttnParams {
+  const bf16* q; int q_ld;               // query row r, head h at q + r*q_ld + h*DH
+  int hq, hkv, group;                    // group = hq / hkv
+  int rows_per_seq;                      // query rows of one sequence (tree rows, or LSA layers)
+  const bf16* kA; const bf16* vA; int capA; int posA_ld;   // segment A: (seq*capA + j)*posA_ld + g*DH
+  const int* lenA; int nA_fixed;         // valid positions: lenA[seq] or the fixed count
+  const bf16* kB; const bf16* vB; int capB;                // segment B: ((seq*capB + slot)*hkv + g)*DH
+  const int* slotsB; int slots_ld; int nB; int n_slots;    // row's ancestor slots [nB]; slots in use
+  int n_split;                           // splits of segment A
+  int n_parts;                           // n_split + (segment B ? 1 : 0)
+  int q_tiles;                           // query tiles per (seq, kv head)
+  float* part_o; float* part_ml;         // [R*hq][n_parts][DH], [R*hq][n_parts][2]
+  bf16* out;                             // [R, hq*DH]
+  float scale_log2;                      // log2(e) / sqrt(DH)
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+  const int sz = valid ? 16 : 0;         // zero-fills the 16 bytes when the source row does not exist
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Byte offset of (row, 16-byte chunk) in a tile of DH-wide bf16 rows, chunks XOR-swizzled by the row.
+template <int DH>
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  return (uint32_t)(row * (DH * 2) + ((chunk ^ (row & 7)) << 4));
+}
+
+template <int DH>
+__global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
+  constexpr int CH = DH / 8;                 // 16-byte chunks per row
+  constexpr int KS = DH / 16;                // k-steps of the Q.K^T product
+  constexpr int TILE_BYTES = AT_KB * DH * 2;
+  extern __shared__ __align__(128) uint8_t at_smem[];
+  __shared__ unsigned long long allow[16][4];     // per sequence row: bit per tree slot (<= 256 slots)
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int part = blockIdx.x;
+  const int g = blockIdx.y / P.q_tiles, qt = blockIdx.y - g * P.q_tiles;
+  const int seq = blockIdx.z;
+  const int QT = nwarps * 16;                // queries per tile
+  const int Qn = P.rows_per_seq * P.group;   // queries per (seq, kv head)
+  const uint32_t sQ = smem_u32(at_smem);
+  const uint32_t sKV = sQ + QT * DH * 2;     // [2 stages][K tile | V tile]
+
+  const bool tree_part = part >= P.n_split;
+  // key range of this part
+  int k_begin, k_end;
+  if (!tree_part) {
+    const int len = P.lenA ? P.lenA[seq] : P.nA_fixed;
+    const int blocks = (len + AT_KB - 1) / AT_KB;
+    const int b0 = (int)(((long long)part * blocks) / P.n_split), b1 = (int)(((long long)(part + 1) * blocks) / P.n_split);
+    k_begin = b0 * AT_KB;
+    k_end = min(b1 * AT_KB, len);
+  } else {
+    k_begin = 0;
+    k_end = P.n_slots;
+    if (threadIdx.x < 64) allow[threadIdx.x >> 2][threadIdx.x & 3] = 0ull;
+    __syncthreads();
+    if (threadIdx.x < P.rows_per_seq && threadIdx.x < 16) {
+      const int r = seq * P.rows_per_seq + threadIdx.x;
+      for (int i = 0; i < P.nB; ++i) {
+        const int slot = P.slotsB[(size_t)r * P.slots_ld + i];
+        if (slot >= 0 && slot < 256) allow[threadIdx.x][slot >> 6] |= 1ull << (slot & 63);
+      }
+    }
+  }
+
+  // ---- Q tile -> shared (zero rows for queries beyond Qn) ----
+  for (int i = threadIdx.x; i < QT * CH; i += blockDim.x) {
+    const int ql = i / CH, c = i - ql * CH;
+    const int qi = qt * QT + ql;
+    const bool valid = qi < Qn;
+    const int row = seq * P.rows_per_seq + (valid ? qi / P.group : 0);
+    const int head = g * P.group + (valid ? qi % P.group : 0);
+    cp_async16(sQ + tile_off<DH>(ql, c), P.q + (size_t)row * P.q_ld + head * DH + c * 8, valid);
+  }
+  cp_async_commit();
+
+  auto load_block = [&](int stage, int k0) {
+    const uint32_t sK = sKV + stage * 2 * TILE_BYTES, sV = sK + TILE_BYTES;
+    for (int i = threadIdx.x; i < AT_KB * CH; i += blockDim.x) {
+      const int kr = i / CH, c = i - kr * CH;
+      const int j = k0 + kr;
+      const bool valid = j < k_end;
+      size_t off;
+      if (!tree_part) off = ((size_t)seq * P.capA + (valid ? j : 0)) * P.posA_ld + g * DH + c * 8;
+      else off = (((size_t)seq * P.capB + (valid ? j : 0)) * P.hkv + g) * DH + c * 8;
+      cp_async16(sK + tile_off<DH>(kr, c), (tree_part ? P.kB : P.kA) + off, valid);
+      cp_async16(sV + tile_off<DH>(kr, c), (tree_part ? P.vB : P.vA) + off, valid);
+    }
+  };
+
+  const int n_blocks = (k_end - k_begin + AT_KB - 1) / AT_KB;
+  if (n_blocks > 0) load_block(0, k_begin);
+  cp_async_commit();
+  cp_async_wait<1>();            // Q has landed
+  __syncthreads();
+
+  // ---- Q fragments of this warp's 16 queries ----
+  uint32_t qf[KS][4];
+  {
+    const int row = warp * 16 + (lane & 15);
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks)
+      ldsm_x4(sQ + tile_off<DH>(row, ks * 2 + (lane >> 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+  }
+  const int gq = lane >> 2, tq = lane & 3;
+  // the two query rows of this thread: warp*16 + gq and + 8
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+  float o[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  int seqrow[2];                 // sequence-local row of each query (for the tree mask)
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int qi = qt * QT + warp * 16 + gq + 8 * h;
+    seqrow[h] = qi < Qn ? qi / P.group : 0;
+  }
+
+  for (int blk = 0; blk < n_blocks; ++blk) {
+    const int stage = blk & 1;
+    if (blk + 1 < n_blocks) load_block(stage ^ 1, k_begin + (blk + 1) * AT_KB);
+    cp_async_commit();
+    cp_async_wait<1>();          // block `blk` has landed
+    __syncthreads();
+    const uint32_t sK = sKV + stage * 2 * TILE_BYTES, sV = sK + TILE_BYTES;
+    const int k0 = k_begin + blk * AT_KB;
+
+    // S = Q K^T over the block's 64 keys: 8 n-tiles of 8 keys
+    float s[AT_KB / 8][4];
+#pragma unroll
+    for (int nt = 0; nt < AT_KB / 8; ++nt) {
+      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+      for (int ks2 = 0; ks2 < KS / 2; ++ks2) {
+        uint32_t b0, b1, b2, b3;       // two k-steps: chunks 4*ks2 .. 4*ks2+3 of key row nt*8 + lane%8
+        ldsm_x4(sK + tile_off<DH>(nt * 8 + (lane & 7), ks2 * 4 + (lane >> 3)), b0, b1, b2, b3);
+        mma_bf16_16816(s[nt], qf[2 * ks2], b0, b1);
+        mma_bf16_16816(s[nt], qf[2 * ks2 + 1], b2, b3);
+      }
+    }
+    // scale, mask, block row max
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < AT_KB / 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = k0 + nt * 8 + tq * 2 + (e & 1);
+        const int h = e >> 1;
+        bool ok = key < k_end;
+        if (tree_part && ok) ok = (allow[seqrow[h]][key >> 6] >> (key & 63)) & 1ull;
+        const float v = ok ? s[nt][e] * P.scale_log2 : -INFINITY;
+        s[nt][e] = v;
+        mx[h] = fmaxf(mx[h], v);
+      }
+    }
+    float corr[2], msub[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+      mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+      const float mn = fmaxf(m_run[h], mx[h]);
+      corr[h] = (m_run[h] == -INFINITY) ? 0.f : exp2f(m_run[h] - mn);
+      msub[h] = (mn == -INFINITY) ? 0.f : mn;      // a fully masked row keeps p = exp2(-inf) = 0
+      m_run[h] = mn;
+    }
+    float rs[2] = {0.f, 0.f};
+    uint32_t pf[AT_KB / 16][4];
+#pragma unroll
+    for (int nt = 0; nt < AT_KB / 8; ++nt) {
+      const float p0 = exp2f(s[nt][0] - msub[0]), p1 = exp2f(s[nt][1] - msub[0]);
+      const float p2 = exp2f(s[nt][2] - msub[1]), p3 = exp2f(s[nt][3] - msub[1]);
+      rs[0] += p0 + p1;
+      rs[1] += p2 + p3;
+      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) l_run[h] = l_run[h] * corr[h] + rs[h];
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) {
+      o[i][0] *= corr[0]; o[i][1] *= corr[0];
+      o[i][2] *= corr[1]; o[i][3] *= corr[1];
+    }
+    // O += P V: k-steps of 16 keys, n-tiles of 8 output columns (two per ldmatrix)
+#pragma unroll
+    for (int kk = 0; kk < AT_KB / 16; ++kk) {
+#pragma unroll
+      for (int n2 = 0; n2 < DH / 16; ++n2) {
+        uint32_t b0, b1, b2, b3;
+        const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        ldsm_x4_t(sV + tile_off<DH>(key, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
+        mma_bf16_16816(o[2 * n2], pf[kk], b0, b1);
+        mma_bf16_16816(o[2 * n2 + 1], pf[kk], b2, b3);
+      }
+    }
+    __syncthreads();             // the stage may be overwritten by the next prefetch
+  }
+  cp_async_wait<0>();
+
+  // ---- finish: row sums across the quad, then write ----
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 1);
+    l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int qi = qt * QT + warp * 16 + gq + 8 * h;
+    if (qi >= Qn) continue;
+    const int row = seq * P.rows_per_seq + qi / P.group;
+    const int head = g * P.group + qi % P.group;
+    if (P.n_parts == 1) {
+      const float inv = l_run[h] > 0.f ? 1.f / l_run[h] : 0.f;
+      bf16* dst = P.out + ((size_t)row * P.hq + head) * DH;
+#pragma unroll
+      for (int i = 0; i < DH / 8; ++i)
+        *reinterpret_cast<uint32_t*>(dst + i * 8 + tq * 2) = pack_bf16(o[i][2 * h] * inv, o[i][2 * h + 1] * inv);
+    } else {
+      const size_t pidx = ((size_t)row * P.hq + head) * P.n_parts + part;
+      float* dst = P.part_o + pidx * DH;
+#pragma unroll
+      for (int i = 0; i < DH / 8; ++i)
+        *reinterpret_cast<float2*>(dst + i * 8 + tq * 2) = make_float2(o[i][2 * h], o[i][2 * h + 1]);
+      if (tq == 0) {
+        P.part_ml[pidx * 2 + 0] = m_run[h];      // log2 domain
+        P.part_ml[pidx * 2 + 1] = l_run[h];
+      }
+    }
+  }
+}
+
+// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One block of DH threads per (row, head).
+template <int DH>
+__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_parts,
+                                    bf16* __restrict__ out) {
+  const size_t rh = blockIdx.x;
+  const int d = threadIdx.x;
+  float M = -INFINITY;
+  for (int p = 0; p < n_parts; ++p) M = fmaxf(M, part_ml[(rh * n_parts + p) * 2]);
+  float L = 0.f, acc = 0.f;
+  for (int p = 0; p < n_parts; ++p) {
+    const float m = part_ml[(rh * n_parts + p) * 2];
+    if (m == -INFINITY) continue;
+    const float w = exp2f(m - M);
+    L += w * part_ml[(rh * n_parts + p) * 2 + 1];
+    acc += w * part_o[(rh * n_parts + p) * DH + d];
+  }
+  out[rh * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+}
+
+}  // namespace moa

@@ -135,6 +135,68 @@ __global__ void residual_norm_kernel(float* __restrict__ xres, const float* __re
   }
 }
 
+// Same operation spread over a thread-block cluster of 8 CTAs per row: each CTA owns K/8 columns, keeps
+// them in registers, and the row's sum of squares is exchanged through distributed shared memory (added
+// in rank order, so the result does not depend on scheduling). Needs K % 8 == 0 and K <= 16384.
+constexpr int RN_CLUSTER = 8;
+constexpr int RN_MAX_PER_THREAD = 8;
+
+template <typename T>
+__global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
+    residual_norm_cluster_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
+                                 int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
+                                 T* __restrict__ hidden_out) {
+  __shared__ float red[33];
+  __shared__ float cta_ss;
+  const int r = blockIdx.y;
+  const int rank = blockIdx.x;                       // cluster spans blockIdx.x = 0..7
+  const int cpc = K / RN_CLUSTER;                    // columns per CTA
+  const int c0 = rank * cpc;
+  float v[RN_MAX_PER_THREAD];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RN_MAX_PER_THREAD; ++i) {
+    const int c = threadIdx.x + i * 256;
+    v[i] = 0.f;
+    if (c < cpc) {
+      const size_t idx = (size_t)r * K + c0 + c;
+      float a = xres[idx];
+      if (part) a += sum_splits(part + idx, plane, splits);
+      xres[idx] = a;
+      v[i] = a;
+      ss += a * a;
+    }
+  }
+  if (gain == nullptr && hidden_out == nullptr) return;     // uniform over the whole grid
+  ss = block_sum(ss, red);
+  if (threadIdx.x == 0) cta_ss = ss;
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float total = 0.f;
+  {
+    const uint32_t local = (uint32_t)__cvta_generic_to_shared(&cta_ss);
+#pragma unroll
+    for (int j = 0; j < RN_CLUSTER; ++j) {
+      uint32_t remote;
+      float x;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(j));
+      asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(x) : "r"(remote) : "memory");
+      total += x;
+    }
+  }
+  // no CTA may exit (and release its shared memory) before every peer has read its slot
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+  const float rinv = rsqrtf(total / (float)K + eps);
+#pragma unroll
+  for (int i = 0; i < RN_MAX_PER_THREAD; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (c < cpc) {
+      const size_t idx = (size_t)r * K + c0 + c;
+      if (hidden_out) hidden_out[idx] = from_f<T>(v[i]);
+      if (gain) xn[idx] = from_f<T>(v[i] * rinv * to_f<T>(gain[c0 + c]));
+    }
+  }
+}
+
 // h = silu(sum gate) * (sum up): a partial plane row holds [gate | up] (2F columns).
 template <typename T>
 __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
@@ -215,21 +277,28 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
     for (int sp = 0; sp < splits; ++sp) a += row0[(size_t)sp * plane + c];
     return a;
   };
-  if (qdst) {
-    for (int i = threadIdx.x; i < hq * half; i += blockDim.x) {
-      const int h = i / half, j = i - h * half;
+  // blockIdx.y walks the heads: query heads (when qdst is given), then key heads, then value heads
+  int h = blockIdx.y;
+  const int nqh = qdst ? hq : 0;
+  if (h < nqh) {
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
       const float x1 = row(q_off + h * dh + j), x2 = row(q_off + h * dh + half + j);
       qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
       qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
     }
+    return;
   }
-  for (int i = threadIdx.x; i < hkv * half; i += blockDim.x) {
-    const int h = i / half, j = i - h * half;
-    const float x1 = row(k_off + h * dh + j), x2 = row(k_off + h * dh + half + j);
-    kdst[dst * hkv * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
-    kdst[dst * hkv * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+  h -= nqh;
+  if (h < hkv) {
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+      const float x1 = row(k_off + h * dh + j), x2 = row(k_off + h * dh + half + j);
+      kdst[dst * hkv * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
+      kdst[dst * hkv * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+    }
+    return;
   }
-  for (int i = threadIdx.x; i < hkv * dh; i += blockDim.x) vdst[dst * hkv * dh + i] = from_f<T>(row(v_off + i));
+  h -= hkv;
+  for (int j = threadIdx.x; j < dh; j += blockDim.x) vdst[dst * hkv * dh + h * dh + j] = from_f<T>(row(v_off + h * dh + j));
 }
 
 // Cross-attention cache append: fp32 [n, hkv*dh] k and v rows -> T cache rows at (seq, ca_len[seq] + i).
@@ -346,14 +415,14 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
 template <typename T>
 __global__ void mean_layers_kernel(const float* __restrict__ Z, int S, int D, float* __restrict__ kvf,
                                    T* __restrict__ kv_out) {
-  const int t = blockIdx.x;
-  for (int c = threadIdx.x; c < D; c += blockDim.x) {
-    float s = 0.f;
-    for (int l = 0; l < S; ++l) s += Z[((size_t)t * S + l) * D + c];
-    s *= 1.f / (float)S;
-    kvf[(size_t)t * D + c] = s;
-    if (kv_out) kv_out[(size_t)t * D + c] = from_f<T>(s);
-  }
+  const int t = blockIdx.x;                                   // grid (tokens, ceil(D / blockDim.x))
+  const int c = blockIdx.y * blockDim.x + threadIdx.x;
+  if (c >= D) return;
+  float s = 0.f;
+  for (int l = 0; l < S; ++l) s += Z[((size_t)t * S + l) * D + c];
+  s *= 1.f / (float)S;
+  kvf[(size_t)t * D + c] = s;
+  if (kv_out) kv_out[(size_t)t * D + c] = from_f<T>(s);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -62,8 +62,6 @@ __host__ __device__ constexpr int ws_smem_bytes(int npad) { return ws_stages(npa
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -355,11 +353,26 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 }
 
 // ---------------------------------------------------------------------------------------------
-// LM-head merge: one block per activation row combines the per-slice partials into
-// logsumexp and the global top-B, ordered by (log-probability descending, id ascending).
+// LM-head merge: one block per activation row combines the per-slice partials into logsumexp and
+// the global top-B, ordered by (log-probability descending, id ascending).
+//   1. logsumexp from the slices' (max, sum exp).
+//   2. threshold = the B-th best of the slice heads (each slice list is sorted, so its head is its
+//      best): B rounds of "best element ranking strictly after the previous pick", per warp and then
+//      over the 32 warp lists.
+//   3. survivors = candidates ranking at or before the threshold; only slices whose head does can
+//      contribute, so there are at most B*B of them. They are ranked by counting.
 // ---------------------------------------------------------------------------------------------
 constexpr int MERGE_THREADS = 1024;
 constexpr int MERGE_MAXB = 16;
+
+__device__ __forceinline__ void warp_best(float& bv, int& bi) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ranks_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+  }
+}
 
 __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __restrict__ p_max,
                                                                  const float* __restrict__ p_sum,
@@ -369,9 +382,17 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   __shared__ float red[33];
   __shared__ float w_val[32][MERGE_MAXB];
   __shared__ int w_id[32][MERGE_MAXB];
+  __shared__ float t_val;
+  __shared__ int t_id;
+  __shared__ float s_val[MERGE_MAXB * MERGE_MAXB];
+  __shared__ int s_id[MERGE_MAXB * MERGE_MAXB];
+  __shared__ int n_surv;
   const int r = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  // logsumexp over all slices
+  const int NONE = 0x7fffffff;
+  if (tid == 0) n_surv = 0;
+  if (tid < B) { ids[(size_t)r * B + tid] = -1; logp[(size_t)r * B + tid] = -INFINITY; }
+  // 1. logsumexp over all slices
   float m = -INFINITY;
   for (int s = tid; s < n_sub; s += MERGE_THREADS) m = fmaxf(m, p_max[(size_t)s * R + r]);
   m = block_max(m, red);
@@ -382,70 +403,71 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   }
   se = block_sum(se, red);
   const float lse = m + logf(se);
-  // thread-local top-B over this thread's slices (each slice list is already sorted)
-  float tv[MERGE_MAXB];
-  int ti[MERGE_MAXB];
-#pragma unroll
-  for (int i = 0; i < MERGE_MAXB; ++i) { tv[i] = -INFINITY; ti[i] = 0x7fffffff; }
+  // 2a. per warp: the B best slice heads among this warp's slices
+  float pv = INFINITY;
+  int pi = -1;
+  for (int round = 0; round < B; ++round) {
+    float bv = -INFINITY;
+    int bi = NONE;
+    for (int s = tid; s < n_sub; s += MERGE_THREADS) {
+      const float v = c_val[((size_t)s * R + r) * B];
+      const int id = c_id[((size_t)s * R + r) * B];
+      if (ranks_before(pv, pi, v, id) && ranks_before(v, id, bv, bi)) { bv = v; bi = id; }
+    }
+    warp_best(bv, bi);
+    pv = bv;
+    pi = bi;
+    if (lane == 0) { w_val[wid][round] = bv; w_id[wid][round] = bi; }
+    if (bi == NONE) {                       // this warp has run out of heads
+      for (int k = round + 1; k < B; ++k)
+        if (lane == 0) { w_val[wid][k] = -INFINITY; w_id[wid][k] = NONE; }
+      break;
+    }
+  }
+  __syncthreads();
+  // 2b. warp 0: the B-th best over the 32 sorted warp lists
+  if (wid == 0) {
+    float qv = INFINITY;
+    int qi = -1;
+    for (int round = 0; round < B; ++round) {
+      float bv = -INFINITY;
+      int bi = NONE;
+      for (int k = 0; k < B; ++k) {
+        const float v = w_val[lane][k];
+        const int id = w_id[lane][k];
+        if (ranks_before(qv, qi, v, id)) { bv = v; bi = id; break; }   // sorted: first one after the last pick
+      }
+      warp_best(bv, bi);
+      qv = bv;
+      qi = bi;
+    }
+    if (lane == 0) { t_val = qv; t_id = qi; }
+  }
+  __syncthreads();
+  const float tv = t_val;
+  const int ti = t_id;
+  // 3. survivors
   for (int s = tid; s < n_sub; s += MERGE_THREADS) {
     const float* cv = c_val + ((size_t)s * R + r) * B;
     const int* ci = c_id + ((size_t)s * R + r) * B;
     for (int c = 0; c < B; ++c) {
       const float v = cv[c];
       const int id = ci[c];
-      if (!ranks_before(v, id, tv[B - 1], ti[B - 1])) break;   // sorted list: the rest ranks lower still
-      // insert into the sorted local list
-      float nv = v;
-      int ni = id;
-#pragma unroll
-      for (int i = 0; i < MERGE_MAXB; ++i) {
-        if (i < B && ranks_before(nv, ni, tv[i], ti[i])) {
-          const float sv = tv[i]; const int si = ti[i];
-          tv[i] = nv; ti[i] = ni;
-          nv = sv; ni = si;
-        }
-      }
+      if (ranks_before(tv, ti, v, id)) break;          // strictly after the threshold: so is the rest
+      const int at = atomicAdd(&n_surv, 1);
+      if (at < MERGE_MAXB * MERGE_MAXB) { s_val[at] = v; s_id[at] = id; }
     }
-  }
-  // warp level: B rounds of arg-best over the 32 thread heads
-  int head = 0;
-  for (int round = 0; round < B; ++round) {
-    float hv = -INFINITY;
-    int hi = 0x7fffffff;
-#pragma unroll
-    for (int i = 0; i < MERGE_MAXB; ++i)
-      if (i == head) { hv = tv[i]; hi = ti[i]; }
-    float bv = hv;
-    int bi = hi;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ranks_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if (hi == bi && hv == bv && bi != 0x7fffffff) ++head;
-    if (lane == 0) { w_val[wid][round] = bv; w_id[wid][round] = bi; }
   }
   __syncthreads();
-  // block level: warp 0 merges the 32 sorted warp lists the same way
-  if (wid == 0) {
-    int h2 = 0;
-    for (int round = 0; round < B; ++round) {
-      const float hv = h2 < B ? w_val[lane][h2] : -INFINITY;
-      const int hi = h2 < B ? w_id[lane][h2] : 0x7fffffff;
-      float bv = hv;
-      int bi = hi;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ranks_before(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-      }
-      if (hi == bi && hv == bv && bi != 0x7fffffff) ++h2;
-      if (lane == 0) {
-        ids[(size_t)r * B + round] = bi == 0x7fffffff ? -1 : bi;
-        logp[(size_t)r * B + round] = bv - lse;
-      }
+  const int ns = n_surv < MERGE_MAXB * MERGE_MAXB ? n_surv : MERGE_MAXB * MERGE_MAXB;
+  if (tid < ns) {
+    const float v = s_val[tid];
+    const int id = s_id[tid];
+    int rank = 0;
+    for (int j = 0; j < ns; ++j) rank += ranks_before(s_val[j], s_id[j], v, id) ? 1 : 0;
+    if (rank < B && id != NONE) {
+      ids[(size_t)r * B + rank] = id;
+      logp[(size_t)r * B + rank] = v - lse;
     }
   }
 }
