@@ -126,6 +126,25 @@ moa_status moa_lsa_forward(moa_ctx *ctx, moa_state *st, const void *h_stack, con
 moa_status moa_sa_append(moa_ctx *ctx, moa_state *st, const int32_t *tok, const int32_t *n_host, int32_t batch,
                          void *ws, size_t ws_bytes, void *stream);
 
+/* The same operation as moa_sa_append for callers that cannot provide a workspace because they cannot
+ * allocate device memory at that point: code running between other components that have already handed
+ * all device memory to their own pools, or a serving loop in which a cudaMalloc (a device-wide
+ * synchronisation) is not allowed. The paper has no counterpart; this is a convenience of the library.
+ * Its scratch is a fixed array inside the library (4.5 MiB of device memory, held by every GPU on which
+ * the library is loaded, until the process exits), so the call allocates and frees nothing. Inputs and
+ * outputs are still the caller's: tok, the caches in st.
+ *   Limits: sum(n_host) <= MOA_SA_STATIC_MAX_TOKENS, sum(n_host) * d_model * sizeof(T) <= 512 KiB and
+ *   sum(n_host) * 2 * sa_hkv * head_dim * 4 <= 4 MiB; beyond them MOA_ERR_WORKSPACE is returned, nothing
+ *   is launched, and moa_last_cuda_error() holds the limits in words.
+ *   The first call on a device looks up the array's device address (a CUDA runtime query made with that
+ *   device current); make that first call outside any stream capture.
+ *   All calls on one device share the array. It keeps the previous call's contents; nothing in it has
+ *   to start at zero, because every element a call reads was written earlier in the same call. Two calls
+ *   whose kernels can overlap on the GPU (different streams) race on it: serialise them. */
+#define MOA_SA_STATIC_MAX_TOKENS 32
+moa_status moa_sa_append_static(moa_ctx *ctx, moa_state *st, const int32_t *tok, const int32_t *n_host, int32_t batch,
+                                void *stream);
+
 /* Starts a draft tree per sequence (Section 2.2). root_tok: device int32 [batch], the last verified
  * token; it sits at position sa_len[b]. Sets st->step = 0. */
 moa_status moa_tree_begin(moa_ctx *ctx, moa_state *st, const int32_t *root_tok, int32_t batch, void *stream);

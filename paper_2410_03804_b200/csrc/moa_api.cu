@@ -4,6 +4,7 @@
 
 #include <stdio.h>
 #include <string.h>
+#include <mutex>
 #include <new>
 
 #include "moa_attn.cuh"
@@ -919,6 +920,74 @@ moa_status moa_tree_attn_mask(const int32_t* parent, int32_t batch, int32_t n, v
       parent, batch, n, packed ? nullptr : (unsigned char*)mask_out, packed ? (unsigned long long*)mask_out : nullptr);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// moa_sa_append_static: moa_sa_append with its scratch in a fixed device array of this library.
+// ---------------------------------------------------------------------------------------------
+enum : size_t { SA_STATIC_XN_BYTES = 512u * 1024u, SA_STATIC_PART_BYTES = 4u * 1024u * 1024u };
+static __device__ __align__(256) unsigned char g_sa_static_scratch[SA_STATIC_XN_BYTES + SA_STATIC_PART_BYTES];
+enum { SA_STATIC_MAX_DEVICES = 64 };
+static void* g_sa_static_ptr[SA_STATIC_MAX_DEVICES];    // device address of the array on each device, 0 = not looked up
+static std::mutex g_sa_static_mutex;
+
+// Device address of the scratch array on the current device. The array's name is only a host-side handle
+// of the symbol, so the address is asked for once per device, with that device current.
+static moa_status sa_static_scratch(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess && (dev < 0 || dev >= SA_STATIC_MAX_DEVICES)) e = cudaErrorInvalidDevice;
+  if (e == cudaSuccess) {
+    std::lock_guard<std::mutex> lock(g_sa_static_mutex);
+    if (!g_sa_static_ptr[dev]) {
+      void* ptr = nullptr;
+      e = cudaGetSymbolAddress((void**)&ptr, g_sa_static_scratch);
+      if (e == cudaSuccess && ptr) g_sa_static_ptr[dev] = ptr;
+    }
+    *out = g_sa_static_ptr[dev];
+  }
+  if (e != cudaSuccess || !*out) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_sa_append_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    return MOA_ERR_CUDA;
+  }
+  return MOA_OK;
+}
+
+moa_status moa_sa_append_static(moa_ctx* ctx, moa_state* st, const int32_t* tok, const int32_t* n_host, int32_t batch,
+                                void* stream) {
+  MOA_TRY(check_state(ctx, st, batch));
+  if (!n_host) return MOA_ERR_NULL;
+  SeqSplit split;
+  MOA_TRY(make_split(n_host, batch, &split));
+  const int total = split.off[batch];
+  if (total > 0 && !tok) return MOA_ERR_NULL;
+  for (int b = 0; b < batch; ++b)
+    if ((long long)st->sa_len_host[b] + n_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
+  const moa_config& c = ctx->c;
+  const size_t kv_row_bytes = (size_t)2 * c.sa_hkv * c.head_dim * sizeof(float);
+  if (total > MOA_SA_STATIC_MAX_TOKENS || (size_t)total * c.d_model * ctx->elt > SA_STATIC_XN_BYTES ||
+      (size_t)total * kv_row_bytes > SA_STATIC_PART_BYTES) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err),
+             "moa_sa_append_static: %d tokens of width %d exceed the fixed scratch (at most %d tokens, %zu bytes of "
+             "normalised rows, %zu bytes of projected rows)",
+             total, c.d_model, (int)MOA_SA_STATIC_MAX_TOKENS, (size_t)SA_STATIC_XN_BYTES, (size_t)SA_STATIC_PART_BYTES);
+    return MOA_ERR_WORKSPACE;
+  }
+  void* scratch = nullptr;
+  MOA_TRY(sa_static_scratch(&scratch));
+  // the two regions moa_sa_append carves out of a caller workspace, laid over the fixed array instead
+  Workspace p;
+  memset(&p, 0, sizeof(p));
+  p.xn = 0;
+  p.part = SA_STATIC_XN_BYTES;
+  p.rows_cap = MOA_SA_STATIC_MAX_TOKENS;                         // one pass
+  p.part_rows = (int)(SA_STATIC_PART_BYTES / kv_row_bytes);      // bounds the K-split planes
+  p.total = SA_STATIC_XN_BYTES + SA_STATIC_PART_BYTES;
+  moa_status r = c.dtype == MOA_F32 ? sa_append_t<float>(ctx, st, tok, split, (char*)scratch, p, (cudaStream_t)stream)
+                                    : sa_append_t<bf16>(ctx, st, tok, split, (char*)scratch, p, (cudaStream_t)stream);
+  if (r == MOA_OK)
+    for (int b = 0; b < batch; ++b) st->sa_len_host[b] += n_host[b];
+  return r;
 }
 
 moa_status moa_state_status(moa_ctx* ctx, moa_state* st, void* stream) {

@@ -20,7 +20,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
 MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
-           "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_tree_begin", "moa_draft_step",
+           "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end",
            "moa_launch_count"]
 
@@ -87,6 +87,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_state_set_len.argtypes = [vp, C.POINTER(MoaState), i32, vp, i32, vp]
     lib.moa_lsa_forward.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, vp, sz, vp]
     lib.moa_sa_append.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, sz, vp]
+    lib.moa_sa_append_static.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp]
     lib.moa_tree_begin.argtypes = [vp, C.POINTER(MoaState), vp, i32, vp]
     lib.moa_draft_step.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, sz, vp]
     lib.moa_tree_expand.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -105,7 +106,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
 
 def _check(status: int, what: str):
     if status != MOA_OK:
-        detail = load_library().moa_last_cuda_error().decode() if status == 9 else ""
+        detail = load_library().moa_last_cuda_error().decode() if status in (5, 9) else ""
         raise MoaError(status, what, detail)
 
 
@@ -224,6 +225,15 @@ class MoA:
         assert tok.numel() == sum(n)
         _check(self.lib.moa_sa_append(self.h, C.byref(self.st), _ptr(tok), _host_i32(n), len(n), _ptr(self.ws),
                                       self.ws_bytes, _stream(stream)), "moa_sa_append")
+
+    def moa_sa_append_static(self, tok: torch.Tensor, n, stream=None):
+        """moa_sa_append without a workspace: the library's fixed scratch array is used, nothing is allocated.
+        For callers that cannot allocate device memory; at most 32 tokens per call (see include/moa.h)."""
+        assert tok.is_cuda and tok.dtype == torch.int32 and tok.is_contiguous()
+        n = [int(v) for v in n]
+        assert tok.numel() == sum(n)
+        _check(self.lib.moa_sa_append_static(self.h, C.byref(self.st), _ptr(tok), _host_i32(n), len(n),
+                                             _stream(stream)), "moa_sa_append_static")
 
     def moa_tree_begin(self, root_tok: torch.Tensor, stream=None):
         assert root_tok.is_cuda and root_tok.dtype == torch.int32 and root_tok.is_contiguous()
