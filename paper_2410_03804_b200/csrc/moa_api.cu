@@ -51,7 +51,7 @@ struct moa_ctx {
 // workspace carving (same arithmetic in moa_state_bytes and in the calls)
 // ---------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, total;
+  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, q32, total;
   int rows_cap, draft_rows, chunk_tok, part_rows, wide;
   long long att_units;   // (row, head, part) triples the split-attention partial buffers hold
 };
@@ -92,6 +92,7 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   p.att_units = (long long)c.tree_topk * gmax * 2 * 160 + 2ll * p.draft_rows * hqmax;
   p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
   p.att_ml = take(elt == 2 ? (size_t)p.att_units * 2 * sizeof(float) : 256);           // their (max, sum)
+  p.q32 = take(elt == 2 ? (size_t)p.draft_rows * hqmax * c.head_dim * sizeof(float) : 256);   // draft-step queries, fp32
   p.total = o;
   return p;
 }
@@ -262,13 +263,13 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
   return MOA_OK;
 }
 
-template <int DH>
+template <int DH, bool QSPLIT>
 static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nseq, int nwarps) {
   static bool attr_set = false;
-  const int smem = nwarps * 16 * DH * 2 + 4 * AT_KB * DH * 2;
+  const int smem = (QSPLIT ? 2 : 1) * nwarps * 16 * DH * 2 + 4 * AT_KB * DH * 2;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         8 * 16 * DH * 2 + 4 * AT_KB * DH * 2);
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<DH, QSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (QSPLIT ? 2 : 1) * 8 * 16 * DH * 2 + 4 * AT_KB * DH * 2);
     if (e != cudaSuccess) {
       snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
       return MOA_ERR_CUDA;
@@ -276,7 +277,7 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
     attr_set = true;
   }
   dim3 grid(P.n_parts, P.hkv * P.q_tiles, nseq);
-  attn_split_kernel<DH><<<grid, nwarps * 32, smem, s>>>(P);
+  attn_split_kernel<DH, QSPLIT><<<grid, nwarps * 32, smem, s>>>(P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
     attn_combine_kernel<DH><<<nseq * P.rows_per_seq * P.hq, DH, 0, s>>>(P.part_o, P.part_ml, P.n_parts, P.out);
@@ -288,8 +289,8 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
 // softmax(q K^T / sqrt(dh)) V for R = nseq * rows_per_seq query rows. Segment A: a cache (or the LSA rows
 // themselves) with max_len positions at most on the host's count; segment B: tree slots masked per row.
 template <typename T>
-static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int dh, const T* q, int q_ld,
-                            int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
+static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int dh, const T* q,
+                            const float* q32, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
                             int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
                             int slots_ld, int nB, int n_slots, int rows_per_seq, T* out) {
   if (R <= 0) return MOA_OK;
@@ -297,7 +298,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     AttnParams P;
     memset(&P, 0, sizeof(P));
     const int nseq = R / rows_per_seq;
-    P.q = (const bf16*)q; P.q_ld = q_ld;
+    P.q = (const bf16*)q; P.q32 = q32; P.q_ld = q_ld;
     P.hq = hq; P.hkv = hkv; P.group = hq / hkv;
     P.rows_per_seq = rows_per_seq;
     P.kA = (const bf16*)kA; P.vA = (const bf16*)vA; P.capA = capA; P.posA_ld = posA_ld;
@@ -319,7 +320,8 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.part_ml = (float*)(ws + p.att_ml);
     P.out = (bf16*)out;
     P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
-    return dh == 128 ? launch_attn_split<128>(s, P, nseq, nwarps) : launch_attn_split<64>(s, P, nseq, nwarps);
+    if (q32) return dh == 128 ? launch_attn_split<128, true>(s, P, nseq, nwarps) : launch_attn_split<64, true>(s, P, nseq, nwarps);
+    return dh == 128 ? launch_attn_split<128, false>(s, P, nseq, nwarps) : launch_attn_split<64, false>(s, P, nseq, nwarps);
   }
   dim3 grid(R, hq);
   if (dh == 128)
@@ -406,7 +408,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
       MOA_CHECK_LAUNCH();
     }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
-    MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld,
+    MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, nullptr, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld,
                          nullptr, S, S, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0, S, obuf));
     // out-projection + residual, MLP + residual
     const void* W1[1] = {w.lsa_wo};
@@ -460,7 +462,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
     rr.split = split;
     rr.row0 = t0;
     rope_store_kernel<T><<<dim3(R, 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
-                                           c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
+                                           c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (float*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
     MOA_CHECK_LAUNCH();
   }
   add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split);
@@ -540,6 +542,8 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   T* xn = (T*)(ws + p.xn);
   T* narrow = (T*)(ws + p.narrow);
   T* obuf = (T*)(ws + p.obuf);
+  // bf16 path: the queries of both attentions stay in fp32 and are split into two bf16 terms by the kernel
+  float* q32 = sizeof(T) == 2 ? (float*)(ws + p.q32) : nullptr;
   LinOut lo;
 
   // ---- self-attention block ----
@@ -558,14 +562,14 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   rr.B = B;
   rr.slots = L.NS;
   rope_store_kernel<T><<<dim3(R, c.sa_hq + 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
-                                         dh, c.sa_rope_theta, st->sa_len, rr, narrow, tk, tv);
+                                         dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, tk, tv);
   MOA_CHECK_LAUNCH();
   int max_sa = 0, max_ca = 0;
   for (int b = 0; b < batch; ++b) {
     max_sa = imax(max_sa, st->sa_len_host[b]);
     max_ca = imax(max_ca, st->ca_len_host[b]);
   }
-  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
                        c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
                        step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
   {
@@ -584,10 +588,11 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     const int N1[1] = {cq};
     MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
     const size_t tot = (size_t)R * cq;
-    sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
+    if (q32) sum_cast_kernel<float><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, q32);
+    else sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
     MOA_CHECK_LAUNCH();
   }
-  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,
                        c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0,
                        rows_per_seq, obuf));
   {

@@ -22,6 +22,7 @@ constexpr int AT_KB = 64;        // keys per block
 
 struct AttnParams {
   const bf16* q; int q_ld;               // query row r, head h at q + r*q_ld + h*DH
+  const float* q32;                      // QSPLIT kernels: the same layout in fp32 (q is unused then)
   int hq, hkv, group;                    // group = hq / hkv
   int rows_per_seq;                      // query rows of one sequence (tree rows, or LSA layers)
   const bf16* kA; const bf16* vA; int capA; int posA_ld;   // segment A: (seq*capA + j)*posA_ld + g*DH
@@ -68,7 +69,11 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
   return (uint32_t)(row * (DH * 2) + ((chunk ^ (row & 7)) << 4));
 }
 
-template <int DH>
+// QSPLIT: the queries arrive in fp32 and are split into two bf16 terms (q = hi + lo, lo = the part of q
+// that hi's 8-bit mantissa dropped); scores are Q_hi.K^T + Q_lo.K^T, so they carry the queries at about 16 bits
+// of mantissa while the cached keys stay in their 16-bit storage type. This keeps a peaked softmax (keys
+// with outlier channels) from amplifying the rounding of q.
+template <int DH, bool QSPLIT>
 __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int KS = DH / 16;                // k-steps of the Q.K^T product
@@ -83,7 +88,8 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   const int QT = nwarps * 16;                // queries per tile
   const int Qn = P.rows_per_seq * P.group;   // queries per (seq, kv head)
   const uint32_t sQ = smem_u32(at_smem);
-  const uint32_t sKV = sQ + QT * DH * 2;     // [2 stages][K tile | V tile]
+  const uint32_t sQlo = sQ + QT * DH * 2;    // QSPLIT only
+  const uint32_t sKV = sQ + (QSPLIT ? 2 : 1) * QT * DH * 2;     // [2 stages][K tile | V tile]
 
   const bool tree_part = part >= P.n_split;
   // key range of this part
@@ -115,7 +121,26 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     const bool valid = qi < Qn;
     const int row = seq * P.rows_per_seq + (valid ? qi / P.group : 0);
     const int head = g * P.group + (valid ? qi % P.group : 0);
-    cp_async16(sQ + tile_off<DH>(ql, c), P.q + (size_t)row * P.q_ld + head * DH + c * 8, valid);
+    if (QSPLIT) {
+      uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+      if (valid) {
+        const float4* src = reinterpret_cast<const float4*>(P.q32 + (size_t)row * P.q_ld + head * DH + c * 8);
+        const float4 a = src[0], b = src[1];
+        const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bf16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
+          hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+          lo[e] = pack_bf16(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
+        }
+      }
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQ + tile_off<DH>(ql, c)), "r"(hi[0]), "r"(hi[1]),
+                   "r"(hi[2]), "r"(hi[3]) : "memory");
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQlo + tile_off<DH>(ql, c)), "r"(lo[0]), "r"(lo[1]),
+                   "r"(lo[2]), "r"(lo[3]) : "memory");
+    } else {
+      cp_async16(sQ + tile_off<DH>(ql, c), P.q + (size_t)row * P.q_ld + head * DH + c * 8, valid);
+    }
   }
   cp_async_commit();
 
@@ -172,14 +197,25 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     // S = Q K^T over the block's 64 keys: 8 n-tiles of 8 keys
     float s[AT_KB / 8][4];
 #pragma unroll
-    for (int nt = 0; nt < AT_KB / 8; ++nt) {
-      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    for (int nt = 0; nt < AT_KB / 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
-      for (int ks2 = 0; ks2 < KS / 2; ++ks2) {
+    for (int ks2 = 0; ks2 < KS / 2; ++ks2) {
+      uint32_t ql0[4], ql1[4];         // QSPLIT: the low query terms of these two k-steps
+      if (QSPLIT) {
+        const int row = warp * 16 + (lane & 15);
+        ldsm_x4(sQlo + tile_off<DH>(row, (2 * ks2) * 2 + (lane >> 4)), ql0[0], ql0[1], ql0[2], ql0[3]);
+        ldsm_x4(sQlo + tile_off<DH>(row, (2 * ks2 + 1) * 2 + (lane >> 4)), ql1[0], ql1[1], ql1[2], ql1[3]);
+      }
+#pragma unroll
+      for (int nt = 0; nt < AT_KB / 8; ++nt) {
         uint32_t b0, b1, b2, b3;       // two k-steps: chunks 4*ks2 .. 4*ks2+3 of key row nt*8 + lane%8
         ldsm_x4(sK + tile_off<DH>(nt * 8 + (lane & 7), ks2 * 4 + (lane >> 3)), b0, b1, b2, b3);
         mma_bf16_16816(s[nt], qf[2 * ks2], b0, b1);
         mma_bf16_16816(s[nt], qf[2 * ks2 + 1], b2, b3);
+        if (QSPLIT) {
+          mma_bf16_16816(s[nt], ql0, b0, b1);
+          mma_bf16_16816(s[nt], ql1, b2, b3);
+        }
       }
     }
     // scale, mask, block row max

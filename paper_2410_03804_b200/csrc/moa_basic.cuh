@@ -221,7 +221,7 @@ __global__ void sum_cast_kernel(const float* __restrict__ part, int splits, size
 // ---------------------------------------------------------------------------------------------
 // Rotary embedding + stores. One block per row. The input may be `splits` partial planes (plane
 // elements apart) that are summed on the fly.
-//   q (optional): fp32 [R, hq*dh] at qkv + q_off (leading dim ld) -> rotated, T [R, hq*dh]
+//   q (optional): fp32 [R, hq*dh] at qkv + q_off (leading dim ld) -> rotated, T [R, hq*dh] (or fp32 into qdst32)
 //   k, v: fp32 [R, hkv*dh] -> k rotated; written as T to  kdst/vdst + dst_index(row) * hkv*dh
 // Row r sits at position pos_base[seq(r)] + pos_add(r). Angles are formed in double:
 // angle = pos * theta^(-2i/dh), element i paired with i + dh/2. theta == 0: no rotation.
@@ -240,7 +240,8 @@ template <typename T>
 __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, size_t plane, int ld, int q_off, int k_off,
                                   int v_off,
                                   int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
-                                  RopeRows rr, T* __restrict__ qdst, T* __restrict__ kdst, T* __restrict__ vdst) {
+                                  RopeRows rr, T* __restrict__ qdst, float* __restrict__ qdst32, T* __restrict__ kdst,
+                                  T* __restrict__ vdst) {
   __shared__ float cs[64], sn[64];
   const int r = blockIdx.x;
   int seq, pos_add;
@@ -283,8 +284,13 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
   if (h < nqh) {
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
       const float x1 = row(q_off + h * dh + j), x2 = row(q_off + h * dh + half + j);
-      qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
-      qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+      if (qdst32) {                    // rotated queries kept in fp32 (the attention kernel splits them)
+        qdst32[(size_t)r * hq * dh + h * dh + j] = x1 * cs[j] - x2 * sn[j];
+        qdst32[(size_t)r * hq * dh + h * dh + half + j] = x2 * cs[j] + x1 * sn[j];
+      } else {
+        qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
+        qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+      }
     }
     return;
   }

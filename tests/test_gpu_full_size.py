@@ -1,0 +1,84 @@
+"""Parity at the full sizes of configs 2-5, in the launch configuration the benchmark times.
+
+The oracle cannot walk every row of the large configs in reasonable time, so it computes sampled outputs one
+by one (whole sequences of the batch, single LSA tokens) and every other output is checked through
+properties that hold at any size (tree well-formed, scores monotone, finite values). Same tolerances as
+the small-shape parity tests."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_03804_b200 import synth
+from tests import helpers as H
+from tests.test_gpu_parity import run_cycle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def llama8b():
+    """Config 2's drafter (weights, CUDA context, oracles), shared by the c2 and c4 cases."""
+    p = synth.PRESETS["c2"]
+    w = synth.make_weights(p)
+    g = H.make_gpu(p, w, max_ctx=32768 + 64, lsa_chunk_tokens=p.lsa_tokens)
+    oracles = H.make_oracles(p, w)
+    yield p, w, g, oracles
+    g.close()
+
+
+def _given_caches_cycle(p, g, oracles, seqs=None):
+    """LSA on the cycle's new tokens (checked against the oracle on sampled sequences), then a teacher-forced
+    tree over the synthetic caches."""
+    tol = H.tol_of(p)
+    exact, _ = oracles
+    nb, A = p.batch, p.lsa_tokens
+    seqs = list(range(nb)) if seqs is None else seqs
+    caK, caV = synth.make_cache(p, "ca")
+    saK, saV = synth.make_cache(p, "sa")
+    stats = run_cycle(p, g, oracles, None, None, synth.make_root(p), ca_cache=(caK, caV), sa_cache=(saK, saV), seqs=seqs)
+    # the cycle's LSA step on top of the filled cache: appended CA rows against the oracle
+    h = synth.make_h_stack(p, nb * A)
+    kv = g.moa_lsa_forward(h.cuda(), [A] * nb)
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0
+    assert g.ca_len[:nb].tolist() == [p.ctx + A] * nb
+    assert bool(torch.isfinite(kv.float()).all())
+    for b in seqs:
+        toks = [0, A - 1] if len(seqs) < nb else list(range(A))
+        for t in toks:
+            kv_o = exact.lsa_forward(H.np32(h[b * A + t][None]))
+            H.assert_rows_close(H.np32(kv[b * A + t].cpu())[None], kv_o, tol, f"LSA kv seq {b} tok {t}")
+            K_o, V_o = exact.ca_kv(kv_o)
+            H.assert_rows_close(H.np32(g.ca_k[b, p.ctx + t].cpu()).reshape(1, -1), K_o.reshape(1, -1), tol, "CA K append")
+            H.assert_rows_close(H.np32(g.ca_v[b, p.ctx + t].cpu()).reshape(1, -1), V_o.reshape(1, -1), tol, "CA V append")
+    return stats
+
+
+def test_c2_llama8b_full_cycle(llama8b):
+    """Config 2: d 4096, 32 stacked layers, 32/8 heads x 128, context 2048, vocabulary 128256, tree 10/6/60.
+    Every one of the 51 forward rows and all 5 LSA tokens are checked."""
+    p, w, g, oracles = llama8b
+    stats = _given_caches_cycle(p, g, oracles)
+    assert stats["rows"] == 1 + 5 * 10
+
+
+def test_c4_long_context_32k(llama8b):
+    """Config 4: config 2's drafter over 32768-entry caches (both attentions), every row checked."""
+    p2, w, g, oracles = llama8b
+    p = synth.scaled(p2, name="c4", ctx=32768)
+    stats = _given_caches_cycle(p, g, oracles)
+    assert stats["rows"] == 1 + 5 * 10
+
+
+def test_c5_llama70b_batch16_sampled_sequences():
+    """Config 5: d 8192, 80 layers, 64/8 heads, batch 16 x context 4096. The oracle walks sequences 0 and 15
+    (first and last of the batch) row by row and two LSA tokens of each; the other 14 sequences are checked
+    through the tree properties."""
+    p = synth.PRESETS["c5"]
+    w = synth.make_weights(p)
+    g = H.make_gpu(p, w, max_ctx=p.ctx + 64, lsa_chunk_tokens=p.batch * p.lsa_tokens)
+    oracles = H.make_oracles(p, w)
+    del w
+    stats = _given_caches_cycle(p, g, oracles, seqs=[0, 15])
+    assert stats["rows"] == 2 * (1 + 5 * 10)
+    g.close()

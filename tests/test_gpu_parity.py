@@ -17,49 +17,53 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def oracle_cycle(p, dr, h_stack, prompt, root, ca_cache, sa_cache, forced=None):
-    """The oracle's side of one drafting cycle. forced[b] = per-step (ids, logp) to expand with."""
+def oracle_cycle(p, dr, h_stack, prompt, root, ca_cache, sa_cache, forced=None, seqs=None):
+    """The oracle's side of one drafting cycle, for the sequences listed in seqs (default: all).
+    forced[b] = per-step (ids, logp) to expand with. Per-sequence results are dicts keyed by b."""
     nb = p.batch
-    out = {}
-    if ca_cache is None:
-        n = h_stack.shape[0] // nb
-        out["kv"] = dr.lsa_forward(H.np32(h_stack))
-        caK, caV = dr.ca_kv(out["kv"])
-        out["caK"], out["caV"] = caK.reshape(nb, n, *caK.shape[1:]), caV.reshape(nb, n, *caV.shape[1:])
-    else:
-        out["caK"], out["caV"] = H.np32(ca_cache[0]), H.np32(ca_cache[1])
-    if sa_cache is None:
-        n = prompt.shape[1]
-        out["saK"] = np.zeros((nb, n, p.sa_hkv, p.head_dim))
-        out["saV"] = np.zeros_like(out["saK"])
-        for b in range(nb):
+    seqs = list(range(nb)) if seqs is None else list(seqs)
+    out = {"kv": {}, "caK": {}, "caV": {}, "saK": {}, "saV": {}, "trees": {}}
+    for b in seqs:
+        if ca_cache is None:
+            n = h_stack.shape[0] // nb
+            out["kv"][b] = dr.lsa_forward(H.np32(h_stack[b * n:(b + 1) * n]))
+            out["caK"][b], out["caV"][b] = dr.ca_kv(out["kv"][b])
+        else:
+            out["caK"][b], out["caV"][b] = H.np32(ca_cache[0][b]), H.np32(ca_cache[1][b])
+        if sa_cache is None:
             out["saK"][b], out["saV"][b] = dr.sa_prefix(prompt[b].tolist())
-    else:
-        out["saK"], out["saV"] = H.np32(sa_cache[0]), H.np32(sa_cache[1])
-    out["trees"] = [O.draft_tree(dr, int(root[b]), out["saK"][b], out["saV"][b], out["caK"][b], out["caV"][b],
-                                 p.tree_topk, p.tree_depth, p.tree_keep, forced=None if forced is None else forced[b])
-                    for b in range(nb)]
+        else:
+            out["saK"][b], out["saV"][b] = H.np32(sa_cache[0][b]), H.np32(sa_cache[1][b])
+        out["trees"][b] = O.draft_tree(dr, int(root[b]), out["saK"][b], out["saV"][b], out["caK"][b], out["caV"][b],
+                                       p.tree_topk, p.tree_depth, p.tree_keep,
+                                       forced=None if forced is None else forced[b])
     return out
 
 
-def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None):
+def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None, seqs=None):
     """One drafting cycle on both sides. The tree follows the deciding oracle's top-B (teacher forcing);
-    values are compared with the unrounded oracle walking the same tree."""
+    values are compared with the unrounded oracle walking the same tree. With seqs given, the oracle runs
+    only on those sequences of the batch (sampled outputs); the others expand with the GPU's own lists."""
     exact, dec = oracles
     tol = H.tol_of(p)
     nb = p.batch
     B, D = p.tree_topk, p.tree_depth
-    od = oracle_cycle(p, dec, h_stack, prompt, root, ca_cache, sa_cache)
-    forced = [[([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in od["trees"][b][1]] for b in range(nb)]
-    ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced)
+    seqs = list(range(nb)) if seqs is None else list(seqs)
+    od = oracle_cycle(p, dec, h_stack, prompt, root, ca_cache, sa_cache, seqs=seqs)
+    forced = {b: [([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in od["trees"][b][1]] for b in seqs}
+    ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced, seqs=seqs)
     stats = dict(rows=0, exact=0, worst_hidden=0.0)
     if ca_cache is None:
         n_tok = [h_stack.shape[0] // nb] * nb
+        n = n_tok[0]
         kv = g.moa_lsa_forward(h_stack.cuda(), n_tok)
         torch.cuda.synchronize()
-        stats["lsa"] = H.assert_rows_close(H.np32(kv.cpu()), ox["kv"], tol, "LSA kv")
-        H.assert_rows_close(H.np32(g.ca_k[:nb, :n_tok[0]].cpu()), ox["caK"], tol, "CA K cache")
-        H.assert_rows_close(H.np32(g.ca_v[:nb, :n_tok[0]].cpu()), ox["caV"], tol, "CA V cache")
+        stats["lsa"] = 0.0
+        for b in seqs:
+            stats["lsa"] = max(stats["lsa"], H.assert_rows_close(H.np32(kv[b * n:(b + 1) * n].cpu()), ox["kv"][b], tol,
+                                                                 "LSA kv"))
+            H.assert_rows_close(H.np32(g.ca_k[b, :n].cpu()), ox["caK"][b], tol, "CA K cache")
+            H.assert_rows_close(H.np32(g.ca_v[b, :n].cpu()), ox["caV"][b], tol, "CA V cache")
         assert g.ca_len[:nb].tolist() == n_tok
     else:
         g.fill_cache("ca", ca_cache[0].cuda(), ca_cache[1].cuda())
@@ -67,8 +71,9 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
         n = prompt.shape[1]
         g.moa_sa_append(prompt.reshape(-1).cuda(), [n] * nb)
         torch.cuda.synchronize()
-        H.assert_rows_close(H.np32(g.sa_k[:nb, :n].cpu()), ox["saK"], tol, "SA K cache")
-        H.assert_rows_close(H.np32(g.sa_v[:nb, :n].cpu()), ox["saV"], tol, "SA V cache")
+        for b in seqs:
+            H.assert_rows_close(H.np32(g.sa_k[b, :n].cpu()), ox["saK"][b], tol, "SA K cache")
+            H.assert_rows_close(H.np32(g.sa_v[b, :n].cpu()), ox["saV"][b], tol, "SA V cache")
         assert g.sa_len[:nb].tolist() == [n] * nb
     else:
         g.fill_cache("sa", sa_cache[0].cuda(), sa_cache[1].cuda())
@@ -79,9 +84,8 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
         torch.cuda.synchronize()
         ids, lp, hid = ids.cpu().numpy(), lp.cpu().numpy(), H.np32(hid.cpu())
         rs = 1 if s == 0 else B
-        f_ids = np.zeros((nb * rs, B), np.int32)
-        f_lp = np.zeros((nb * rs, B), np.float32)
-        for b in range(nb):
+        f_ids, f_lp = ids.copy(), lp.copy()          # unsampled sequences follow the GPU's own choices
+        for b in seqs:
             for r in range(rs):
                 gr = b * rs + r
                 rx, rd = ox["trees"][b][1][s][r], od["trees"][b][1][s][r]
@@ -99,11 +103,17 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
     torch.cuda.synchronize()
     assert g.moa_state_status() == 0
     tok, parent, depth, score, n = [t.cpu().numpy() for t in outs]
-    for b in range(nb):
+    for b in seqs:
         otok, opar, odep, osc = O.tree_finalize(od["trees"][b][0])
         k = len(otok)
         assert n[b] == k and np.array_equal(tok[b, :k], otok) and np.array_equal(parent[b, :k], opar)
         assert np.array_equal(depth[b, :k], odep) and np.array_equal(score[b, :k].view(np.int32), osc.view(np.int32))
+    for b in range(nb):                              # properties that hold for every sequence, sampled or not
+        k = int(n[b])
+        assert 1 <= k <= p.tree_keep + 1 and parent[b, 0] == -1 and depth[b, 0] == 0
+        assert np.all(parent[b, 1:k] < np.arange(1, k)) and np.all(parent[b, 1:k] >= 0)
+        assert np.array_equal(depth[b, 1:k], depth[b, parent[b, 1:k]] + 1)
+        assert np.all(score[b, 1:k] <= score[b, parent[b, 1:k]])
     print(f"[parity {p.name} {p.dtype}] {stats}")
     return stats
 
