@@ -1,0 +1,259 @@
+// Phase machine, part 1: descriptors, small device helpers and the static GEMM schedule.
+//
+// The phase machine is one persistent cooperative kernel that runs a whole drafter forward (or a whole
+// LSA pass) as a list of phases separated by grid-wide barriers; see moa_phases.cuh for the kernel and
+// the reasons. This file holds what its parts share.
+//
+// Activation operands ("X buffers") may carry each value as TWO bf16 terms, hi + lo, where lo is what
+// hi's 8-bit mantissa dropped. The MMA then runs over N = 2 x padded rows and the epilogue adds the two
+// column halves, so activations enter every product with ~16 bits of mantissa while weights and caches
+// stay in their 16-bit storage type. With few rows this is free: the stream is HBM-bound and N only
+// grows from 16 to 32.
+#pragma once
+#include "moa_attn.cuh"
+#include "moa_basic.cuh"
+#include "moa_wstream.cuh"
+
+namespace moa {
+
+constexpr int PM_THREADS = 256;
+constexpr int PM_WORKERS = 192;          // warps 2..7
+constexpr int PM_WWARPS = 6;
+constexpr int PM_MAX_OPS = 28;
+constexpr int PM_MAX_GEMMS = 10;
+constexpr int PM_MAX_STAGES = 12;
+constexpr int PM_KB = 32;                // keys per attention block
+constexpr int PM_KVST = 4;               // key/value blocks in flight per attention unit
+constexpr int PM_MAXCH = 6;              // 8-element chunks a thread keeps of one row (rows up to 9216 wide)
+constexpr int PM_MERGE_OWN = 24;         // vocabulary slices one thread owns in the LM-head merge
+
+enum PmKind : int {
+  PH_GEMM = 0, PH_EMBED_NORM, PH_ROWS_NORM, PH_RESNORM, PH_ROPE, PH_ATTN, PH_COMBINE, PH_SILU, PH_SUMCAST,
+  PH_MEAN_NORM, PH_CACHE_APPEND, PH_MERGE
+};
+
+struct PmGemm {            // (its tensor maps are PmParams.tm[gemm][0..2] weights, [3] activations)
+  int n_seg, seg_n[3], seg_tile0[3], seg_col[3];
+  int tiles_total;         // weight tiles (gated: gate/up tile pairs)
+  int kb_total, splits, row_blocks;
+  int units, rot;          // tiles_total * splits * row_blocks; unit u runs on CTA (u + rot) % grid
+  int mode;                // 0 fp32 split planes, 1 LM-head partial top-B, 2 bf16 store, 3 residual add, 4 gated SwiGLU
+  int R;                   // valid activation rows
+  int xsplit;              // X buffer carries hi | lo halves (lo rows start at NB/2)
+  int rows_per_block;      // X rows per unit: NB, or 128 when gated
+  int ldo;                 // modes 0, 3: leading dimension of out
+  int ld16;                // modes 2, 4
+  int B;                   // mode 1
+  int n_sub;               // mode 1: partial lists per activation row
+  size_t plane;            // mode 0: elements between split planes
+  float* out;              // mode 0: planes; mode 3: fp32 residual stream
+  bf16* out16;             // modes 2, 4
+  float *p_max, *p_sum, *c_val;   // mode 1: [n_sub][R], [n_sub][R], [n_sub][R][B]
+  int* c_id;
+};
+
+struct PmOp {
+  int kind;
+  int gemm;                // PH_GEMM: which; glue: the GEMM whose split planes are consumed (-1: none)
+  int rows, cols;          // rows and width the op works on
+  const void* p[12];
+  int i[16];
+  float f[2];
+};
+
+struct PmParams {
+  CUtensorMap tm[PM_MAX_GEMMS][4];   // per GEMM: weight matrices [n_i, K] (box 64 x 128, swizzle 128B) and, last,
+                                     // its X buffer [rows, K] (box 64 x NB; gated: 64 x 128)
+  PmGemm g[PM_MAX_GEMMS];
+  PmOp op[PM_MAX_OPS];
+  SeqSplit split;          // PH_CACHE_APPEND
+  int n_ops, n_gemms;
+  int stages;              // ring depth
+  int alias_attn;          // attention scratch lies over the ring: no weight run-ahead across phases
+  uint32_t attn_off;       // byte offset of the attention scratch from the aligned shared-memory base
+  int* sync;               // device int[4]: [0] barrier counter, [1] abort word, [2] exit counter
+  int* flags;              // device int[grid * 32]: per-CTA barrier flag, one 128-byte line each (zero between launches)
+  int* status;             // device status word
+  unsigned long long* trace;   // [2 * PM_MAX_OPS + 1] ns timestamps of CTA 0: start, then per phase: work done, barrier passed
+};
+
+// What every role reads all the time, copied from the kernel parameters into shared memory at start-up
+// (the tensor maps stay in parameter space, where TMA wants them).
+struct PmSmem {
+  PmOp op[PM_MAX_OPS];
+  PmGemm g[PM_MAX_GEMMS];
+  SeqSplit split;
+  int n_ops;
+  float red[8];            // worker-wide reductions
+};
+constexpr int PM_FIXED_SMEM = 1024 + 512 + (int)((sizeof(PmSmem) + 127) / 128) * 128;   // alignment slack, barriers, PmSmem
+
+template <int NB>
+__host__ __device__ constexpr int pm_stage_bytes() { return WS_W_BYTES + NB * WS_BK * 2; }
+
+// ---------------------------------------------------------------------------------------------
+// small helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void wbar() { asm volatile("bar.sync 1, %0;" ::"n"(PM_WORKERS) : "memory"); }
+
+__device__ __forceinline__ float worker_sum(float v, float* red, int wt) {
+  v = warp_sum(v);
+  if ((wt & 31) == 0) red[wt >> 5] = v;
+  wbar();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < PM_WWARPS; ++i) t += red[i];
+  wbar();
+  return t;
+}
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+
+// 8 consecutive fp32 values: sum of `splits` planes (plane elements apart), read past L1. The loads of four
+// planes are issued before any of them is used, so a row costs one memory round trip per four planes.
+__device__ __forceinline__ void load8_planes(const float* p, int splits, size_t plane, float* v) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = 0.f;
+  int s = 0;
+  for (; s + 4 <= splits; s += 4) {
+    float4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { a[u] = ldcg4(p + (size_t)(s + u) * plane); b[u] = ldcg4(p + (size_t)(s + u) * plane + 4); }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      v[0] += a[u].x; v[1] += a[u].y; v[2] += a[u].z; v[3] += a[u].w;
+      v[4] += b[u].x; v[5] += b[u].y; v[6] += b[u].z; v[7] += b[u].w;
+    }
+  }
+  float4 a[3], b[3];
+#pragma unroll
+  for (int u = 0; u < 3; ++u)
+    if (s + u < splits) { a[u] = ldcg4(p + (size_t)(s + u) * plane); b[u] = ldcg4(p + (size_t)(s + u) * plane + 4); }
+#pragma unroll
+  for (int u = 0; u < 3; ++u)
+    if (s + u < splits) {
+      v[0] += a[u].x; v[1] += a[u].y; v[2] += a[u].z; v[3] += a[u].w;
+      v[4] += b[u].x; v[5] += b[u].y; v[6] += b[u].z; v[7] += b[u].w;
+    }
+}
+
+// One fp32 value as the sum of its split planes, loads issued four at a time.
+__device__ __forceinline__ float load1_planes(const float* p, int splits, size_t plane) {
+  float acc = 0.f;
+  int s = 0;
+  for (; s + 4 <= splits; s += 4) {
+    const float a = __ldcg(p + (size_t)s * plane), b = __ldcg(p + (size_t)(s + 1) * plane);
+    const float c = __ldcg(p + (size_t)(s + 2) * plane), d = __ldcg(p + (size_t)(s + 3) * plane);
+    acc += a; acc += b; acc += c; acc += d;
+  }
+  float t[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+  for (int u = 0; u < 3; ++u)
+    if (s + u < splits) t[u] = __ldcg(p + (size_t)(s + u) * plane);
+  return acc + t[0] + t[1] + t[2];
+}
+
+__device__ __forceinline__ void bf16x8_to_float(const uint4 u, float* v) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+// Stores 8 values into an X buffer row as bf16: hi at row r, and (lo_rows > 0) the remainder at row lo_rows + r.
+__device__ __forceinline__ void xbuf_store8(bf16* xb, size_t K, int r, int k, int lo_rows, const float* v) {
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const bf16 h0 = __float2bfloat16_rn(v[2 * e]), h1 = __float2bfloat16_rn(v[2 * e + 1]);
+    hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+    lo[e] = pack_bf16(v[2 * e] - __bfloat162float(h0), v[2 * e + 1] - __bfloat162float(h1));
+  }
+  *reinterpret_cast<uint4*>(xb + (size_t)r * K + k) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+  if (lo_rows > 0) *reinterpret_cast<uint4*>(xb + (size_t)(lo_rows + r) * K + k) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// static schedule of the GEMM phases as seen by one CTA (same arithmetic in the three roles)
+// ---------------------------------------------------------------------------------------------
+struct PmUnit {
+  int seg, n0, kb0, kb1, split, tile, rb;
+};
+
+__device__ __forceinline__ void pm_decode(const PmGemm& G, int u, PmUnit& d) {
+  // unit -> (row-block group, tile, row block in group) with 4 row blocks per group, or (tile, split)
+  int tile, rb = 0, split = 0;
+  if (G.row_blocks > 1) {
+    const int per_group = G.tiles_total * 4;
+    const int grp = u / per_group;
+    const int rem = u - grp * per_group;
+    const int left = G.row_blocks - grp * 4;
+    const int ge = left < 4 ? left : 4;
+    tile = rem / ge;
+    rb = grp * 4 + (rem - tile * ge);
+  } else {
+    tile = u / G.splits;
+    split = u - tile * G.splits;
+  }
+  d.tile = tile; d.rb = rb; d.split = split;
+  int seg = 0;
+  if (G.n_seg > 1 && tile >= G.seg_tile0[1]) seg = 1;
+  if (G.n_seg > 2 && tile >= G.seg_tile0[2]) seg = 2;
+  if (G.mode == 4) seg = 0;
+  d.seg = seg;
+  d.n0 = (tile - G.seg_tile0[seg]) * WS_BM;
+  d.kb0 = (int)(((long long)split * G.kb_total) / G.splits);
+  d.kb1 = (int)(((long long)(split + 1) * G.kb_total) / G.splits);
+}
+
+__device__ __forceinline__ int pm_first_unit(const PmGemm& G) {
+  const int g = (int)gridDim.x;
+  int u = ((int)blockIdx.x - G.rot) % g;
+  if (u < 0) u += g;
+  return u;
+}
+
+// Cursor over (GEMM phase, unit, k block) of this CTA, in schedule order, with the per-unit values the
+// producer needs for every stage worked out once per unit.
+struct PmCursor {
+  int opi;      // index into the phase list of the current GEMM phase (n_ops: done)
+  int u, kb, kb1;
+  const CUtensorMap* tw;   // weight map of the unit's segment
+  const CUtensorMap* tw2;  // gated: the up-projection map, else null
+  const CUtensorMap* tx;
+  int n0, xrow;            // weight-tile row, activation-tile row
+  uint32_t bytes, xoff;    // bytes one stage receives; offset of the activation tile inside the stage
+  __device__ __forceinline__ void seek(const PmSmem& S, const PmParams& P) {     // first stage at or after (opi, u)
+    while (opi < S.n_ops) {
+      if (S.op[opi].kind == PH_GEMM) {
+        const int gi = S.op[opi].gemm;
+        const PmGemm& G = S.g[gi];
+        if (u < 0) u = pm_first_unit(G);
+        if (u < G.units) {
+          PmUnit d;
+          pm_decode(G, u, d);
+          kb = d.kb0; kb1 = d.kb1;
+          const bool gated = G.mode == 4;
+          tw = &P.tm[gi][d.seg]; tw2 = gated ? &P.tm[gi][1] : nullptr; tx = &P.tm[gi][3];
+          n0 = d.n0; xrow = d.rb * G.rows_per_block;
+          xoff = gated ? 2 * WS_W_BYTES : WS_W_BYTES;
+          bytes = xoff + (uint32_t)G.rows_per_block * WS_BK * 2;
+          return;
+        }
+      }
+      ++opi;
+      u = -1;
+    }
+  }
+  __device__ __forceinline__ void init(const PmSmem& S, const PmParams& P) { opi = 0; u = -1; kb = 0; kb1 = 0; seek(S, P); }
+  __device__ __forceinline__ bool done(const PmSmem& S) const { return opi >= S.n_ops; }
+  __device__ __forceinline__ void next(const PmSmem& S, const PmParams& P) {
+    if (++kb < kb1) return;
+    u += (int)gridDim.x;
+    seek(S, P);
+  }
+};
+
+}  // namespace moa
