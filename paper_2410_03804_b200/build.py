@@ -15,7 +15,7 @@ def _newest_source() -> float:
     t = 0.0
     for root in (CSRC, os.path.join(os.path.dirname(HERE), "include")):
         for f in os.listdir(root):
-            if f.endswith((".cu", ".cuh", ".h")):
+            if f.endswith((".cu", ".cuh", ".h", ".inc")):
                 t = max(t, os.path.getmtime(os.path.join(root, f)))
     return t
 

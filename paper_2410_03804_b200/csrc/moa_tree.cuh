@@ -9,7 +9,8 @@ namespace moa {
 // Byte offsets inside the caller-owned tree blob.
 struct TreeLayout {
   int nb, B, D, P, NS;     // sequences, breadth, depth, pool size per sequence, tree K/V slots per sequence
-  size_t status;           // int[4]
+  size_t status;           // int[8]: [0] status word, [4..6] grid-barrier counter, abort word, exit counter
+  size_t flags;            // int[256 * 32]: per-CTA grid-barrier flags of the fused kernels, one 128-byte line each
   size_t root_tok;         // int[nb]
   size_t frontier;         // int[nb*B]        pool index of each frontier node (-1: the root)
   size_t row_tok;          // int[2][nb*B]     token of each row, double-buffered by step parity
@@ -27,7 +28,8 @@ __host__ inline TreeLayout make_tree_layout(int nb, int B, int D, int hkv, int d
   L.NS = 1 + B * (D - 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
-  L.status = take(4 * sizeof(int));
+  L.status = take(8 * sizeof(int));
+  L.flags = take((size_t)256 * 32 * sizeof(int));
   L.root_tok = take((size_t)nb * sizeof(int));
   L.frontier = take((size_t)nb * B * sizeof(int));
   L.row_tok = take((size_t)2 * nb * B * sizeof(int));
