@@ -88,7 +88,9 @@ typedef struct {
   void *ca_k, *ca_v;        /* T [max_batch, max_ctx, ca_hkv, head_dim]: cross-attention keys / values   */
   void *sa_k, *sa_v;        /* T [max_batch, max_ctx, sa_hkv, head_dim]: rotated self-attention prefix   */
   int32_t *ca_len, *sa_len; /* device int32 [max_batch]: valid positions; written only by the library    */
-  void *tree;               /* device blob of moa_state_bytes().tree_bytes: node pool, frontier, tree K/V */
+  void *tree;               /* device blob of moa_state_bytes().tree_bytes: node pool, frontier, tree K/V, barrier
+                               words of the fused kernels. ZERO IT ONCE after allocating it (and again after a call
+                               reported MOA_ERR_TIMEOUT through moa_state_status) */
   int32_t *ca_len_host, *sa_len_host; /* HOST int32 [max_batch]: mirrors kept by the library             */
   int32_t step;             /* HOST: draft steps done since moa_tree_begin, -1 before it; library-owned  */
 } moa_state;
@@ -185,6 +187,15 @@ moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
  * Do not use inside a stream capture. */
 moa_status moa_profile_begin(moa_ctx *ctx);
 moa_status moa_profile_end(moa_ctx *ctx, double *ms_total, int32_t *launches);
+/* Phase timing of the LAST fused launch (on the bf16 path a drafter forward or an LSA pass runs as one
+ * persistent kernel made of phases separated by grid-wide barriers). Valid when that launch was made between
+ * moa_profile_begin and moa_profile_end with the same workspace. us_out[i] = microseconds phase i took on CTA 0
+ * including its closing barrier, wait_us_out[i] (may be NULL) = the part of it CTA 0 spent in that barrier,
+ * kind_out[i] = its kind (0 GEMM, 1 embed+norm, 2 row norm, 3 residual+norm, 4 rotary, 5 attention,
+ * 6 attention merge, 7 SwiGLU, 8 sum+cast, 9 layer mean+norm, 10 cache append, 11 LM-head merge).
+ * Synchronises the stream. HOST output arrays of `cap` entries. */
+moa_status moa_profile_phases(moa_ctx *ctx, const void *ws, size_t ws_bytes, int32_t cap, double *us_out,
+                              double *wait_us_out, int32_t *kind_out, int32_t *n_out, void *stream);
 /* Kernels launched so far by this host thread through the library. */
 int64_t moa_launch_count(void);
 

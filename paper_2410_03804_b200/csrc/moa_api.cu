@@ -9,6 +9,7 @@
 
 #include "moa_attn.cuh"
 #include "moa_basic.cuh"
+#include "moa_phases.cuh"
 #include "moa_tree.cuh"
 #include "moa_wstream.cuh"
 
@@ -40,6 +41,10 @@ struct moa_ctx {
   WeightMap wmap[WMAP_MAX];
   int n_wmap;
   bool fast;           // weight-streaming tcgen05 GEMMs usable
+  bool coop;           // cooperative launches available: the phase-machine kernels are used
+  int smem_optin;      // largest dynamic shared memory a CTA may ask for
+  int last_n_ops;      // phase kinds of the last fused launch (for moa_profile_phases)
+  int last_kinds[PM_MAX_OPS];
   // measurement hooks: event pairs around the LM-head launches
   bool prof_on;
   int prof_n;
@@ -51,7 +56,7 @@ struct moa_ctx {
 // workspace carving (same arithmetic in moa_state_bytes and in the calls)
 // ---------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, q32, total;
+  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, q32, trace, total;
   int rows_cap, draft_rows, chunk_tok, part_rows, wide;
   long long att_units;   // (row, head, part) triples the split-attention partial buffers hold
 };
@@ -77,22 +82,24 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
   p.xres = take((size_t)p.rows_cap * dmax * sizeof(float));      // residual stream, fp32
-  p.xn = take((size_t)p.rows_cap * dmax * elt);                  // normalised GEMM operand, T
+  const size_t xpad = 128;                                       // an X buffer's low-order half starts up to 128 rows in
+  p.xn = take(((size_t)p.rows_cap + xpad) * dmax * elt);         // normalised GEMM operand, T
   p.part = take((size_t)p.part_rows * p.wide * sizeof(float));   // GEMM outputs: K-split partial planes, fp32
-  p.narrow = take((size_t)p.rows_cap * narrow * elt);            // q|k|v or silu(gate)*up, T
-  p.obuf = take((size_t)p.rows_cap * omax * elt);                // attention output, T
+  p.narrow = take(((size_t)p.rows_cap + xpad) * narrow * elt);   // q|k|v or silu(gate)*up, T
+  p.obuf = take(((size_t)p.rows_cap + xpad) * omax * elt);       // attention output, T
   p.logits = take(elt == 4 ? (size_t)p.draft_rows * c.vocab * sizeof(float) : 256);   // fp32 path only
   p.pmax = take(n_sub * p.draft_rows * sizeof(float));           // LM-head partials per 32-row vocabulary slice
   p.psum = take(n_sub * p.draft_rows * sizeof(float));
   p.cval = take(n_sub * p.draft_rows * c.tree_topk * sizeof(float));
   p.cid = take(n_sub * p.draft_rows * c.tree_topk * sizeof(int));
   p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));   // LSA output rows, fp32
-  p.kvn = take((size_t)chunk_tok * c.d_stack * elt);             // their normalised copy, T
+  p.kvn = take(((size_t)chunk_tok + xpad) * c.d_stack * elt);    // their normalised copy, T
   const int gmax = imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), hqmax = imax(c.sa_hq, c.ca_hq);
   p.att_units = (long long)c.tree_topk * gmax * 2 * 160 + 2ll * p.draft_rows * hqmax;
   p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
   p.att_ml = take(elt == 2 ? (size_t)p.att_units * 2 * sizeof(float) : 256);           // their (max, sum)
   p.q32 = take(elt == 2 ? (size_t)p.draft_rows * hqmax * c.head_dim * sizeof(float) : 256);   // draft-step queries, fp32
+  p.trace = take((2 * PM_MAX_OPS + 2) * sizeof(unsigned long long));   // phase timestamps of the last fused launch
   p.total = o;
   return p;
 }
@@ -152,7 +159,7 @@ static const WeightMap* find_wmap(const moa_ctx* ctx, const void* w) {
 
 // K-split count: best use of the SMs' waves, fewest splits among near-equal choices.
 static int pick_splits(int tiles, int kb_total, int R, int part_rows, int sms) {
-  const int smax = imax(1, imin(imin(16, kb_total), part_rows / imax(R, 1)));
+  const int smax = imax(1, imin(imin(8, kb_total), part_rows / imax(R, 1)));
   int best = 1;
   double best_eff = 0.0;
   for (int s = 1; s <= smax; ++s) {
@@ -609,6 +616,377 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
 }
 
 // ---------------------------------------------------------------------------------------------
+// phase-machine paths (bf16): one cooperative kernel per drafter forward / per LSA pass
+// ---------------------------------------------------------------------------------------------
+struct PmBuild {
+  PmParams P;
+  moa_ctx* ctx;
+  int NB, xsplit, lo_rows, grid;
+  int unit_run;          // units scheduled so far (rotates the CTA that gets unit 0 of the next GEMM)
+  size_t attn_bytes;
+  bool dense;
+  moa_status err;
+};
+
+static void pm_init(PmBuild& b, moa_ctx* ctx, int R, bool dense, void* tree, const TreeLayout& L, char* ws,
+                    const Workspace& p) {
+  memset(&b.P, 0, sizeof(b.P));
+  b.ctx = ctx;
+  b.dense = dense;
+  b.grid = ctx->sm_count;
+  b.unit_run = 0;
+  b.attn_bytes = 4096;
+  b.err = MOA_OK;
+  if (dense) { b.NB = 256; b.xsplit = 0; }
+  else if (R <= 16) { b.NB = 32; b.xsplit = 1; }
+  else if (R <= 32) { b.NB = 64; b.xsplit = 1; }
+  else if (R <= 64) { b.NB = 128; b.xsplit = 1; }
+  else if (R <= 128) { b.NB = 256; b.xsplit = 1; }
+  else { b.NB = 256; b.xsplit = 0; }
+  b.lo_rows = b.xsplit ? b.NB / 2 : 0;
+  b.P.sync = (int*)((char*)tree + L.status) + 4;
+  b.P.flags = (int*)((char*)tree + L.flags);
+  b.P.status = (int*)((char*)tree + L.status);
+  b.P.trace = ctx->prof_on ? (unsigned long long*)(ws + p.trace) : nullptr;
+}
+
+static PmOp* pm_op(PmBuild& b, int kind, int gemm, int rows, int cols) {
+  if (b.P.n_ops >= PM_MAX_OPS) { b.err = MOA_ERR_SHAPE; return &b.P.op[PM_MAX_OPS - 1]; }
+  PmOp* op = &b.P.op[b.P.n_ops++];
+  memset(op, 0, sizeof(*op));
+  op->kind = kind; op->gemm = gemm; op->rows = rows; op->cols = cols;
+  return op;
+}
+
+// Adds a GEMM phase: X buffer [R (+ low half), K] times up to three weight matrices. mode as in PmGemm.
+static int pm_gemm(PmBuild& b, const void* X, int R, int K, int nseg, const void* const* W, const int* N, int mode,
+                   float* part, int part_rows) {
+  if (b.P.n_gemms >= PM_MAX_GEMMS) { b.err = MOA_ERR_SHAPE; return 0; }
+  const int gi = b.P.n_gemms++;
+  PmGemm& G = b.P.g[gi];
+  memset(&G, 0, sizeof(G));
+  G.n_seg = nseg; G.mode = mode; G.R = R; G.xsplit = b.xsplit;
+  int tiles = 0, col = 0;
+  for (int i = 0; i < nseg; ++i) {
+    const WeightMap* wm = find_wmap(b.ctx, W[i]);
+    if (!wm) { b.err = MOA_ERR_SHAPE; return gi; }
+    b.P.tm[gi][i] = wm->tm;
+    G.seg_n[i] = N[i]; G.seg_tile0[i] = tiles; G.seg_col[i] = col;
+    tiles += (N[i] + WS_BM - 1) / WS_BM;
+    col += N[i];
+  }
+  if (mode == 4) tiles = (N[0] + WS_BM - 1) / WS_BM;      // gate and up tiles travel in pairs
+  G.tiles_total = tiles;
+  G.kb_total = K / WS_BK;
+  G.rows_per_block = mode == 4 ? 128 : b.NB;
+  G.row_blocks = b.dense && mode >= 2 ? (R + G.rows_per_block - 1) / G.rows_per_block : 1;
+  G.splits = mode == 0 ? pick_splits(tiles, G.kb_total, R, part_rows, b.grid) : 1;
+  G.units = tiles * G.splits * G.row_blocks;
+  G.rot = b.unit_run % b.grid;
+  b.unit_run += G.units;
+  G.ldo = col;
+  G.plane = (size_t)R * col;
+  G.out = part;
+  const int rows_total = b.xsplit ? b.lo_rows + R : R;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows_total};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)WS_BK, (cuuint32_t)G.rows_per_block};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = b.ctx->encode(&b.P.tm[gi][3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled (activations) failed (%d)", (int)r);
+    b.err = MOA_ERR_CUDA;
+  }
+  pm_op(b, PH_GEMM, gi, R, col);
+  return gi;
+}
+
+template <int NB>
+static moa_status pm_launch_nb(cudaStream_t s, const PmParams& P, int grid, size_t smem) {
+  static size_t attr = 0;
+  if (smem > attr) {
+    cudaError_t e = cudaFuncSetAttribute(phase_machine_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+      snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+      return MOA_ERR_CUDA;
+    }
+    attr = smem;
+  }
+  void* args[1] = {(void*)&P};
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)phase_machine_kernel<NB>, dim3(grid), dim3(PM_THREADS), args,
+                                              smem, s);
+  ++g_launches;
+  if (e != cudaSuccess) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "cooperative launch: %s", cudaGetErrorString(e));
+    return MOA_ERR_CUDA;
+  }
+  return MOA_OK;
+}
+
+static moa_status pm_launch(PmBuild& b, cudaStream_t s) {
+  if (b.err != MOA_OK) return b.err;
+  b.ctx->last_n_ops = b.P.n_ops;
+  for (int i = 0; i < b.P.n_ops; ++i) b.ctx->last_kinds[i] = b.P.op[i].kind;
+  const int stage = WS_W_BYTES + b.NB * WS_BK * 2;
+  const size_t fixed = PM_FIXED_SMEM;                     // alignment slack, barriers, descriptor copies
+  const size_t budget = (size_t)b.ctx->smem_optin;
+  const size_t ring_room = budget - fixed - (b.dense ? 0 : b.attn_bytes);
+  int stages = (int)(ring_room / stage);
+  if (stages > PM_MAX_STAGES) stages = PM_MAX_STAGES;
+  if (stages < 2 || (b.dense && (size_t)stages * stage < b.attn_bytes)) return MOA_ERR_SHAPE;
+  b.P.stages = stages;
+  b.P.alias_attn = b.dense ? 1 : 0;
+  b.P.attn_off = b.dense ? 0u : (uint32_t)((size_t)stages * stage + (PM_FIXED_SMEM - 1024));
+  const size_t smem = fixed + (size_t)stages * stage + (b.dense ? 0 : b.attn_bytes);
+  switch (b.NB) {
+    case 32: return pm_launch_nb<32>(s, b.P, b.grid, smem);
+    case 64: return pm_launch_nb<64>(s, b.P, b.grid, smem);
+    case 128: return pm_launch_nb<128>(s, b.P, b.grid, smem);
+    default: return pm_launch_nb<256>(s, b.P, b.grid, smem);
+  }
+}
+
+// attention phase + (when it has several parts) the merge of the parts; result in the X buffer `out`
+static void pm_attention_ops(PmBuild& b, const Workspace& p, char* ws, int R, int n_seq, int rows_per_seq, int hq, int hkv,
+                             int dh, const bf16* q16, const float* q32, int q_ld, int q_gemm, const bf16* kA,
+                             const bf16* vA, int capA, int posA_ld, const int* lenA, int nA_fixed, int max_len,
+                             const bf16* kB, const bf16* vB, int capB, const int* slotsB, int slots_ld, int nB,
+                             int n_slots, bf16* out) {
+  const int group = hq / hkv, Qn = rows_per_seq * group;
+  const int q_tiles = (Qn + PM_WWARPS * 16 - 1) / (PM_WWARPS * 16);
+  const int has_tree = (kB != nullptr && nB > 0) ? 1 : 0;
+  const int blocks = imax(1, (max_len + PM_KB - 1) / PM_KB);
+  int n_split = imax(1, imin(blocks, b.grid / imax(1, n_seq * hkv * q_tiles) - has_tree));
+  const long long per_part = (long long)R * hq;
+  while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
+  if (n_split + has_tree > 1 && per_part * (n_split + has_tree) > p.att_units) { b.err = MOA_ERR_WORKSPACE; return; }
+  const int n_parts = n_split + has_tree;
+  {
+    const int q_rows = Qn < PM_WWARPS * 16 ? ((Qn + 15) & ~15) : PM_WWARPS * 16;
+    const size_t need = (size_t)2 * q_rows * dh * 2 + (size_t)2 * PM_KVST * PM_KB * dh * 2 + 512;
+    if (need > b.attn_bytes) b.attn_bytes = need;
+  }
+  PmOp* op = pm_op(b, PH_ATTN, q_gemm, R, n_seq);
+  op->p[0] = q16; op->p[1] = q32; op->p[2] = kA; op->p[3] = vA; op->p[4] = lenA; op->p[5] = kB; op->p[6] = vB;
+  op->p[7] = slotsB; op->p[8] = ws + p.att_o; op->p[9] = ws + p.att_ml; op->p[10] = out;
+  op->i[0] = q_ld; op->i[1] = hq; op->i[2] = hkv; op->i[3] = rows_per_seq; op->i[4] = capA; op->i[5] = posA_ld;
+  op->i[6] = nA_fixed; op->i[7] = capB; op->i[8] = slots_ld; op->i[9] = nB; op->i[10] = n_slots; op->i[11] = n_split;
+  op->i[12] = q_gemm >= 0 ? b.P.g[q_gemm].splits : 1; op->i[13] = b.lo_rows; op->i[14] = dh;
+  op->f[0] = 1.4426950408889634f / sqrtf((float)dh);
+  if (n_parts > 1) {
+    PmOp* c = pm_op(b, PH_COMBINE, -1, R, hq);
+    c->p[0] = ws + p.att_o; c->p[1] = ws + p.att_ml; c->p[2] = out;
+    c->i[0] = n_parts; c->i[1] = dh; c->i[2] = b.lo_rows;
+  }
+}
+
+static void pm_resnorm(PmBuild& b, int gemm, int R, int K, float* xres, const void* gain, bf16* xn, void* hidden,
+                       float eps) {
+  PmOp* op = pm_op(b, PH_RESNORM, gemm, R, K);
+  op->p[2] = gain; op->p[3] = xres; op->p[4] = xn; op->p[5] = hidden;
+  op->i[1] = b.lo_rows; op->f[0] = eps;
+}
+
+// MLP phases on xn = RMSNorm(xres): [gate | up] GEMM, SwiGLU, down GEMM. Returns the down GEMM's index.
+static int pm_mlp(PmBuild& b, const Workspace& p, char* ws, int R, int K, int F, const void* wgate, const void* wup,
+                  const void* wdown) {
+  float* part = (float*)(ws + p.part);
+  bf16* xn = (bf16*)(ws + p.xn);
+  bf16* h = (bf16*)(ws + p.narrow);
+  const void* W2[2] = {wgate, wup};
+  const int N2[2] = {F, F};
+  const int g = pm_gemm(b, xn, R, K, 2, W2, N2, 0, part, p.part_rows);
+  PmOp* op = pm_op(b, PH_SILU, g, R, F);
+  op->p[0] = h; op->i[1] = b.lo_rows;
+  const void* W1[1] = {wdown};
+  const int N1[1] = {K};
+  return pm_gemm(b, h, R, F, 1, W1, N1, 0, part, p.part_rows);
+}
+
+static moa_status draft_step_pm(moa_ctx* ctx, moa_state* st, int batch, int* topk_id, float* topk_logp, void* hidden_out,
+                                char* ws, const Workspace& p, cudaStream_t s) {
+  const moa_config& c = ctx->c;
+  const moa_weights& w = ctx->w;
+  const TreeLayout& L = ctx->tl;
+  const TreePtrs tp = tree_ptrs(st->tree, L);
+  const int step = st->step, B = c.tree_topk, D = c.tree_depth;
+  const int R = step == 0 ? batch : batch * B;
+  const int rows_per_seq = step == 0 ? 1 : B;
+  const int nbB = c.max_batch * B;
+  const int E = c.d_model, dh = c.head_dim, V = c.vocab;
+  const int cur = step & 1;
+  const int* row_tok = tp.row_tok + (size_t)cur * nbB;
+  const int* row_anc = tp.row_anc + (size_t)cur * nbB * D;
+  bf16* tk = (bf16*)((char*)st->tree + L.tk);
+  bf16* tv = (bf16*)((char*)st->tree + L.tv);
+  float* xres = (float*)(ws + p.xres);
+  bf16* xn = (bf16*)(ws + p.xn);
+  bf16* obuf = (bf16*)(ws + p.obuf);
+  float* q32 = (float*)(ws + p.q32);
+  float* part = (float*)(ws + p.part);
+  int max_sa = 0, max_ca = 0;
+  for (int b = 0; b < batch; ++b) {
+    max_sa = imax(max_sa, st->sa_len_host[b]);
+    max_ca = imax(max_ca, st->ca_len_host[b]);
+  }
+  PmBuild b;
+  pm_init(b, ctx, R, false, st->tree, L, ws, p);
+  const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh, cq = c.ca_hq * dh, ckv = c.ca_hkv * dh;
+  // ---- self-attention block ----
+  {
+    PmOp* op = pm_op(b, PH_EMBED_NORM, -1, R, E);
+    op->p[0] = w.embed; op->p[1] = row_tok; op->p[2] = w.sa_norm1; op->p[3] = xres; op->p[4] = xn;
+    op->i[0] = V; op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
+  }
+  {
+    const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
+    const int N3[3] = {nq, nkv, nkv};
+    const int g = pm_gemm(b, xn, R, E, 3, W3, N3, 0, part, p.part_rows);
+    PmOp* op = pm_op(b, PH_ROPE, g, R, nq + 2 * nkv);
+    op->p[0] = q32; op->p[1] = tk; op->p[2] = tv; op->p[3] = st->sa_len;
+    op->i[0] = c.sa_hq; op->i[1] = c.sa_hkv; op->i[2] = dh; op->i[3] = step; op->i[4] = B; op->i[5] = L.NS;
+    op->f[0] = c.sa_rope_theta;
+  }
+  pm_attention_ops(b, p, ws, R, batch, rows_per_seq, c.sa_hq, c.sa_hkv, dh, nullptr, q32, nq, -1, (const bf16*)st->sa_k,
+                   (const bf16*)st->sa_v, c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
+                   step == 0 ? 1 : 1 + step * B, obuf);
+  {
+    const void* W1[1] = {w.sa_wo};
+    const int N1[1] = {E};
+    const int g = pm_gemm(b, obuf, R, nq, 1, W1, N1, 0, part, p.part_rows);
+    pm_resnorm(b, g, R, E, xres, w.sa_norm2, xn, nullptr, c.rms_eps);
+  }
+  {
+    const int g = pm_mlp(b, p, ws, R, E, c.sa_mlp, w.sa_wgate, w.sa_wup, w.sa_wdown);
+    // ---- cross-attention block ----
+    pm_resnorm(b, g, R, E, xres, w.ca_normq, xn, nullptr, c.rms_eps);
+  }
+  {
+    const void* W1[1] = {w.ca_wq};
+    const int N1[1] = {cq};
+    const int g = pm_gemm(b, xn, R, E, 1, W1, N1, 0, part, p.part_rows);
+    pm_attention_ops(b, p, ws, R, batch, rows_per_seq, c.ca_hq, c.ca_hkv, dh, nullptr, part, cq, g, (const bf16*)st->ca_k,
+                     (const bf16*)st->ca_v, c.max_ctx, ckv, st->ca_len, 0, max_ca, nullptr, nullptr, 0, nullptr, 0, 0, 0,
+                     obuf);
+  }
+  {
+    const void* W1[1] = {w.ca_wo};
+    const int N1[1] = {E};
+    const int g = pm_gemm(b, obuf, R, cq, 1, W1, N1, 0, part, p.part_rows);
+    pm_resnorm(b, g, R, E, xres, w.ca_norm2, xn, nullptr, c.rms_eps);
+  }
+  {
+    const int g = pm_mlp(b, p, ws, R, E, c.ca_mlp, w.ca_wgate, w.ca_wup, w.ca_wdown);
+    // ---- LM head, log-softmax, top-B ----
+    pm_resnorm(b, g, R, E, xres, w.final_norm, xn, hidden_out, c.rms_eps);
+  }
+  {
+    const void* W1[1] = {w.lm_head};
+    const int N1[1] = {V};
+    const int g = pm_gemm(b, xn, R, E, 1, W1, N1, 1, nullptr, 0);
+    PmGemm& G = b.P.g[g];
+    G.B = B;
+    G.p_max = (float*)(ws + p.pmax); G.p_sum = (float*)(ws + p.psum);
+    G.c_val = (float*)(ws + p.cval); G.c_id = (int*)(ws + p.cid);
+    G.n_sub = 4 * G.tiles_total;
+    if (G.n_sub > PM_MERGE_OWN * PM_WORKERS) return MOA_ERR_SHAPE;       // ruled out by pm_usable()
+    PmOp* op = pm_op(b, PH_MERGE, g, R, V);
+    op->p[0] = topk_id; op->p[1] = topk_logp; op->i[1] = B;
+  }
+  return pm_launch(b, s);
+}
+
+// One LSA pass over nt tokens (rows t0*S .. of h_stack): small regime (split planes + glue) or dense regime.
+static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt, int t0, const SeqSplit& split,
+                              bf16* kv_out, char* ws, const Workspace& p, cudaStream_t s) {
+  const moa_config& c = ctx->c;
+  const moa_weights& w = ctx->w;
+  const TreeLayout& L = ctx->tl;
+  const int S = c.n_stack, D = c.d_stack, dh = c.head_dim, F = c.lsa_mlp;
+  const int nq = c.lsa_hq * dh, nkv = c.lsa_hkv * dh, ld = nq + 2 * nkv, ckv = c.ca_hkv * dh;
+  const int R = nt * S;
+  const bool dense = R > 256;
+  float* xres = (float*)(ws + p.xres);
+  bf16* xn = (bf16*)(ws + p.xn);
+  bf16* narrow = (bf16*)(ws + p.narrow);
+  bf16* obuf = (bf16*)(ws + p.obuf);
+  float* part = (float*)(ws + p.part);
+  float* kvf = (float*)(ws + p.kvf);
+  bf16* kvn = (bf16*)(ws + p.kvn);
+  PmBuild b;
+  pm_init(b, ctx, R, dense, st->tree, L, ws, p);
+  b.P.split = split;
+  {
+    PmOp* op = pm_op(b, PH_ROWS_NORM, -1, R, D);
+    op->p[0] = x; op->p[2] = w.lsa_norm1; op->p[3] = xres; op->p[4] = xn;
+    op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
+  }
+  const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
+  const int N3[3] = {nq, nkv, nkv};
+  const void* Wo[1] = {w.lsa_wo};
+  const int No[1] = {D};
+  int g_down;
+  if (!dense) {
+    const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 0, part, p.part_rows);
+    PmOp* op = pm_op(b, PH_SUMCAST, g0, R, ld);
+    op->p[0] = narrow;
+    pm_attention_ops(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, nullptr, ld, -1, narrow + nq, narrow + nq + nkv,
+                     S, ld, nullptr, S, S, nullptr, nullptr, 0, nullptr, 0, 0, 0, obuf);
+    const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 0, part, p.part_rows);
+    pm_resnorm(b, g1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
+    g_down = pm_mlp(b, p, ws, R, D, F, w.lsa_wgate, w.lsa_wup, w.lsa_wdown);
+  } else {
+    const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 2, nullptr, 0);
+    b.P.g[g0].out16 = narrow; b.P.g[g0].ld16 = ld;
+    pm_attention_ops(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, nullptr, ld, -1, narrow + nq, narrow + nq + nkv,
+                     S, ld, nullptr, S, S, nullptr, nullptr, 0, nullptr, 0, 0, 0, obuf);
+    const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 3, xres, 0);
+    b.P.g[g1].ldo = D;
+    pm_resnorm(b, -1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
+    const void* W2[2] = {w.lsa_wgate, w.lsa_wup};
+    const int N2[2] = {F, F};
+    const int g2 = pm_gemm(b, xn, R, D, 2, W2, N2, 4, nullptr, 0);
+    b.P.g[g2].out16 = narrow; b.P.g[g2].ld16 = F;
+    const void* Wd[1] = {w.lsa_wdown};
+    const int g3 = pm_gemm(b, narrow, R, F, 1, Wd, No, 3, xres, 0);
+    b.P.g[g3].ldo = D;
+    g_down = -1;
+  }
+  {
+    PmOp* op = pm_op(b, PH_MEAN_NORM, g_down, nt, D);
+    op->p[0] = xres; op->p[1] = kvf; op->p[2] = kv_out; op->p[3] = w.ca_normkv; op->p[4] = kvn;
+    op->i[0] = S; op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
+  }
+  {
+    const void* W2[2] = {w.ca_wk, w.ca_wv};
+    const int N2[2] = {ckv, ckv};
+    const int g = pm_gemm(b, kvn, nt, D, 2, W2, N2, 0, part, p.part_rows);
+    PmOp* op = pm_op(b, PH_CACHE_APPEND, g, nt, 2 * ckv);
+    op->p[0] = st->ca_len; op->p[1] = st->ca_k; op->p[2] = st->ca_v;
+    op->i[0] = ckv; op->i[1] = c.max_ctx; op->i[2] = t0;
+  }
+  return pm_launch(b, s);
+}
+
+static bool pm_usable(const moa_ctx* ctx) {
+  if (!ctx->fast || !ctx->coop || ctx->c.dtype != MOA_BF16 || ctx->sm_count > 256) return false;
+  const moa_weights& w = ctx->w;
+  const void* all[] = {w.lm_head, w.lsa_wq, w.lsa_wk, w.lsa_wv, w.lsa_wo, w.lsa_wgate, w.lsa_wup, w.lsa_wdown,
+                       w.sa_wq, w.sa_wk, w.sa_wv, w.sa_wo, w.sa_wgate, w.sa_wup, w.sa_wdown,
+                       w.ca_wq, w.ca_wk, w.ca_wv, w.ca_wo, w.ca_wgate, w.ca_wup, w.ca_wdown};
+  for (const void* m : all)
+    if (!find_wmap(ctx, m)) return false;
+  const moa_config& c = ctx->c;
+  const int widths[] = {c.d_model, c.d_stack, c.lsa_mlp, c.sa_mlp, c.ca_mlp};
+  for (int v : widths)
+    if (v % 64 != 0) return false;
+  if (4 * ((c.vocab + WS_BM - 1) / WS_BM) > PM_MERGE_OWN * PM_WORKERS) return false;
+  return true;
+}
+
+// ---------------------------------------------------------------------------------------------
 // exported functions
 // ---------------------------------------------------------------------------------------------
 extern "C" {
@@ -684,6 +1062,9 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
   ctx->encode = nullptr;
   ctx->n_wmap = 0;
   ctx->fast = false;
+  ctx->coop = prop.cooperativeLaunch != 0;
+  ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
+  ctx->last_n_ops = 0;
   if (cfg->dtype == MOA_BF16) {
     // tensor maps of every weight matrix whose inner dimension the streaming GEMM can take
     void* fn = nullptr;
@@ -772,6 +1153,29 @@ moa_status moa_profile_end(moa_ctx* ctx, double* ms_total, int32_t* launches) {
 
 int64_t moa_launch_count(void) { return g_launches; }
 
+moa_status moa_profile_phases(moa_ctx* ctx, const void* ws, size_t ws_bytes, int32_t cap, double* us_out,
+                              double* wait_us_out, int32_t* kind_out, int32_t* n_out, void* stream) {
+  if (!ctx || !ws || !us_out || !kind_out || !n_out) return MOA_ERR_NULL;
+  const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
+  if (chunk < 1) return MOA_ERR_WORKSPACE;
+  const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  unsigned long long t[2 * PM_MAX_OPS + 1];
+  cudaError_t e = cudaMemcpyAsync(t, (const char*)ws + p.trace, sizeof(t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_profile_phases: %s", cudaGetErrorString(e));
+    return MOA_ERR_CUDA;
+  }
+  const int n = ctx->last_n_ops < cap ? ctx->last_n_ops : cap;
+  for (int i = 0; i < n; ++i) {
+    us_out[i] = (double)(t[2 * i + 2] - t[2 * i]) * 1e-3;
+    if (wait_us_out) wait_us_out[i] = (double)(t[2 * i + 2] - t[2 * i + 1]) * 1e-3;
+    kind_out[i] = ctx->last_kinds[i];
+  }
+  *n_out = n;
+  return MOA_OK;
+}
+
 moa_status moa_state_bytes(const moa_ctx* ctx, int32_t lsa_chunk_tokens, size_t* tree_bytes, size_t* workspace_bytes) {
   if (!ctx) return MOA_ERR_NULL;
   if (lsa_chunk_tokens < 1) return MOA_ERR_SHAPE;
@@ -837,9 +1241,26 @@ moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, con
   const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
   const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
-  moa_status r = ctx->c.dtype == MOA_F32
-                     ? lsa_forward_t<float>(ctx, st, h_stack, split, kv_out, (char*)ws, p, (cudaStream_t)stream)
-                     : lsa_forward_t<bf16>(ctx, st, h_stack, split, kv_out, (char*)ws, p, (cudaStream_t)stream);
+  moa_status r;
+  if (pm_usable(ctx)) {
+    r = MOA_OK;
+    const int S = ctx->c.n_stack, D = ctx->c.d_stack;
+    // passes of at most 256 tokens (the key/value projection of a pass is one activation block)
+    const int per_pass = imin(p.chunk_tok, 256);
+    for (int t0 = 0; t0 < total && r == MOA_OK; t0 += per_pass) {
+      const int nt = imin(per_pass, total - t0);
+      r = lsa_pass_pm(ctx, st, (const bf16*)h_stack + (size_t)t0 * S * D, nt, t0, split,
+                      kv_out ? (bf16*)kv_out + (size_t)t0 * D : nullptr, (char*)ws, p, (cudaStream_t)stream);
+    }
+    if (r == MOA_OK) {
+      add_len_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(st->ca_len, split);
+      MOA_CHECK_LAUNCH();
+    }
+  } else {
+    r = ctx->c.dtype == MOA_F32
+            ? lsa_forward_t<float>(ctx, st, h_stack, split, kv_out, (char*)ws, p, (cudaStream_t)stream)
+            : lsa_forward_t<bf16>(ctx, st, h_stack, split, kv_out, (char*)ws, p, (cudaStream_t)stream);
+  }
   if (r == MOA_OK)
     for (int b = 0; b < batch; ++b) st->ca_len_host[b] += n_tok_host[b];
   return r;
@@ -887,6 +1308,8 @@ moa_status moa_draft_step(moa_ctx* ctx, moa_state* st, int32_t batch, int32_t* t
   const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
   const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  if (pm_usable(ctx))
+    return draft_step_pm(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream);
   return ctx->c.dtype == MOA_F32
              ? draft_step_t<float>(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream)
              : draft_step_t<bf16>(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream);

@@ -21,7 +21,7 @@ MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
-           "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end",
+           "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
 
 
@@ -95,6 +95,8 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_state_status.argtypes = [vp, C.POINTER(MoaState), vp]
     lib.moa_profile_begin.argtypes = [vp]
     lib.moa_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
+    lib.moa_profile_phases.argtypes = [vp, vp, sz, i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i32),
+                                       C.POINTER(i32), vp]
     lib.moa_launch_count.argtypes = []
     for n in EXPORTS:
         if n not in ("moa_destroy", "moa_status_str", "moa_last_cuda_error", "moa_launch_count"):
@@ -286,6 +288,18 @@ class MoA:
         ms, n = C.c_double(), C.c_int32()
         _check(self.lib.moa_profile_end(self.h, C.byref(ms), C.byref(n)), "moa_profile_end")
         return ms.value, n.value
+
+    PHASE_KINDS = ["gemm", "embed_norm", "rows_norm", "res_norm", "rope", "attention", "attn_merge", "swiglu",
+                   "sum_cast", "mean_norm", "cache_append", "lm_merge"]
+
+    def moa_profile_phases(self, stream=None):
+        """[(kind name, microseconds, of which in the closing barrier)] of the last fused launch made while
+        profiling was on."""
+        cap = 32
+        us, wait, kinds, n = (C.c_double * cap)(), (C.c_double * cap)(), (C.c_int32 * cap)(), C.c_int32()
+        _check(self.lib.moa_profile_phases(self.h, _ptr(self.ws), self.ws_bytes, cap, us, wait, kinds, C.byref(n),
+                                           _stream(stream)), "moa_profile_phases")
+        return [(self.PHASE_KINDS[kinds[i]], us[i], wait[i]) for i in range(n.value)]
 
     def moa_launch_count(self) -> int:
         return int(self.lib.moa_launch_count())
