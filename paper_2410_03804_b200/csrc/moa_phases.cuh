@@ -23,6 +23,36 @@
 
 namespace moa {
 
+// A chain of tcgen05.mma instructions that accumulate into the same TMEM tile is serialised by the tensor
+// pipe's latency, and with few activation rows (small N) that latency, not the math, sets the pace: four
+// dependent K=16 steps per 16 KB weight stage cost about as much time as HBM needs to deliver the stage. So the
+// k-steps of a stage rotate over PM_ACC independent accumulators, and the epilogue adds them up.
+template <int NB>
+__host__ __device__ constexpr int pm_acc() { return NB <= 64 ? 4 : (NB <= 128 ? 2 : 1); }
+
+// 16 accumulator columns starting at column c of the unit's buffer: sum over the independent accumulators and,
+// for a split X buffer, over the hi and lo halves.
+template <int NB>
+__device__ __forceinline__ void pm_ld16(uint32_t taddr, int c, int xsplit, float* v) {
+  tc_ld16(taddr + c, v);
+#pragma unroll
+  for (int a = 1; a < pm_acc<NB>(); ++a) {
+    float w[16];
+    tc_ld16(taddr + a * NB + c, w);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] += w[i];
+  }
+  if (xsplit) {
+#pragma unroll
+    for (int a = 0; a < pm_acc<NB>(); ++a) {
+      float w[16];
+      tc_ld16(taddr + a * NB + NB / 2 + c, w);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] += w[i];
+    }
+  }
+}
+
 // ---- epilogue of one GEMM unit: TMEM accumulator -> global, by the four epilogue warps ----
 template <int NB>
 __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, uint32_t taddr, int q, int lane) {
@@ -35,13 +65,7 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
 #pragma unroll 1
     for (int c0 = 0; c0 < rows; c0 += 16) {
       float v[16];
-      tc_ld16(taddr + c0, v);
-      if (Gm.xsplit) {
-        float w[16];
-        tc_ld16(taddr + NB / 2 + c0, w);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] += w[i];
-      }
+      pm_ld16<NB>(taddr, c0, Gm.xsplit, v);
       if (valid) {
 #pragma unroll
         for (int i = 0; i < 16; ++i)
@@ -53,7 +77,7 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
 #pragma unroll 1
     for (int c0 = 0; c0 < rows; c0 += 16) {
       float v[16];
-      tc_ld16(taddr + c0, v);
+      pm_ld16<NB>(taddr, c0, 0, v);
       if (valid) {
         if (Gm.mode == 2) {
 #pragma unroll
@@ -90,13 +114,7 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
 #pragma unroll 1
     for (int c0 = 0; c0 < rows; c0 += 16) {
       float v[16];
-      tc_ld16(taddr + c0, v);
-      if (Gm.xsplit) {
-        float w[16];
-        tc_ld16(taddr + NB / 2 + c0, w);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] += w[i];
-      }
+      pm_ld16<NB>(taddr, c0, Gm.xsplit, v);
 #pragma unroll 1
       for (int i = 0; i < 16; ++i) {
         const int r = c0 + i;
@@ -133,13 +151,67 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
   }
 }
 
+// ---- MMA issuer role (one thread): walks the static schedule, one tcgen05.mma group per ring stage ----
+template <int NB>
+__device__ __noinline__ void pm_mma_role(const PmSmem& S, uint32_t base, uint32_t bar0, uint32_t tmem_base, int STAGES,
+                                         volatile int* abort_flag) {
+  constexpr int STAGE_BYTES = pm_stage_bytes<NB>();
+  constexpr int ACC = pm_acc<NB>();
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (PM_MAX_STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * PM_MAX_STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * PM_MAX_STAGES + 2 + b); };
+  const int G = (int)gridDim.x;
+  int slot = 0;                     // ring slot and its phase parity, advanced stage by stage
+  uint32_t slot_ph = 0;
+  const uint64_t desc0 = umma_desc_sw128(base);   // descriptor of slot 0; slots lie STAGE_BYTES apart (< 256 KB in all)
+  int j = 0;
+  bool ok = true;
+  for (int opi = 0; opi < S.n_ops && ok; ++opi) {
+    if (S.op[opi].kind != PH_GEMM) continue;
+    const PmGemm& Gm = S.g[S.op[opi].gemm];
+    const bool gated = Gm.mode == 4;
+    const uint32_t idesc = umma_idesc_bf16(WS_BM, gated ? 128 : NB);
+    for (int u = pm_first_unit(Gm); u < Gm.units && ok; u += G, ++j) {
+      PmUnit d;
+      pm_decode(Gm, u, d);
+      const int buf = j & 1;
+      const uint32_t bph = (uint32_t)(j >> 1) & 1u;
+      if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(buf * ACC * NB);
+      for (int kb = d.kb0; kb < d.kb1; ++kb) {
+        if (!mbar_wait(full_bar(slot), slot_ph, abort_flag)) { ok = false; break; }
+        const uint64_t adesc = desc0 + (uint64_t)(slot * (STAGE_BYTES >> 4));
+        const uint64_t bdesc = adesc + (uint64_t)((gated ? 2 * WS_W_BYTES : WS_W_BYTES) >> 4);
+        const uint32_t acc0 = kb > d.kb0 ? 1u : 0u;
+#pragma unroll
+        for (int kk = 0; kk < WS_BK / 16; ++kk)   // k-step kk accumulates into accumulator kk % ACC
+          tc_mma_bf16(d_tmem + (uint32_t)((kk % ACC) * NB), adesc + 2u * kk, bdesc + 2u * kk, idesc,
+                      (acc0 | (kk >= ACC)) ? 1u : 0u);
+        if (gated) {
+          const uint64_t adesc2 = adesc + (uint64_t)(WS_W_BYTES >> 4);
+#pragma unroll
+          for (int kk = 0; kk < WS_BK / 16; ++kk)
+            tc_mma_bf16(d_tmem + 128u, adesc2 + 2u * kk, bdesc + 2u * kk, idesc, (acc0 | (kk > 0)) ? 1u : 0u);
+        }
+        tc_commit(empty_bar(slot));
+        if (++slot == STAGES) { slot = 0; slot_ph ^= 1u; }
+      }
+      if (ok) tc_commit(tfull_bar(buf));
+    }
+  }
+
+}
+
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
 template <int NB>
 __global__ void __launch_bounds__(PM_THREADS, 1) phase_machine_kernel(const __grid_constant__ PmParams P) {
   constexpr int STAGE_BYTES = pm_stage_bytes<NB>();
-  constexpr uint32_t TMEM_COLS = (2 * NB) < 32 ? 32 : (2 * NB);
+  constexpr int ACC = pm_acc<NB>();
+  constexpr uint32_t TMEM_COLS = 2 * ACC * NB;        // two buffers of ACC accumulators (64 .. 512 columns)
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -282,47 +354,7 @@ __global__ void __launch_bounds__(PM_THREADS, 1) phase_machine_kernel(const __gr
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      int j = 0;
-      bool ok = true;
-      for (int opi = 0; opi < S.n_ops && ok; ++opi) {
-        if (S.op[opi].kind != PH_GEMM) continue;
-        const PmGemm& Gm = S.g[S.op[opi].gemm];
-        const bool gated = Gm.mode == 4;
-        const uint32_t idesc = umma_idesc_bf16(WS_BM, gated ? 128 : NB);
-        for (int u = pm_first_unit(Gm); u < Gm.units && ok; u += G, ++j) {
-          PmUnit d;
-          pm_decode(Gm, u, d);
-          const int buf = j & 1;
-          const uint32_t bph = (uint32_t)(j >> 1) & 1u;
-          if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NB);
-          for (int kb = d.kb0; kb < d.kb1; ++kb, ++it) {
-            const int s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1u;
-            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t wa = base + s * STAGE_BYTES;
-            const uint64_t adesc = umma_desc_sw128(wa);
-            const uint64_t bdesc = umma_desc_sw128(wa + (gated ? 2 * WS_W_BYTES : WS_W_BYTES));
-            const uint32_t acc0 = kb > d.kb0 ? 1u : 0u;
-#pragma unroll
-            for (int kk = 0; kk < WS_BK / 16; ++kk)
-              tc_mma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (acc0 | (kk > 0)) ? 1u : 0u);
-            if (gated) {
-              const uint64_t adesc2 = umma_desc_sw128(wa + WS_W_BYTES);
-#pragma unroll
-              for (int kk = 0; kk < WS_BK / 16; ++kk)
-                tc_mma_bf16(d_tmem + 128u, adesc2 + 2u * kk, bdesc + 2u * kk, idesc, (acc0 | (kk > 0)) ? 1u : 0u);
-            }
-            tc_commit(empty_bar(s));
-          }
-          if (ok) tc_commit(tfull_bar(buf));
-        }
-      }
-    }
+    if (lane == 0) pm_mma_role<NB>(S, base, bar0, tmem_base, STAGES, abort_flag);
   } else {
 #include "moa_phases_workers.inc"
   }

@@ -23,7 +23,7 @@ constexpr int PM_MAX_OPS = 28;
 constexpr int PM_MAX_GEMMS = 10;
 constexpr int PM_MAX_STAGES = 12;
 constexpr int PM_KB = 32;                // keys per attention block
-constexpr int PM_KVST = 4;               // key/value blocks in flight per attention unit
+constexpr int PM_KVST = 2;               // key/value blocks in flight per attention unit
 constexpr int PM_MAXCH = 6;              // 8-element chunks a thread keeps of one row (rows up to 9216 wide)
 constexpr int PM_MERGE_OWN = 24;         // vocabulary slices one thread owns in the LM-head merge
 

@@ -82,3 +82,32 @@ def test_c5_llama70b_batch16_sampled_sequences():
     stats = _given_caches_cycle(p, g, oracles, seqs=[0, 15])
     assert stats["rows"] == 2 * (1 + 5 * 10)
     g.close()
+
+
+def test_c3_lsa_prefill_sampled_tokens():
+    """Config 3: LSA over 8192 tokens x 33 stacked activations x 4096 (32 heads x 128, MHA), the dense-row
+    regime (tensor-core GEMMs with fused epilogues). The oracle computes sampled tokens one by one: the first
+    and last token of the input, of the first pass and of the last pass, and a few in between; every output
+    row is checked to be finite and the appended cache rows against the oracle's for the same tokens."""
+    p = synth.PRESETS["c3"]
+    n_tok = p.lsa_tokens
+    lsa = ("lsa_norm1", "lsa_wq", "lsa_wk", "lsa_wv", "lsa_wo", "lsa_norm2", "lsa_wgate", "lsa_wup", "lsa_wdown",
+           "ca_normkv", "ca_wk", "ca_wv")
+    small = synth.scaled(p, vocab=256)                      # the LSA pass touches neither the embedding nor the LM head
+    w = synth.make_weights(small)
+    g = H.make_gpu(small, w, max_ctx=n_tok, lsa_chunk_tokens=256)
+    exact = H.make_oracle(small, {k: w[k] for k in lsa})
+    h = synth.make_h_stack(p, n_tok)
+    kv = g.moa_lsa_forward(h.cuda(), [n_tok])
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0
+    assert int(g.ca_len[0]) == n_tok
+    assert bool(torch.isfinite(kv.float()).all())
+    tol = H.tol_of(p)
+    for t in [0, 1, 255, 256, 257, 4095, 4096, 7935, 7936, 8190, 8191]:
+        kv_o = exact.lsa_forward(H.np32(h[t][None]))
+        H.assert_rows_close(H.np32(kv[t].cpu())[None], kv_o, tol, f"LSA kv tok {t}")
+        K_o, V_o = exact.ca_kv(kv_o)
+        H.assert_rows_close(H.np32(g.ca_k[0, t].cpu()).reshape(1, -1), K_o.reshape(1, -1), tol, f"CA K tok {t}")
+        H.assert_rows_close(H.np32(g.ca_v[0, t].cpu()).reshape(1, -1), V_o.reshape(1, -1), tol, f"CA V tok {t}")
+    g.close()
