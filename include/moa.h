@@ -100,6 +100,13 @@ typedef struct {
 moa_status moa_create(const moa_config *cfg, const moa_weights *w, moa_ctx **out);
 void moa_destroy(moa_ctx *ctx);
 
+/* Options. MOA_OPT_FUSED_STEP (bf16 only): run moa_draft_step, and moa_lsa_forward passes of any size, as ONE
+ * persistent cooperative kernel (phases separated by grid-wide barriers, weights prefetched across phases,
+ * activations carried as two bf16 terms) instead of a chain of launches. Same results within tolerance, closer
+ * to the fp64 values; off by default because the chain is faster at small row counts. */
+#define MOA_OPT_FUSED_STEP 1
+moa_status moa_set_option(moa_ctx *ctx, int32_t option, int32_t value);
+
 /* Sizes in bytes of moa_state.tree and of the workspace every compute call needs.
  * lsa_chunk_tokens (>= 1) is the number of tokens moa_lsa_forward processes per internal
  * pass; a larger value needs a larger workspace. */

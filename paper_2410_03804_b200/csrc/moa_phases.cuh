@@ -138,13 +138,14 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
             if (want_better == other_better) { val = ov; id = oi; }
           }
         }
+        const size_t at = (size_t)r * Gm.n_sub + sub;
         if (lane < B) {
-          Gm.c_val[((size_t)sub * Gm.R + r) * B + lane] = val;
-          Gm.c_id[((size_t)sub * Gm.R + r) * B + lane] = id;
+          Gm.c_val[at * B + lane] = val;
+          Gm.c_id[at * B + lane] = id;
         }
         if (lane == 0) {
-          Gm.p_max[(size_t)sub * Gm.R + r] = wmax;
-          Gm.p_sum[(size_t)sub * Gm.R + r] = wsum;
+          Gm.p_max[at] = wmax;
+          Gm.p_sum[at] = wsum;
         }
       }
     }

@@ -48,7 +48,7 @@ struct PmGemm {            // (its tensor maps are PmParams.tm[gemm][0..2] weigh
   size_t plane;            // mode 0: elements between split planes
   float* out;              // mode 0: planes; mode 3: fp32 residual stream
   bf16* out16;             // modes 2, 4
-  float *p_max, *p_sum, *c_val;   // mode 1: [n_sub][R], [n_sub][R], [n_sub][R][B]
+  float *p_max, *p_sum, *c_val;   // mode 1: [R][n_sub], [R][n_sub], [R][n_sub][B]
   int* c_id;
 };
 

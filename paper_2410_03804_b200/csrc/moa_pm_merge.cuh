@@ -44,10 +44,10 @@ __device__ __noinline__ void pm_merge(PmSmem& S, const PmOp& op, uint8_t* scratc
       const int s = wt + j * PM_WORKERS;
       hv[j] = -INFINITY; hi[j] = NONE; pm[j] = -INFINITY; ps[j] = 0.f;
       if (s < n_sub) {
-        hv[j] = __ldcg(c_val + ((size_t)s * R + r) * B);
-        hi[j] = __ldcg(c_id + ((size_t)s * R + r) * B);
-        pm[j] = __ldcg(p_max + (size_t)s * R + r);
-        ps[j] = __ldcg(p_sum + (size_t)s * R + r);
+        hv[j] = __ldcg(c_val + ((size_t)r * n_sub + s) * B);
+        hi[j] = __ldcg(c_id + ((size_t)r * n_sub + s) * B);
+        pm[j] = __ldcg(p_max + (size_t)r * n_sub + s);
+        ps[j] = __ldcg(p_sum + (size_t)r * n_sub + s);
       }
     }
 #pragma unroll
@@ -107,8 +107,8 @@ __device__ __noinline__ void pm_merge(PmSmem& S, const PmOp& op, uint8_t* scratc
       const int s = wt + j * PM_WORKERS;
       if (s >= n_sub || hi[j] == NONE || ranks_before(tv, ti, hv[j], hi[j])) continue;
       for (int c = 0; c < B; ++c) {
-        const float v = c == 0 ? hv[j] : __ldcg(c_val + ((size_t)s * R + r) * B + c);
-        const int id = c == 0 ? hi[j] : __ldcg(c_id + ((size_t)s * R + r) * B + c);
+        const float v = c == 0 ? hv[j] : __ldcg(c_val + ((size_t)r * n_sub + s) * B + c);
+        const int id = c == 0 ? hi[j] : __ldcg(c_id + ((size_t)r * n_sub + s) * B + c);
         if (ranks_before(tv, ti, v, id)) break;
         const int at = atomicAdd(n_surv, 1);
         if (at < 256) { s_val[at] = v; s_id[at] = id; }

@@ -46,10 +46,10 @@ struct WsParams {
   float* out;              // mode 0: plane `split` starts at out + split * plane; row r, column c at [r * ldo + c]
   size_t plane;            // mode 0: elements between two partial planes
   int B;                   // mode 1
-  float* p_max;            // mode 1: [4*tiles][R]
-  float* p_sum;            //         [4*tiles][R]
-  float* c_val;            //         [4*tiles][R][B]
-  int* c_id;               //         [4*tiles][R][B]
+  float* p_max;            // mode 1: [R][4*tiles]
+  float* p_sum;            //         [R][4*tiles]
+  float* c_val;            //         [R][4*tiles][B]
+  int* c_id;               //         [R][4*tiles][B]
   int* status;             // device status word (may be nullptr)
 };
 
@@ -309,6 +309,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
         }
       } else {
         const int sub = tile * 4 + q;                         // 32-row vocabulary slice
+        const int n_sub = 4 * P.tiles_total;
         const int B = P.B;
 #pragma unroll 1
         for (int c0 = 0; c0 < NPAD; c0 += 16) {
@@ -338,13 +339,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
                 if (want_better == other_better) { val = ov; id = oi; }
               }
             }
+            const size_t at = (size_t)r * n_sub + sub;       // row-major over slices: the merge reads them coalesced
             if (lane < B) {
-              P.c_val[((size_t)sub * P.R + r) * B + lane] = val;
-              P.c_id[((size_t)sub * P.R + r) * B + lane] = id;
+              P.c_val[at * B + lane] = val;
+              P.c_id[at * B + lane] = id;
             }
             if (lane == 0) {
-              P.p_max[(size_t)sub * P.R + r] = wmax;
-              P.p_sum[(size_t)sub * P.R + r] = wsum;
+              P.p_max[at] = wmax;
+              P.p_sum[at] = wsum;
             }
           }
         }
@@ -366,16 +368,19 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 
 // ---------------------------------------------------------------------------------------------
 // LM-head merge: one block per activation row combines the per-slice partials into logsumexp and
-// the global top-B, ordered by (log-probability descending, id ascending).
-//   1. logsumexp from the slices' (max, sum exp).
-//   2. threshold = the B-th best of the slice heads (each slice list is sorted, so its head is its
-//      best): B rounds of "best element ranking strictly after the previous pick", per warp and then
-//      over the 32 warp lists.
-//   3. survivors = candidates ranking at or before the threshold; only slices whose head does can
-//      contribute, so there are at most B*B of them. They are ranked by counting.
+// the global top-B, ordered by (log-probability descending, id ascending). Built for few dependent
+// memory round trips (the kernel is latency-bound):
+//   1. every thread loads (max, sum exp, best value, best id) of the <= MERGE_OWN slices it owns, coalesced;
+//   2. logsumexp from the (max, sum exp) pairs;
+//   3. threshold = the B-th best slice head (each slice list is sorted, so its head is its best): B rounds
+//      of "best ranking strictly after the previous pick", per warp over registers, then over the warp lists;
+//   4. only slices whose head ranks at or before the threshold can contribute (at most B of them): their
+//      owners load the whole B-entry list at once and keep what passes the threshold (at most B*B survivors);
+//   5. the survivors are ranked by counting.
 // ---------------------------------------------------------------------------------------------
 constexpr int MERGE_THREADS = 1024;
 constexpr int MERGE_MAXB = 16;
+constexpr int MERGE_OWN = 8;          // slices per thread: up to 8192 slices = 262144 vocabulary rows
 
 __device__ __forceinline__ void warp_best(float& bv, int& bi) {
 #pragma unroll
@@ -402,54 +407,59 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   const int r = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int NONE = 0x7fffffff;
+  const size_t row = (size_t)r * n_sub;
   if (tid == 0) n_surv = 0;
   if (tid < B) { ids[(size_t)r * B + tid] = -1; logp[(size_t)r * B + tid] = -INFINITY; }
-  // 1. logsumexp over all slices
+  // 1. this thread's slices
+  float hv[MERGE_OWN], pm[MERGE_OWN], ps[MERGE_OWN];
+  int hi[MERGE_OWN];
+#pragma unroll
+  for (int j = 0; j < MERGE_OWN; ++j) {
+    const int s = tid + j * MERGE_THREADS;
+    const bool in = s < n_sub;
+    pm[j] = in ? p_max[row + s] : -INFINITY;
+    ps[j] = in ? p_sum[row + s] : 0.f;
+    hv[j] = in ? c_val[(row + s) * B] : -INFINITY;
+    hi[j] = in ? c_id[(row + s) * B] : NONE;
+  }
+  // 2. logsumexp
   float m = -INFINITY;
-  for (int s = tid; s < n_sub; s += MERGE_THREADS) m = fmaxf(m, p_max[(size_t)s * R + r]);
+#pragma unroll
+  for (int j = 0; j < MERGE_OWN; ++j) m = fmaxf(m, pm[j]);
   m = block_max(m, red);
   float se = 0.f;
-  for (int s = tid; s < n_sub; s += MERGE_THREADS) {
-    const float pm = p_max[(size_t)s * R + r];
-    if (pm > -INFINITY) se += p_sum[(size_t)s * R + r] * __expf(pm - m);
-  }
+#pragma unroll
+  for (int j = 0; j < MERGE_OWN; ++j)
+    if (pm[j] > -INFINITY) se += ps[j] * __expf(pm[j] - m);
   se = block_sum(se, red);
   const float lse = m + logf(se);
-  // 2a. per warp: the B best slice heads among this warp's slices
+  // 3a. per warp: the B best heads among this warp's slices
   float pv = INFINITY;
   int pi = -1;
   for (int round = 0; round < B; ++round) {
     float bv = -INFINITY;
     int bi = NONE;
-    for (int s = tid; s < n_sub; s += MERGE_THREADS) {
-      const float v = c_val[((size_t)s * R + r) * B];
-      const int id = c_id[((size_t)s * R + r) * B];
-      if (ranks_before(pv, pi, v, id) && ranks_before(v, id, bv, bi)) { bv = v; bi = id; }
-    }
+#pragma unroll
+    for (int j = 0; j < MERGE_OWN; ++j)
+      if (ranks_before(pv, pi, hv[j], hi[j]) && ranks_before(hv[j], hi[j], bv, bi)) { bv = hv[j]; bi = hi[j]; }
     warp_best(bv, bi);
     pv = bv;
     pi = bi;
     if (lane == 0) { w_val[wid][round] = bv; w_id[wid][round] = bi; }
-    if (bi == NONE) {                       // this warp has run out of heads
-      for (int k = round + 1; k < B; ++k)
-        if (lane == 0) { w_val[wid][k] = -INFINITY; w_id[wid][k] = NONE; }
-      break;
-    }
   }
   __syncthreads();
-  // 2b. warp 0: the B-th best over the 32 sorted warp lists
+  // 3b. warp 0: the B-th best over the 32 sorted warp lists
   if (wid == 0) {
     float qv = INFINITY;
     int qi = -1;
+    int cur = 0;                                  // this lane's list is sorted: a cursor is enough
     for (int round = 0; round < B; ++round) {
-      float bv = -INFINITY;
-      int bi = NONE;
-      for (int k = 0; k < B; ++k) {
-        const float v = w_val[lane][k];
-        const int id = w_id[lane][k];
-        if (ranks_before(qv, qi, v, id)) { bv = v; bi = id; break; }   // sorted: first one after the last pick
-      }
+      float bv = cur < B ? w_val[lane][cur] : -INFINITY;
+      int bi = cur < B ? w_id[lane][cur] : NONE;
+      const float mv = bv;
+      const int mi = bi;
       warp_best(bv, bi);
+      if (mv == bv && mi == bi && bi != NONE) ++cur;   // this lane's head was taken
       qv = bv;
       qi = bi;
     }
@@ -458,26 +468,34 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   __syncthreads();
   const float tv = t_val;
   const int ti = t_id;
-  // 3. survivors
-  for (int s = tid; s < n_sub; s += MERGE_THREADS) {
-    const float* cv = c_val + ((size_t)s * R + r) * B;
-    const int* ci = c_id + ((size_t)s * R + r) * B;
-    for (int c = 0; c < B; ++c) {
-      const float v = cv[c];
-      const int id = ci[c];
-      if (ranks_before(tv, ti, v, id)) break;          // strictly after the threshold: so is the rest
+  // 4. survivors: whole lists of the slices whose head passes, loaded at once
+#pragma unroll
+  for (int j = 0; j < MERGE_OWN; ++j) {
+    const int s = tid + j * MERGE_THREADS;
+    if (s >= n_sub || hi[j] == NONE || ranks_before(tv, ti, hv[j], hi[j])) continue;
+    float lv[MERGE_MAXB];
+    int li[MERGE_MAXB];
+#pragma unroll
+    for (int c = 0; c < MERGE_MAXB; ++c) {
+      lv[c] = c < B ? c_val[(row + s) * B + c] : -INFINITY;
+      li[c] = c < B ? c_id[(row + s) * B + c] : NONE;
+    }
+#pragma unroll
+    for (int c = 0; c < MERGE_MAXB; ++c) {
+      if (c >= B || li[c] == NONE || ranks_before(tv, ti, lv[c], li[c])) continue;
       const int at = atomicAdd(&n_surv, 1);
-      if (at < MERGE_MAXB * MERGE_MAXB) { s_val[at] = v; s_id[at] = id; }
+      if (at < MERGE_MAXB * MERGE_MAXB) { s_val[at] = lv[c]; s_id[at] = li[c]; }
     }
   }
   __syncthreads();
+  // 5. rank by counting
   const int ns = n_surv < MERGE_MAXB * MERGE_MAXB ? n_surv : MERGE_MAXB * MERGE_MAXB;
   if (tid < ns) {
     const float v = s_val[tid];
     const int id = s_id[tid];
     int rank = 0;
     for (int j = 0; j < ns; ++j) rank += ranks_before(s_val[j], s_id[j], v, id) ? 1 : 0;
-    if (rank < B && id != NONE) {
+    if (rank < B) {
       ids[(size_t)r * B + rank] = id;
       logp[(size_t)r * B + rank] = v - lse;
     }

@@ -19,7 +19,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
                 "ERR_STATE", "ERR_ARCH", "ERR_CUDA", "ERR_TIMEOUT"]
 MOA_OK = 0
 
-EXPORTS = ["moa_create", "moa_destroy", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
+EXPORTS = ["moa_create", "moa_destroy", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
@@ -79,6 +79,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_create.argtypes = [C.POINTER(MoaConfig), C.POINTER(MoaWeights), C.POINTER(vp)]
     lib.moa_destroy.argtypes = [vp]
     lib.moa_destroy.restype = None
+    lib.moa_set_option.argtypes = [vp, i32, i32]
     lib.moa_state_bytes.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.moa_status_str.argtypes = [i32]
     lib.moa_status_str.restype = C.c_char_p
@@ -146,7 +147,8 @@ class MoA:
     weights: dict name -> CUDA tensor (dtype float32 or bfloat16, as cfg['dtype'] says).
     cfg keys: the fields of moa_config except dtype/max_* (given separately)."""
 
-    def __init__(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int, lsa_chunk_tokens: int = 8):
+    def __init__(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int, lsa_chunk_tokens: int = 8,
+                 fused_step: bool = False):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2410_03804_b200 needs a CUDA device (B200, sm_100a); there is no CPU path")
@@ -171,6 +173,8 @@ class MoA:
         h = C.c_void_p()
         _check(self.lib.moa_create(C.byref(c), C.byref(w), C.byref(h)), "moa_create")
         self.h = h
+        if fused_step:
+            _check(self.lib.moa_set_option(self.h, 1, 1), "moa_set_option")
         self.device = weights["embed"].device
         tb, wb = C.c_size_t(), C.c_size_t()
         _check(self.lib.moa_state_bytes(self.h, int(lsa_chunk_tokens), C.byref(tb), C.byref(wb)), "moa_state_bytes")

@@ -40,10 +40,11 @@ def make_oracles(p: synth.Preset, weights_cpu: dict, cache_f64=True):
     return exact, dec
 
 
-def make_gpu(p: synth.Preset, weights_cpu: dict, max_ctx: int, lsa_chunk_tokens: int = 8, max_batch=None):
+def make_gpu(p: synth.Preset, weights_cpu: dict, max_ctx: int, lsa_chunk_tokens: int = 8, max_batch=None,
+             fused_step: bool = False):
     from paper_2410_03804_b200 import moa
     w = {k: v.cuda() for k, v in weights_cpu.items()}
-    return moa.MoA(cfg_of(p), w, max_batch or p.batch, max_ctx, lsa_chunk_tokens)
+    return moa.MoA(cfg_of(p), w, max_batch or p.batch, max_ctx, lsa_chunk_tokens, fused_step=fused_step)
 
 
 def assert_rows_close(got, want, tol, what=""):

@@ -62,6 +62,16 @@ def test_c2_llama8b_full_cycle(llama8b):
     assert stats["rows"] == 1 + 5 * 10
 
 
+def test_c2_llama8b_fused_single_kernel_forward():
+    """Config 2 again with every forward as one persistent kernel (MOA_OPT_FUSED_STEP): same checks."""
+    p = synth.PRESETS["c2"]
+    w = synth.make_weights(p)
+    g = H.make_gpu(p, w, max_ctx=p.ctx + 64, lsa_chunk_tokens=p.lsa_tokens, fused_step=True)
+    stats = _given_caches_cycle(p, g, H.make_oracles(p, w))
+    assert stats["rows"] == 1 + 5 * 10
+    g.close()
+
+
 def test_c4_long_context_32k(llama8b):
     """Config 4: config 2's drafter over 32768-entry caches (both attentions), every row checked."""
     p2, w, g, oracles = llama8b

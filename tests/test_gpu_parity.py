@@ -156,15 +156,16 @@ def test_c1_free_running_tree_matches_oracle():
     assert np.array_equal(mask[0], O.tree_mask(opar))
 
 
-@pytest.mark.parametrize("dtype,batch", [("bf16", 1), ("bf16", 3), ("f32", 2)])
-def test_reduced_llama_shape(dtype, batch):
+@pytest.mark.parametrize("dtype,batch,fused", [("bf16", 1, False), ("bf16", 3, False), ("f32", 2, False),
+                                               ("bf16", 1, True), ("bf16", 3, True)])
+def test_reduced_llama_shape(dtype, batch, fused):
     """A reduced Llama-3-shaped drafter: GQA 8/2 x 128, ragged vocab, several sequences,
     stacked activations with the std ramp and outlier channels of config 2."""
     p = synth.scaled(synth.PRESETS["c2"], d_model=512, n_stack=5, d_stack=384, vocab=5003, lsa_hq=8, lsa_hkv=2,
                      lsa_mlp=768, sa_hq=8, sa_hkv=2, sa_mlp=64, ca_hq=8, ca_hkv=4, ca_mlp=896, ctx=37, batch=batch,
                      tree_topk=5, tree_depth=3, tree_keep=12, dtype=dtype, lsa_tokens=37)
     w = synth.make_weights(p)
-    g = H.make_gpu(p, w, max_ctx=64, lsa_chunk_tokens=16)
+    g = H.make_gpu(p, w, max_ctx=64, lsa_chunk_tokens=16, fused_step=fused)     # fused: one persistent kernel per forward
     stats = run_cycle(p, g, H.make_oracles(p, w), synth.make_h_stack(p, p.lsa_tokens * batch),
                       synth.make_tokens(p, p.ctx), synth.make_root(p))
     assert stats["rows"] == batch * (1 + 2 * 5)
