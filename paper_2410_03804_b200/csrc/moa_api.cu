@@ -139,6 +139,25 @@ static int chunk_from_bytes(const moa_config& c, size_t elt, size_t ws_bytes) {
 static inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 static inline unsigned blocks_for(size_t total, int threads) { return (unsigned)((total + threads - 1) / threads); }
 
+// Launch with programmatic dependent launch allowed: the kernel may start while its predecessor in the stream is
+// still running and does its independent set-up (and, for the weight-streaming GEMM, its first weight loads)
+// until its griddepcontrol.wait; see pdl_trigger / pdl_wait in moa_common.cuh.
+template <typename... KArgs, typename... Args>
+static void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);     // errors surface through cudaGetLastError()
+}
+
 // 2-D bf16 tensor map: global [rows, k] row-major, box 64 x box_rows, 128-byte swizzle, zero fill outside.
 static bool encode_map(const moa_ctx* ctx, CUtensorMap* tm, const void* ptr, int rows, int k, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
@@ -191,7 +210,7 @@ static moa_status launch_ws(cudaStream_t s, const WsParams& P, int grid) {
     }
     attr_set = true;
   }
-  wstream_gemm_kernel<NPAD><<<grid, WS_THREADS, ws_smem_bytes(NPAD), s>>>(P);
+  launch_pdl(wstream_gemm_kernel<NPAD>, dim3(grid), dim3(WS_THREADS), ws_smem_bytes(NPAD), s, P);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -264,7 +283,7 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
   int col = 0;
   for (int i = 0; i < nseg; ++i) {
     dim3 grid((N[i] + 63) / 64, (R + 63) / 64);
-    gemm_fma_kernel<T><<<grid, 256, 0, s>>>(X, (const T*)W[i], R, N[i], K, nullptr, 0, part + col, ntot);
+    launch_pdl(gemm_fma_kernel<T>, dim3(grid), dim3(256), 0, s, X, (const T*)W[i], R, N[i], K, nullptr, 0, part + col, ntot);
     MOA_CHECK_LAUNCH();
     col += N[i];
   }
@@ -285,10 +304,10 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
     attr_set = true;
   }
   dim3 grid(P.n_parts, P.hkv * P.q_tiles, nseq);
-  attn_split_kernel<DH, QSPLIT><<<grid, nwarps * 32, smem, s>>>(P);
+  launch_pdl(attn_split_kernel<DH, QSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
-    attn_combine_kernel<DH><<<nseq * P.rows_per_seq * P.hq, DH, 0, s>>>(P.part_o, P.part_ml, P.n_parts, P.out);
+    launch_pdl(attn_combine_kernel<DH>, dim3(nseq * P.rows_per_seq * P.hq), dim3(DH), 0, s, P.part_o, P.part_ml, P.n_parts, P.out);
     MOA_CHECK_LAUNCH();
   }
   return MOA_OK;
@@ -333,10 +352,10 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   }
   dim3 grid(R, hq);
   if (dh == 128)
-    attn_rows_kernel<T, 128><<<grid, 128, 0, s>>>(q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
+    launch_pdl(attn_rows_kernel<T, 128>, dim3(grid), dim3(128), 0, s, q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
                                                   slotsB, slots_ld, nB, rows_per_seq, out);
   else
-    attn_rows_kernel<T, 64><<<grid, 128, 0, s>>>(q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
+    launch_pdl(attn_rows_kernel<T, 64>, dim3(grid), dim3(128), 0, s, q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
                                                  slotsB, slots_ld, nB, rows_per_seq, out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
@@ -348,13 +367,13 @@ static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, co
                                 const LinOut* lo, const void* gain, void* hidden_out) {
   if (R <= 0) return MOA_OK;
   if (K % RN_CLUSTER == 0 && K / RN_CLUSTER <= 256 * RN_MAX_PER_THREAD) {
-    residual_norm_cluster_kernel<T><<<dim3(RN_CLUSTER, R), 256, 0, s>>>(
+    launch_pdl(residual_norm_cluster_kernel<T>, dim3(dim3(RN_CLUSTER, R)), dim3(256), 0, s, 
         (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0, lo ? lo->plane : 0, K, (const T*)gain,
         ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out);
     MOA_CHECK_LAUNCH();
     return MOA_OK;
   }
-  residual_norm_kernel<T><<<R, 256, 0, s>>>((float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0,
+  launch_pdl(residual_norm_kernel<T>, dim3(R), dim3(256), 0, s, (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0,
                                             lo ? lo->plane : 0, K, (const T*)gain, ctx->c.rms_eps, (T*)(ws + p.xn),
                                             (T*)hidden_out);
   MOA_CHECK_LAUNCH();
@@ -373,7 +392,7 @@ static moa_status mlp_block(cudaStream_t s, moa_ctx* ctx, const Workspace& p, ch
   MOA_TRY(linear<T>(ctx, s, xn, R, K, 2, W2, N2, ws, p, lo, status_word));
   const size_t total = (size_t)R * F;
   if (total) {
-    silu_mul_split_kernel<T><<<blocks_for(total, 256), 256, 0, s>>>(lo->part, lo->splits, lo->plane, F, h, total);
+    launch_pdl(silu_mul_split_kernel<T>, dim3(blocks_for(total, 256)), dim3(256), 0, s, lo->part, lo->splits, lo->plane, F, h, total);
     MOA_CHECK_LAUNCH();
   }
   const void* W1[1] = {wdown};
@@ -405,14 +424,14 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     const int R = nt * S;
     const T* x = (const T*)h_stack + (size_t)t0 * S * D;
     // pre-norm and q, k, v projections of every (token, layer) row: rows of [q | k | v]
-    rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>(x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn);
+    launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn);
     MOA_CHECK_LAUNCH();
     const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
     const int N3[3] = {nq, nkv, nkv};
     MOA_TRY(linear<T>(ctx, s, xn, R, D, 3, W3, N3, ws, p, &lo, status_word));
     {
       const size_t tot = (size_t)R * ld;
-      sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
+      launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
       MOA_CHECK_LAUNCH();
     }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
@@ -427,16 +446,16 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, D, &lo, nullptr, nullptr));
     // mean over layers
     T* kvo = kv_out ? (T*)kv_out + (size_t)t0 * D : nullptr;
-    mean_layers_kernel<T><<<dim3(nt, (D + 255) / 256), 256, 0, s>>>(xres, S, D, kvf, kvo);
+    launch_pdl(mean_layers_kernel<T>, dim3(dim3(nt, (D + 255) / 256)), dim3(256), 0, s, xres, S, D, kvf, kvo);
     MOA_CHECK_LAUNCH();
     // cross-attention keys / values of the new positions, appended to the cache
-    rmsnorm_rows_kernel<float, T><<<nt, 256, 0, s>>>(kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn);
+    launch_pdl(rmsnorm_rows_kernel<float, T>, dim3(nt), dim3(256), 0, s, kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn);
     MOA_CHECK_LAUNCH();
     const int ckv = c.ca_hkv * dh;
     const void* W2[2] = {w.ca_wk, w.ca_wv};
     const int N2[2] = {ckv, ckv};
     MOA_TRY(linear<T>(ctx, s, kvn, nt, D, 2, W2, N2, ws, p, &lo, status_word));
-    cache_append_kernel<T><<<nt, 256, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * ckv, 0, ckv, ckv, st->ca_len, c.max_ctx,
+    launch_pdl(cache_append_kernel<T>, dim3(nt), dim3(256), 0, s, lo.part, lo.splits, lo.plane, 2 * ckv, 0, ckv, ckv, st->ca_len, c.max_ctx,
                                               split, t0, (T*)st->ca_k, (T*)st->ca_v);
     MOA_CHECK_LAUNCH();
   }
@@ -457,7 +476,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
   LinOut lo;
   for (int t0 = 0; t0 < total; t0 += p.rows_cap) {
     const int R = (total - t0) < p.rows_cap ? (total - t0) : p.rows_cap;
-    rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>((const T*)w.embed, tok + t0, c.vocab, (const T*)w.sa_norm1, E,
+    launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, tok + t0, c.vocab, (const T*)w.sa_norm1, E,
                                                 c.rms_eps, nullptr, xn);
     MOA_CHECK_LAUNCH();
     const void* W2[2] = {w.sa_wk, w.sa_wv};
@@ -469,7 +488,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
     rr.max_ctx = c.max_ctx;
     rr.split = split;
     rr.row0 = t0;
-    rope_store_kernel<T><<<dim3(R, 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
+    launch_pdl(rope_store_kernel<T>, dim3(dim3(R, 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
                                            c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (float*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
     MOA_CHECK_LAUNCH();
   }
@@ -511,7 +530,7 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
     MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count)));
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
-    lm_merge_kernel<<<R, MERGE_THREADS, 0, s>>>(P.p_max, P.p_sum, P.c_val, P.c_id, 4 * P.tiles_total, R, B, topk_id,
+    launch_pdl(lm_merge_kernel, dim3(R), dim3(MERGE_THREADS), 0, s, P.p_max, P.p_sum, P.c_val, P.c_id, 4 * P.tiles_total, R, B, topk_id,
                                                 topk_logp);
     MOA_CHECK_LAUNCH();
     return MOA_OK;
@@ -520,11 +539,11 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
   {
     dim3 grid((V + 63) / 64, (R + 63) / 64);
-    gemm_fma_kernel<T><<<grid, 256, 0, s>>>(xn, (const T*)ctx->w.lm_head, R, V, E, nullptr, 0, logits, V);
+    launch_pdl(gemm_fma_kernel<T>, dim3(grid), dim3(256), 0, s, xn, (const T*)ctx->w.lm_head, R, V, E, nullptr, 0, logits, V);
     MOA_CHECK_LAUNCH();
   }
   if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
-  lse_topk_rows_kernel<<<R, 256, 0, s>>>(logits, V, B, topk_id, topk_logp);
+  launch_pdl(lse_topk_rows_kernel, dim3(R), dim3(256), 0, s, logits, V, B, topk_id, topk_logp);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -556,7 +575,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   LinOut lo;
 
   // ---- self-attention block ----
-  rmsnorm_rows_kernel<T, T><<<R, 256, 0, s>>>((const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn);
+  launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn);
   MOA_CHECK_LAUNCH();
   const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh;
   {
@@ -570,7 +589,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   rr.step = step;
   rr.B = B;
   rr.slots = L.NS;
-  rope_store_kernel<T><<<dim3(R, c.sa_hq + 2 * c.sa_hkv), 64, 0, s>>>(lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
+  launch_pdl(rope_store_kernel<T>, dim3(dim3(R, c.sa_hq + 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
                                          dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, tk, tv);
   MOA_CHECK_LAUNCH();
   int max_sa = 0, max_ca = 0;
@@ -597,8 +616,8 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     const int N1[1] = {cq};
     MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
     const size_t tot = (size_t)R * cq;
-    if (q32) sum_cast_kernel<float><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, q32);
-    else sum_cast_kernel<T><<<blocks_for(tot, 256), 256, 0, s>>>(lo.part, lo.splits, lo.plane, tot, narrow);
+    if (q32) launch_pdl(sum_cast_kernel<float>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, q32);
+    else launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
     MOA_CHECK_LAUNCH();
   }
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,

@@ -75,6 +75,8 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 // with outlier channels) from amplifying the rounding of q.
 template <int DH, bool QSPLIT>
 __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int KS = DH / 16;                // k-steps of the Q.K^T product
   constexpr int TILE_BYTES = AT_KB * DH * 2;
@@ -313,6 +315,8 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
 template <int DH>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_parts,
                                     bf16* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const size_t rh = blockIdx.x;
   const int d = threadIdx.x;
   float M = -INFINITY;

@@ -15,6 +15,8 @@ template <typename TIN, typename T>
 __global__ void rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok, int vocab,
                                     const T* __restrict__ gain, int K, float eps,
                                     float* __restrict__ res_out, T* __restrict__ y) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[33];
   const int r = blockIdx.x;
   const TIN* xr;
@@ -48,6 +50,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) gemm_fma_kernel(const T* __restrict__ A, const T* __restrict__ W,
                                                        int R, int N, int K, const float* res, int ldr,
                                                        float* C, int ldc) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float As[16][64 + 4];
   __shared__ float Ws[16][64 + 4];
   const int tid = threadIdx.x;
@@ -116,6 +120,8 @@ template <typename T>
 __global__ void residual_norm_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
                                      int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
                                      T* __restrict__ hidden_out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[33];
   const int r = blockIdx.x;
   float ss = 0.f;
@@ -146,6 +152,8 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
     residual_norm_cluster_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
                                  int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
                                  T* __restrict__ hidden_out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[33];
   __shared__ float cta_ss;
   const int r = blockIdx.y;
@@ -201,6 +209,8 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
 template <typename T>
 __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
                                       T* __restrict__ h, size_t total) {
+  pdl_trigger();
+  pdl_wait();
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const size_t r = i / F;
@@ -214,6 +224,8 @@ __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits
 template <typename T>
 __global__ void sum_cast_kernel(const float* __restrict__ part, int splits, size_t plane, size_t total,
                                 T* __restrict__ y) {
+  pdl_trigger();
+  pdl_wait();
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < total) y[i] = from_f<T>(sum_splits(part + i, plane, splits));
 }
@@ -242,6 +254,8 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
                                   int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
                                   RopeRows rr, T* __restrict__ qdst, float* __restrict__ qdst32, T* __restrict__ kdst,
                                   T* __restrict__ vdst) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float cs[64], sn[64];
   const int r = blockIdx.x;
   int seq, pos_add;
@@ -313,6 +327,8 @@ __global__ void cache_append_kernel(const float* __restrict__ kv, int splits, si
                                     int width,
                                     const int* __restrict__ len, int max_ctx, SeqSplit split, int row0,
                                     T* __restrict__ kdst, T* __restrict__ vdst) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x;
   const int t = row0 + r;
   const int seq = split.seq_of(t);
@@ -356,6 +372,8 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
                                                         const T* __restrict__ kB, const T* __restrict__ vB, int capB,
                                                         const int* __restrict__ slotsB, int slots_ld, int nB,
                                                         int rows_per_seq, T* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int VEC = DH / 32;
   __shared__ float s_m[4], s_l[4], s_acc[4][DH];
   const int r = blockIdx.x, h = blockIdx.y;
@@ -421,6 +439,8 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
 template <typename T>
 __global__ void mean_layers_kernel(const float* __restrict__ Z, int S, int D, float* __restrict__ kvf,
                                    T* __restrict__ kv_out) {
+  pdl_trigger();
+  pdl_wait();
   const int t = blockIdx.x;                                   // grid (tokens, ceil(D / blockDim.x))
   const int c = blockIdx.y * blockDim.x + threadIdx.x;
   if (c >= D) return;
@@ -441,6 +461,8 @@ __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {   /
 
 __global__ void __launch_bounds__(256) lse_topk_rows_kernel(const float* __restrict__ z, int V, int B,
                                                             int* __restrict__ ids, float* __restrict__ logp) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[33];
   __shared__ float s_v[8];
   __shared__ int s_i[8];

@@ -16,6 +16,13 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// Programmatic dependent launch. A kernel launched with that attribute may begin while the kernel before it in
+// the stream still runs. pdl_trigger() lets the NEXT kernel begin; pdl_wait() blocks until the PREVIOUS kernel has
+// completed and its writes are visible. Every kernel of a chain calls pdl_wait() before it reads or overwrites
+// anything another kernel of the chain touches (so completion stays transitive); both are no-ops otherwise.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int units = P.tiles_total * P.splits;
+  pdl_trigger();       // the next kernel of the chain may start its own set-up
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -220,6 +221,27 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
+      // Weights depend on nothing: the tiles of the first ring pass go out at once. The activations were
+      // written by the kernel before this one, so their tiles wait for it (programmatic dependent launch).
+      uint32_t pre = 0;
+      for (int u = blockIdx.x; u < units && pre < (uint32_t)STAGES; u += gridDim.x) {
+        int seg, n0, kb0, kb1, split, tile;
+        decode(u, seg, n0, kb0, kb1, split, tile);
+        for (int kb = kb0; kb < kb1 && pre < (uint32_t)STAGES; ++kb, ++pre) {
+          mbar_expect_tx(full_bar(pre), STAGE_BYTES);
+          tma_load_2d(base + pre * STAGE_BYTES, &P.tmW[seg], kb * WS_BK, n0, full_bar(pre));
+        }
+      }
+      pdl_wait();
+      {
+        uint32_t i2 = 0;
+        for (int u = blockIdx.x; u < units && i2 < pre; u += gridDim.x) {
+          int seg, n0, kb0, kb1, split, tile;
+          decode(u, seg, n0, kb0, kb1, split, tile);
+          for (int kb = kb0; kb < kb1 && i2 < pre; ++kb, ++i2)
+            tma_load_2d(base + i2 * STAGE_BYTES + WS_W_BYTES, &P.tmX, kb * WS_BK, 0, full_bar(i2));
+        }
+      }
       uint32_t it = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
@@ -227,6 +249,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
         decode(u, seg, n0, kb0, kb1, split, tile);
         const CUtensorMap* tw = &P.tmW[seg];
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
+          if (it < pre) continue;               // went out above
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -396,6 +419,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
                                                                  const float* __restrict__ c_val,
                                                                  const int* __restrict__ c_id, int n_sub, int R, int B,
                                                                  int* __restrict__ ids, float* __restrict__ logp) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[33];
   __shared__ float w_val[32][MERGE_MAXB];
   __shared__ int w_id[32][MERGE_MAXB];
