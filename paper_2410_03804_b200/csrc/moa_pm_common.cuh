@@ -107,74 +107,6 @@ __device__ __forceinline__ float worker_sum(float v, float* red, int wt) {
   return t;
 }
 
-__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
-
-// 8 consecutive fp32 values: sum of `splits` planes (plane elements apart), read past L1. The loads of four
-// planes are issued before any of them is used, so a row costs one memory round trip per four planes.
-__device__ __forceinline__ void load8_planes(const float* p, int splits, size_t plane, float* v) {
-#pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = 0.f;
-  int s = 0;
-  for (; s + 4 <= splits; s += 4) {
-    float4 a[4], b[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) { a[u] = ldcg4(p + (size_t)(s + u) * plane); b[u] = ldcg4(p + (size_t)(s + u) * plane + 4); }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      v[0] += a[u].x; v[1] += a[u].y; v[2] += a[u].z; v[3] += a[u].w;
-      v[4] += b[u].x; v[5] += b[u].y; v[6] += b[u].z; v[7] += b[u].w;
-    }
-  }
-  float4 a[3], b[3];
-#pragma unroll
-  for (int u = 0; u < 3; ++u)
-    if (s + u < splits) { a[u] = ldcg4(p + (size_t)(s + u) * plane); b[u] = ldcg4(p + (size_t)(s + u) * plane + 4); }
-#pragma unroll
-  for (int u = 0; u < 3; ++u)
-    if (s + u < splits) {
-      v[0] += a[u].x; v[1] += a[u].y; v[2] += a[u].z; v[3] += a[u].w;
-      v[4] += b[u].x; v[5] += b[u].y; v[6] += b[u].z; v[7] += b[u].w;
-    }
-}
-
-// One fp32 value as the sum of its split planes, loads issued four at a time.
-__device__ __forceinline__ float load1_planes(const float* p, int splits, size_t plane) {
-  float acc = 0.f;
-  int s = 0;
-  for (; s + 4 <= splits; s += 4) {
-    const float a = __ldcg(p + (size_t)s * plane), b = __ldcg(p + (size_t)(s + 1) * plane);
-    const float c = __ldcg(p + (size_t)(s + 2) * plane), d = __ldcg(p + (size_t)(s + 3) * plane);
-    acc += a; acc += b; acc += c; acc += d;
-  }
-  float t[3] = {0.f, 0.f, 0.f};
-#pragma unroll
-  for (int u = 0; u < 3; ++u)
-    if (s + u < splits) t[u] = __ldcg(p + (size_t)(s + u) * plane);
-  return acc + t[0] + t[1] + t[2];
-}
-
-__device__ __forceinline__ void bf16x8_to_float(const uint4 u, float* v) {
-  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
-}
-
-// Stores 8 values into an X buffer row as bf16: hi at row r, and (lo_rows > 0) the remainder at row lo_rows + r.
-__device__ __forceinline__ void xbuf_store8(bf16* xb, size_t K, int r, int k, int lo_rows, const float* v) {
-  uint32_t hi[4], lo[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const bf16 h0 = __float2bfloat16_rn(v[2 * e]), h1 = __float2bfloat16_rn(v[2 * e + 1]);
-    hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-    lo[e] = pack_bf16(v[2 * e] - __bfloat162float(h0), v[2 * e + 1] - __bfloat162float(h1));
-  }
-  *reinterpret_cast<uint4*>(xb + (size_t)r * K + k) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-  if (lo_rows > 0) *reinterpret_cast<uint4*>(xb + (size_t)(lo_rows + r) * K + k) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-}
-
 // ---------------------------------------------------------------------------------------------
 // static schedule of the GEMM phases as seen by one CTA (same arithmetic in the three roles)
 // ---------------------------------------------------------------------------------------------
