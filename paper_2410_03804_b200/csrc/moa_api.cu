@@ -366,7 +366,7 @@ template <typename T>
 static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, const Workspace& p, int R, int K,
                                 const LinOut* lo, const void* gain, void* hidden_out) {
   if (R <= 0) return MOA_OK;
-  if (K % RN_CLUSTER == 0 && K / RN_CLUSTER <= 256 * RN_MAX_PER_THREAD) {
+  if (K % (RN_CLUSTER * 8) == 0 && K / RN_CLUSTER <= 256 * 8 * (RN_MAX_PER_THREAD / 4)) {
     launch_pdl(residual_norm_cluster_kernel<T>, dim3(dim3(RN_CLUSTER, R)), dim3(256), 0, s, 
         (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0, lo ? lo->plane : 0, K, (const T*)gain,
         ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out);
@@ -392,7 +392,7 @@ static moa_status mlp_block(cudaStream_t s, moa_ctx* ctx, const Workspace& p, ch
   MOA_TRY(linear<T>(ctx, s, xn, R, K, 2, W2, N2, ws, p, lo, status_word));
   const size_t total = (size_t)R * F;
   if (total) {
-    launch_pdl(silu_mul_split_kernel<T>, dim3(blocks_for(total, 256)), dim3(256), 0, s, lo->part, lo->splits, lo->plane, F, h, total);
+    launch_pdl(silu_mul_split_kernel<T>, dim3(blocks_for(total / 8, 256)), dim3(256), 0, s, lo->part, lo->splits, lo->plane, F, h, total);
     MOA_CHECK_LAUNCH();
   }
   const void* W1[1] = {wdown};
@@ -431,7 +431,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     MOA_TRY(linear<T>(ctx, s, xn, R, D, 3, W3, N3, ws, p, &lo, status_word));
     {
       const size_t tot = (size_t)R * ld;
-      launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
+      launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
       MOA_CHECK_LAUNCH();
     }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
@@ -616,8 +616,8 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     const int N1[1] = {cq};
     MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
     const size_t tot = (size_t)R * cq;
-    if (q32) launch_pdl(sum_cast_kernel<float>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, q32);
-    else launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
+    if (q32) launch_pdl(sum_cast_kernel<float>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, q32);
+    else launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
     MOA_CHECK_LAUNCH();
   }
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,

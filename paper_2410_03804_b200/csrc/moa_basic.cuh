@@ -11,10 +11,31 @@ namespace moa {
 // One block per row. Input either gathered from the embedding table (tok != nullptr) or read from
 // x[row]. Optionally also writes the un-normalised row in fp32 (the residual stream).
 // ---------------------------------------------------------------------------------------------
+// 8 consecutive elements <-> fp32 registers
+template <typename T> __device__ __forceinline__ void load8(const T* p, float* v);
+template <> __device__ __forceinline__ void load8<float>(const float* p, float* v) {
+  const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+template <> __device__ __forceinline__ void load8<bf16>(const bf16* p, float* v) {
+  bf16x8_to_float(*reinterpret_cast<const uint4*>(p), v);
+}
+template <typename T> __device__ __forceinline__ void store8(T* p, const float* v);
+template <> __device__ __forceinline__ void store8<float>(float* p, const float* v) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+template <> __device__ __forceinline__ void store8<bf16>(bf16* p, const float* v) {
+  *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]),
+                                            pack_bf16(v[6], v[7]));
+}
+
+constexpr int RN_CHUNKS = 8;     // 8-element chunks of a row one thread of a 256-thread block keeps in registers
+
 template <typename TIN, typename T>
-__global__ void rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok, int vocab,
-                                    const T* __restrict__ gain, int K, float eps,
-                                    float* __restrict__ res_out, T* __restrict__ y) {
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok,
+                                                           int vocab, const T* __restrict__ gain, int K, float eps,
+                                                           float* __restrict__ res_out, T* __restrict__ y) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
@@ -27,17 +48,45 @@ __global__ void rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __rest
   } else {
     xr = x + (size_t)r * K;
   }
+  // one pass: the row's chunks stay in registers between the sum of squares and the scaling (rows wider than
+  // 256 * 8 * RN_CHUNKS elements re-read the rest)
+  const int nch = K >> 3;
+  float v[RN_CHUNKS][8];
   float ss = 0.f;
-  for (int k = threadIdx.x; k < K; k += blockDim.x) {
-    float v = to_f<TIN>(xr[k]);
-    ss += v * v;
+#pragma unroll
+  for (int j = 0; j < RN_CHUNKS; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < nch) {
+      load8<TIN>(xr + c * 8, v[j]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss += v[j][i] * v[j][i];
+    }
+  }
+  for (int c = threadIdx.x + RN_CHUNKS * 256; c < nch; c += 256) {
+    float t8[8];
+    load8<TIN>(xr + c * 8, t8);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ss += t8[i] * t8[i];
   }
   ss = block_sum(ss, red);
   const float rinv = rsqrtf(ss / (float)K + eps);
-  for (int k = threadIdx.x; k < K; k += blockDim.x) {
-    float v = to_f<TIN>(xr[k]);
-    if (res_out) res_out[(size_t)r * K + k] = v;
-    y[(size_t)r * K + k] = from_f<T>(v * rinv * to_f<T>(gain[k]));
+  auto finish = [&](int c, const float* a) {
+    if (res_out) store8<float>(res_out + (size_t)r * K + c * 8, a);
+    float g8[8], o[8];
+    load8<T>(gain + c * 8, g8);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = a[i] * rinv * g8[i];
+    store8<T>(y + (size_t)r * K + c * 8, o);
+  };
+#pragma unroll
+  for (int j = 0; j < RN_CHUNKS; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < nch) finish(c, v[j]);
+  }
+  for (int c = threadIdx.x + RN_CHUNKS * 256; c < nch; c += 256) {
+    float t8[8];
+    load8<TIN>(xr + c * 8, t8);
+    finish(c, t8);
   }
 }
 
@@ -117,33 +166,48 @@ __device__ __forceinline__ float sum_splits(const float* p, size_t plane, int sp
 // xres[r, :] += sum of partial planes [R, K]; then, if gain != nullptr, xn = RMSNorm(xres; gain) as T;
 // optionally also copies the updated xres to hidden_out as T. One block per row.
 template <typename T>
-__global__ void residual_norm_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
-                                     int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
-                                     T* __restrict__ hidden_out) {
+__global__ void __launch_bounds__(256) residual_norm_kernel(float* __restrict__ xres, const float* __restrict__ part,
+                                                            int splits, size_t plane, int K, const T* __restrict__ gain,
+                                                            float eps, T* __restrict__ xn, T* __restrict__ hidden_out) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
   const int r = blockIdx.x;
+  const int nch = K >> 3;
   float ss = 0.f;
-  for (int k = threadIdx.x; k < K; k += blockDim.x) {
-    float v = xres[(size_t)r * K + k];
-    if (part) v += sum_splits(part + (size_t)r * K + k, plane, splits);
-    xres[(size_t)r * K + k] = v;
-    ss += v * v;
+  for (int c = threadIdx.x; c < nch; c += 256) {
+    float v[8];
+    load8<float>(xres + (size_t)r * K + c * 8, v);
+    if (part) {
+      float t8[8];
+      load8_planes(part + (size_t)r * K + c * 8, splits, plane, t8);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] += t8[i];
+      store8<float>(xres + (size_t)r * K + c * 8, v);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ss += v[i] * v[i];
   }
   if (gain == nullptr && hidden_out == nullptr) return;
   ss = block_sum(ss, red);
   const float rinv = rsqrtf(ss / (float)K + eps);
-  for (int k = threadIdx.x; k < K; k += blockDim.x) {
-    const float v = xres[(size_t)r * K + k];
-    if (hidden_out) hidden_out[(size_t)r * K + k] = from_f<T>(v);
-    if (gain) xn[(size_t)r * K + k] = from_f<T>(v * rinv * to_f<T>(gain[k]));
+  for (int c = threadIdx.x; c < nch; c += 256) {
+    float v[8];
+    load8<float>(xres + (size_t)r * K + c * 8, v);        // this thread wrote it
+    if (hidden_out) store8<T>(hidden_out + (size_t)r * K + c * 8, v);
+    if (gain) {
+      float g8[8], o[8];
+      load8<T>(gain + c * 8, g8);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o[i] = v[i] * rinv * g8[i];
+      store8<T>(xn + (size_t)r * K + c * 8, o);
+    }
   }
 }
 
 // Same operation spread over a thread-block cluster of 8 CTAs per row: each CTA owns K/8 columns, keeps
 // them in registers, and the row's sum of squares is exchanged through distributed shared memory (added
-// in rank order, so the result does not depend on scheduling). Needs K % 8 == 0 and K <= 16384.
+// in rank order, so the result does not depend on scheduling). Needs K % 64 == 0 and K <= 32768.
 constexpr int RN_CLUSTER = 8;
 constexpr int RN_MAX_PER_THREAD = 8;
 
@@ -158,21 +222,26 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
   __shared__ float cta_ss;
   const int r = blockIdx.y;
   const int rank = blockIdx.x;                       // cluster spans blockIdx.x = 0..7
-  const int cpc = K / RN_CLUSTER;                    // columns per CTA
+  const int cpc = K / RN_CLUSTER;                    // columns per CTA (a multiple of 8: K % 64 == 0)
   const int c0 = rank * cpc;
-  float v[RN_MAX_PER_THREAD];
+  const int nch = cpc >> 3;
+  float v[RN_MAX_PER_THREAD / 4][8];                 // up to two 8-element chunks per thread
   float ss = 0.f;
 #pragma unroll
-  for (int i = 0; i < RN_MAX_PER_THREAD; ++i) {
-    const int c = threadIdx.x + i * 256;
-    v[i] = 0.f;
-    if (c < cpc) {
-      const size_t idx = (size_t)r * K + c0 + c;
-      float a = xres[idx];
-      if (part) a += sum_splits(part + idx, plane, splits);
-      xres[idx] = a;
-      v[i] = a;
-      ss += a * a;
+  for (int j = 0; j < RN_MAX_PER_THREAD / 4; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < nch) {
+      const size_t idx = (size_t)r * K + c0 + c * 8;
+      load8<float>(xres + idx, v[j]);
+      if (part) {
+        float t8[8];
+        load8_planes(part + idx, splits, plane, t8);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[j][i] += t8[i];
+        store8<float>(xres + idx, v[j]);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ss += v[j][i] * v[j][i];
     }
   }
   if (gain == nullptr && hidden_out == nullptr) return;     // uniform over the whole grid
@@ -195,39 +264,51 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
   const float rinv = rsqrtf(total / (float)K + eps);
 #pragma unroll
-  for (int i = 0; i < RN_MAX_PER_THREAD; ++i) {
-    const int c = threadIdx.x + i * 256;
-    if (c < cpc) {
-      const size_t idx = (size_t)r * K + c0 + c;
-      if (hidden_out) hidden_out[idx] = from_f<T>(v[i]);
-      if (gain) xn[idx] = from_f<T>(v[i] * rinv * to_f<T>(gain[c0 + c]));
+  for (int j = 0; j < RN_MAX_PER_THREAD / 4; ++j) {
+    const int c = threadIdx.x + j * 256;
+    if (c < nch) {
+      const size_t idx = (size_t)r * K + c0 + c * 8;
+      if (hidden_out) store8<T>(hidden_out + idx, v[j]);
+      if (gain) {
+        float g8[8], o[8];
+        load8<T>(gain + c0 + c * 8, g8);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = v[j][i] * rinv * g8[i];
+        store8<T>(xn + idx, o);
+      }
     }
   }
 }
 
-// h = silu(sum gate) * (sum up): a partial plane row holds [gate | up] (2F columns).
+// h = silu(sum gate) * (sum up): a partial plane row holds [gate | up] (2F columns). One thread per 8 columns.
 template <typename T>
 __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
                                       T* __restrict__ h, size_t total) {
   pdl_trigger();
   pdl_wait();
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (i >= total) return;
   const size_t r = i / F;
   const int c = (int)(i - r * F);
-  const float g = sum_splits(part + r * 2 * F + c, plane, splits);
-  const float u = sum_splits(part + r * 2 * F + F + c, plane, splits);
-  h[i] = from_f<T>(g / (1.f + __expf(-g)) * u);
+  float g8[8], u8[8], o[8];
+  load8_planes(part + r * 2 * F + c, splits, plane, g8);
+  load8_planes(part + r * 2 * F + F + c, splits, plane, u8);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) o[k] = g8[k] / (1.f + __expf(-g8[k])) * u8[k];
+  store8<T>(h + i, o);
 }
 
-// y = T(sum of planes), flat.
+// y = T(sum of planes), flat. One thread per 8 elements.
 template <typename T>
 __global__ void sum_cast_kernel(const float* __restrict__ part, int splits, size_t plane, size_t total,
                                 T* __restrict__ y) {
   pdl_trigger();
   pdl_wait();
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < total) y[i] = from_f<T>(sum_splits(part + i, plane, splits));
+  const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (i >= total) return;
+  float v[8];
+  load8_planes(part + i, splits, plane, v);
+  store8<T>(y + i, v);
 }
 
 // ---------------------------------------------------------------------------------------------
