@@ -307,7 +307,8 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
   launch_pdl(attn_split_kernel<DH, QSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
-    launch_pdl(attn_combine_kernel<DH>, dim3(nseq * P.rows_per_seq * P.hq), dim3(DH), 0, s, P.part_o, P.part_ml, P.n_parts, P.out);
+    launch_pdl(attn_combine_kernel<DH>, dim3((nseq * P.rows_per_seq * P.hq + 7) / 8), dim3(256), 0, s, P.part_o, P.part_ml, P.n_parts,
+               nseq * P.rows_per_seq * P.hq, P.out);
     MOA_CHECK_LAUNCH();
   }
   return MOA_OK;

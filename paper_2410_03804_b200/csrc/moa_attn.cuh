@@ -306,25 +306,54 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   }
 }
 
-// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One block of DH threads per (row, head).
+// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One warp per (row, head): the parts'
+// (max, sum) pairs are loaded one per lane, their weights travel by shuffles, and the partial outputs are read
+// four parts at a time, so the merge costs a few memory round trips whatever the number of parts.
 template <int DH>
-__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int n_parts,
-                                    bf16* __restrict__ out) {
+__global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o,
+                                                           const float* __restrict__ part_ml, int n_parts, int n_rh,
+                                                           bf16* __restrict__ out) {
   pdl_trigger();
   pdl_wait();
-  const size_t rh = blockIdx.x;
-  const int d = threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int rh = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (rh >= n_rh) return;
   float M = -INFINITY;
-  for (int p = 0; p < n_parts; ++p) M = fmaxf(M, part_ml[(rh * n_parts + p) * 2]);
-  float L = 0.f, acc = 0.f;
-  for (int p = 0; p < n_parts; ++p) {
-    const float m = part_ml[(rh * n_parts + p) * 2];
-    if (m == -INFINITY) continue;
-    const float w = exp2f(m - M);
-    L += w * part_ml[(rh * n_parts + p) * 2 + 1];
-    acc += w * part_o[(rh * n_parts + p) * DH + d];
+  for (int p0 = 0; p0 < n_parts; p0 += 32) {
+    const float m = p0 + lane < n_parts ? part_ml[((size_t)rh * n_parts + p0 + lane) * 2] : -INFINITY;
+    M = fmaxf(M, warp_max(m));
   }
-  out[rh * DH + d] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+  float L = 0.f, acc[DH / 32];
+#pragma unroll
+  for (int e = 0; e < DH / 32; ++e) acc[e] = 0.f;
+  for (int p0 = 0; p0 < n_parts; p0 += 32) {
+    float wl = 0.f, ww = 0.f;
+    if (p0 + lane < n_parts) {
+      const float2 ml = *reinterpret_cast<const float2*>(part_ml + ((size_t)rh * n_parts + p0 + lane) * 2);
+      ww = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+      wl = ww * ml.y;
+    }
+    L += warp_sum(wl);
+    const int np = min(32, n_parts - p0);
+    for (int pp = 0; pp < np; pp += 4) {
+      float x[4][DH / 32];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int e = 0; e < DH / 32; ++e)
+          x[u][e] = pp + u < np ? part_o[((size_t)rh * n_parts + p0 + pp + u) * DH + lane + 32 * e] : 0.f;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float wu = __shfl_sync(0xffffffffu, ww, (pp + u) & 31);
+        if (pp + u < np)
+#pragma unroll
+          for (int e = 0; e < DH / 32; ++e) acc[e] += wu * x[u][e];
+      }
+    }
+  }
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll
+  for (int e = 0; e < DH / 32; ++e) out[(size_t)rh * DH + lane + 32 * e] = __float2bfloat16_rn(acc[e] * inv);
 }
 
 }  // namespace moa

@@ -368,11 +368,7 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
   }
   __syncthreads();
   const float* row0 = qkv + (size_t)r * ld;
-  auto row = [&](int c) {                 // the K-split partial planes are added in a fixed order
-    float a = 0.f;
-    for (int sp = 0; sp < splits; ++sp) a += row0[(size_t)sp * plane + c];
-    return a;
-  };
+  auto row = [&](int c) { return load1_planes(row0 + c, splits, plane); };   // planes added in a fixed order
   // blockIdx.y walks the heads: query heads (when qdst is given), then key heads, then value heads
   int h = blockIdx.y;
   const int nqh = qdst ? hq : 0;
@@ -415,14 +411,13 @@ __global__ void cache_append_kernel(const float* __restrict__ kv, int splits, si
   const int seq = split.seq_of(t);
   const int i = t - split.off[seq];
   const size_t dst = ((size_t)seq * max_ctx + len[seq] + i) * width;
-  for (int c = threadIdx.x; c < width; c += blockDim.x) {
-    float a = 0.f, b = 0.f;
-    for (int sp = 0; sp < splits; ++sp) {
-      a += kv[(size_t)sp * plane + (size_t)r * ld + k_off + c];
-      b += kv[(size_t)sp * plane + (size_t)r * ld + v_off + c];
-    }
-    kdst[dst + c] = from_f<T>(a);
-    vdst[dst + c] = from_f<T>(b);
+  const int nch = width >> 3;
+  for (int c = threadIdx.x; c < 2 * nch; c += blockDim.x) {      // one thread per 8 columns of k, then of v
+    const bool isv = c >= nch;
+    const int cc = (isv ? c - nch : c) * 8;
+    float v8[8];
+    load8_planes(kv + (size_t)r * ld + (isv ? v_off : k_off) + cc, splits, plane, v8);
+    store8<T>((isv ? vdst : kdst) + dst + cc, v8);
   }
 }
 
