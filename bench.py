@@ -162,6 +162,24 @@ def workload_config(p):
 
 
 # ---------------------------------------------------------------------------------------------------
+# replicas: the path does not shard, so N GPUs run N independent copies of the same cycle
+# ---------------------------------------------------------------------------------------------------
+def replica_aggregate(ms_local: float, units_per_rank: float, device=None):
+    """Whole-job numbers from one rank's device time for its timed region: the slowest rank's time (max over
+    ranks, as every rank must finish) and the units all ranks processed per second. No data-path collective:
+    this all-reduce of one float is measurement only. Works on any initialised process group (NCCL or gloo)."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size() if dist.is_available() and dist.is_initialized() else 1
+    ms = float(ms_local)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms, world * units_per_rank / (ms * 1e-3)
+
+
+# ---------------------------------------------------------------------------------------------------
 # the CUDA path
 # ---------------------------------------------------------------------------------------------------
 def main():
@@ -256,11 +274,7 @@ def main():
             fn()
         stop.record()
         barrier()
-        ms = start.elapsed_time(stop)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms, _ = replica_aggregate(start.elapsed_time(stop), 1.0, dev)
         return ms
 
     for _ in range(args.warmup):
