@@ -44,6 +44,11 @@ def algorithmic_bytes(p) -> dict:
     return dict(step=(sa_w + ca_w + lm + caches) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (wstream_gemm_kernel<16>, mode 1) from the ncu
+# capture summarised in profiles/lm_head_wstream_c2.md; set back to None when that kernel changes.
+LM_HEAD_TRAFFIC = {"c2": 1051065600 + 12941056}
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -180,6 +185,83 @@ def replica_aggregate(ms_local: float, units_per_rank: float, device=None):
 
 
 # ---------------------------------------------------------------------------------------------------
+# config 3: LSA prefill throughput (a dense contraction: reported against the tensor-core roofline)
+# ---------------------------------------------------------------------------------------------------
+def run_lsa_prefill(args, p, dev, rank, world):
+    import torch
+    from paper_2410_03804_b200 import moa, synth
+    n_tok = p.lsa_tokens
+    small = synth.scaled(p, vocab=256)           # the LSA pass touches neither the embedding nor the LM head
+    w = {k: v.to(dev) for k, v in synth.make_weights(small).items()}
+    cfg = {k: small.as_dict()[k] for k in CFG_KEYS}
+    g = moa.MoA(cfg, w, 1, n_tok, lsa_chunk_tokens=256)
+    h_host = synth.make_h_stack(p, n_tok).pin_memory()
+    h_dev = h_host.to(dev)
+    h_stage = torch.empty_like(h_dev)
+    kv_host = torch.empty((n_tok, p.d_stack), dtype=h_dev.dtype).pin_memory()
+
+    def step(h):
+        g.moa_state_set_len("ca", [0])
+        return g.moa_lsa_forward(h, [n_tok], want_kv=True)
+
+    def step_e2e():
+        h_stage.copy_(h_host, non_blocking=True)
+        kv_host.copy_(step(h_stage), non_blocking=True)
+
+    def timed(fn, k):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(k):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return replica_aggregate(a.elapsed_time(b), 1.0, dev)[0]
+
+    for _ in range(args.warmup):
+        step(h_dev)
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    n0 = g.moa_launch_count()
+    g.moa_profile_begin()
+    ms = timed(lambda: step(h_dev), args.steps) / args.steps
+    launches = g.moa_launch_count() - n0
+    ph = g.moa_profile_phases()
+    g.moa_profile_end()
+    ms_e2e = timed(step_e2e, args.steps) / args.steps
+    clocks = sampler.stop()
+    assert g.moa_state_status() == 0
+    if args.phases:
+        sys.stderr.write("[phases, last pass of 256 tokens] " + " ".join(f"{k}:{u:.1f}({w_:.1f})" for k, u, w_ in ph) + "\n")
+    S, D_, F, dh = p.n_stack, p.d_stack, p.lsa_mlp, p.head_dim
+    qkv = (p.lsa_hq + 2 * p.lsa_hkv) * dh
+    flops = n_tok * S * 2.0 * (D_ * qkv + p.lsa_hq * dh * D_ + 3 * D_ * F) + n_tok * p.lsa_hq * 4.0 * S * S * dh
+    peak_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak, kind = 1413.4, "fallback"
+    if os.path.exists(peak_path):
+        with open(peak_path) as f:
+            peak, kind = float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+    tf = flops / (ms * 1e-3) / 1e12
+    gemm_us = sum(u for k, u, _w in ph if k == "gemm")
+    line = {"metric": "lsa_prefill_tokens_per_sec", "value": world * n_tok / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"c3: LSA prefill, {n_tok} tokens x {S} stacked activations x {D_}, {p.lsa_hq} heads x {dh}, "
+                                   f"MLP {F}; one step = moa_lsa_forward over all tokens in passes of 256",
+                       "l2": "inputs larger than L2 (2.2 GB of activations, 436 MB of weights)"},
+            "e2e": {"value": world * n_tok / (ms_e2e * 1e-3), "unit": "tokens/s",
+                    "h2d_bytes_per_step": h_host.numel() * 2, "d2h_bytes_per_step": kv_host.numel() * 2},
+            "gpu_launches": launches, "clocks": clocks,
+            "roofline": {"bound": "tensor", "kernel": "phase_machine_kernel<256> (the whole fused LSA pass)",
+                         "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "peak_kind": f"of {kind}",
+                         "traffic": None, "algorithmic_flops_per_step": flops,
+                         "gemm_phase_share_of_last_pass": gemm_us / max(sum(u for _, u, _w in ph), 1e-9)},
+            "replicas": "replicas only: no data-path collective" if world > 1 else None}
+    if rank == 0:
+        print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------
 # the CUDA path
 # ---------------------------------------------------------------------------------------------------
 def main():
@@ -191,6 +273,9 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every cycle on the stream instead of replaying a CUDA graph")
+    ap.add_argument("--fused-step", action="store_true",
+                    help="every forward as one persistent kernel (MOA_OPT_FUSED_STEP); implies --no-graph")
+    ap.add_argument("--phases", action="store_true", help="with --fused-step or --workload c3: print per-phase times to stderr")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
@@ -213,11 +298,18 @@ def main():
     if world > 1:
         dist.init_process_group("nccl")
     dev = torch.device("cuda", local)
+    if args.workload == "c3":
+        run_lsa_prefill(args, p, dev, rank, world)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    if args.fused_step:
+        args.no_graph = True
     # Replicas only: the path does not shard (one sequence batch per GPU, no data-path collective).
     w = {k: v.to(dev) for k, v in synth.make_weights(p).items()}
     cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
     max_ctx = p.ctx + 64
-    g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens)
+    g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens, fused_step=args.fused_step)
     caK, caV = synth.make_cache(p, "ca")
     saK, saV = synth.make_cache(p, "sa")
     g.fill_cache("ca", caK.to(dev), caV.to(dev))
@@ -239,7 +331,7 @@ def main():
     mask_host = torch.empty((nb, W, W), dtype=torch.uint8).pin_memory()
     lens = [p.ctx] * nb
 
-    def cycle(h, tok, root):
+    def cycle(h, tok, root, show=False):
         g.moa_state_set_len("ca", lens)
         g.moa_state_set_len("sa", lens)
         g.moa_lsa_forward(h, [A] * nb, want_kv=False)
@@ -249,6 +341,10 @@ def main():
         for s in range(D):
             R = nb if s == 0 else nb * B
             ids, lp, _ = g.moa_draft_step(out=(ids_buf[:R], lp_buf[:R], None))
+            if show and s in (0, 1):
+                ph = g.moa_profile_phases()
+                sys.stderr.write(f"[phases, forward {s}] total {sum(u for _, u, _w in ph):.1f} us: " +
+                                 " ".join(f"{k}:{u:.1f}({w_:.1f})" for k, u, w_ in ph) + "\n")
             res = g.moa_tree_expand(ids, lp, out=outs)
         return moa.moa_tree_attn_mask(res[1])
 
@@ -321,6 +417,8 @@ def main():
     # the stream (events cannot be read inside a graph), directly after the timed replays
     g.moa_profile_begin()
     ms_stream = timed(lambda: cycle(h_dev, tok_dev, root_dev), args.steps)
+    if args.fused_step and args.phases:
+        cycle(h_dev, tok_dev, root_dev, show=True)
     lm_ms, lm_n = g.moa_profile_end()
     clocks = sampler.stop()
     launches = launches_per_cycle * args.steps
@@ -346,7 +444,8 @@ def main():
         "ms_per_step_stream_launches": ms_stream / args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "lm_head", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}",
+                     "traffic": LM_HEAD_TRAFFIC.get(p.name),
                      "launches_timed": lm_n, "avg_launch_us": lm_avg_s * 1e6,
                      "timed_over": "the same cycles launched on the stream right after the timed replays",
                      "algorithmic_bytes_per_launch": ab["lm_head"]},
