@@ -199,7 +199,8 @@ moa_status moa_profile_end(moa_ctx *ctx, double *ms_total, int32_t *launches);
  * moa_profile_begin and moa_profile_end with the same workspace. us_out[i] = microseconds phase i took on CTA 0
  * including its closing barrier, wait_us_out[i] (may be NULL) = the part of it CTA 0 spent in that barrier,
  * kind_out[i] = its kind (0 GEMM, 1 embed+norm, 2 row norm, 3 residual+norm, 4 rotary, 5 attention,
- * 6 attention merge, 7 SwiGLU, 8 sum+cast, 9 layer mean+norm, 10 cache append, 11 LM-head merge).
+ * 6 attention merge, 7 SwiGLU, 8 sum+cast, 9 layer mean+norm, 10 cache append, 11 LM-head merge,
+ * 12 layer self-attention).
  * Synchronises the stream. HOST output arrays of `cap` entries. */
 moa_status moa_profile_phases(moa_ctx *ctx, const void *ws, size_t ws_bytes, int32_t cap, double *us_out,
                               double *wait_us_out, int32_t *kind_out, int32_t *n_out, void *stream);

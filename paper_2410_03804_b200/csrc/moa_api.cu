@@ -804,6 +804,28 @@ static void pm_attention_ops(PmBuild& b, const Workspace& p, char* ws, int R, in
   }
 }
 
+// Layer Self-Attention phase: one warp per (token, query head), rows staged by bulk asynchronous copies.
+// Falls back to the general attention phase when the layer stack does not fit (S > 128).
+static void pm_lsa_attention_op(PmBuild& b, const Workspace& p, char* ws, int R, int n_tok, int S, int hq, int hkv, int dh,
+                                const bf16* qkv, int ld, bf16* out) {
+  const int s_pad = (S + 15) & ~15;
+  const size_t per_warp = (size_t)3 * s_pad * (dh * 2 + 16) + 16;
+  const int stage = WS_W_BYTES + b.NB * WS_BK * 2;
+  const size_t avail = b.dense ? (size_t)((b.ctx->smem_optin - PM_FIXED_SMEM) / stage) * stage : (size_t)96 * 1024;
+  const int n_warps = imin(PM_WWARPS, (int)(avail / per_warp));
+  if (S > 128 || n_warps < 1) {
+    const int nq = hq * dh, nkv = hkv * dh;
+    pm_attention_ops(b, p, ws, R, n_tok, S, hq, hkv, dh, qkv, nullptr, ld, -1, qkv + nq, qkv + nq + nkv, S, ld, nullptr, S,
+                     S, nullptr, nullptr, 0, nullptr, 0, 0, 0, out);
+    return;
+  }
+  if (n_warps * per_warp > b.attn_bytes) b.attn_bytes = n_warps * per_warp;
+  PmOp* op = pm_op(b, PH_LSA_ATTN, -1, R, n_tok);
+  op->p[0] = qkv; op->p[1] = out;
+  op->i[0] = ld; op->i[1] = hq; op->i[2] = hkv; op->i[3] = S; op->i[4] = n_warps; op->i[5] = b.lo_rows; op->i[6] = dh;
+  op->f[0] = 1.4426950408889634f / sqrtf((float)dh);
+}
+
 static void pm_resnorm(PmBuild& b, int gemm, int R, int K, float* xres, const void* gain, bf16* xn, void* hidden,
                        float eps) {
   PmOp* op = pm_op(b, PH_RESNORM, gemm, R, K);
@@ -954,16 +976,14 @@ static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt
     const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 0, part, p.part_rows);
     PmOp* op = pm_op(b, PH_SUMCAST, g0, R, ld);
     op->p[0] = narrow;
-    pm_attention_ops(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, nullptr, ld, -1, narrow + nq, narrow + nq + nkv,
-                     S, ld, nullptr, S, S, nullptr, nullptr, 0, nullptr, 0, 0, 0, obuf);
+    pm_lsa_attention_op(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, ld, obuf);
     const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 0, part, p.part_rows);
     pm_resnorm(b, g1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
     g_down = pm_mlp(b, p, ws, R, D, F, w.lsa_wgate, w.lsa_wup, w.lsa_wdown);
   } else {
     const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 2, nullptr, 0);
     b.P.g[g0].out16 = narrow; b.P.g[g0].ld16 = ld;
-    pm_attention_ops(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, nullptr, ld, -1, narrow + nq, narrow + nq + nkv,
-                     S, ld, nullptr, S, S, nullptr, nullptr, 0, nullptr, 0, 0, 0, obuf);
+    pm_lsa_attention_op(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, ld, obuf);
     const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 3, xres, 0);
     b.P.g[g1].ldo = D;
     pm_resnorm(b, -1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);

@@ -19,6 +19,7 @@
 #include "moa_pm_attn.cuh"
 #include "moa_pm_common.cuh"
 #include "moa_pm_glue.cuh"
+#include "moa_pm_lsa.cuh"
 #include "moa_pm_merge.cuh"
 
 namespace moa {

@@ -29,7 +29,7 @@ constexpr int PM_MERGE_OWN = 24;         // vocabulary slices one thread owns in
 
 enum PmKind : int {
   PH_GEMM = 0, PH_EMBED_NORM, PH_ROWS_NORM, PH_RESNORM, PH_ROPE, PH_ATTN, PH_COMBINE, PH_SILU, PH_SUMCAST,
-  PH_MEAN_NORM, PH_CACHE_APPEND, PH_MERGE
+  PH_MEAN_NORM, PH_CACHE_APPEND, PH_MERGE, PH_LSA_ATTN
 };
 
 struct PmGemm {            // (its tensor maps are PmParams.tm[gemm][0..2] weights, [3] activations)

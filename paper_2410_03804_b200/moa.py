@@ -294,7 +294,7 @@ class MoA:
         return ms.value, n.value
 
     PHASE_KINDS = ["gemm", "embed_norm", "rows_norm", "res_norm", "rope", "attention", "attn_merge", "swiglu",
-                   "sum_cast", "mean_norm", "cache_append", "lm_merge"]
+                   "sum_cast", "mean_norm", "cache_append", "lm_merge", "lsa_attention"]
 
     def moa_profile_phases(self, stream=None):
         """[(kind name, microseconds, of which in the closing barrier)] of the last fused launch made while
