@@ -5,10 +5,10 @@
 // tensor cores as the A operand (M = 128) of tcgen05.mma. The R activation rows (R <= 256 per call) are
 // the B operand (N = R padded to 16/32/64/128/256), re-fetched from L2 next to each weight tile.
 // Accumulators live in TMEM, double-buffered so that the epilogue of one tile overlaps the MMAs of the
-// next. One CTA per SM, persistent over work units (weight tile x K split), 6 warps:
+// next. One CTA per SM, persistent over work units (weight tile x K split), 10 warps:
 //   warp 0     : TMA producer (one lane)
 //   warp 1     : TMEM allocation + MMA issue (one lane)
-//   warps 2..5 : epilogue, one TMEM lane quadrant each
+//   warps 2..9 : epilogue, two per TMEM lane quadrant (alternate groups of 16 activation rows)
 // Epilogues:
 //   mode 0: fp32 partial sums, out[split][r][col0 + n]  (the consumer adds the splits in a fixed order,
 //           so results are deterministic and need no atomics or zero-filled buffers)
@@ -25,7 +25,7 @@ namespace moa {
 
 constexpr int WS_BM = 128;         // weight rows per tile (MMA M)
 constexpr int WS_BK = 64;          // k elements per stage: 128 bytes of bf16 = one swizzle row
-constexpr int WS_THREADS = 192;
+constexpr int WS_THREADS = 320;     // TMA warp, MMA warp, eight epilogue warps (two per TMEM lane quadrant)
 constexpr int WS_W_BYTES = WS_BM * WS_BK * 2;
 constexpr int WS_SMEM_BUDGET = 200 * 1024;
 constexpr long long WS_WAIT_CYCLES = 4000000000ll;   // ~2 s at boost clock
@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 128);
+      mbar_init(tempty_bar(b), 256);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -305,6 +305,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int ehalf = (warp - 2) >> 2;      // the quadrant's two warps take alternate groups of 16 activation rows
     int j = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++j) {
@@ -320,7 +321,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
       if (P.mode == 0) {
         float* plane = P.out + (size_t)split * P.plane + P.seg_col[seg] + nrow;
 #pragma unroll 1
-        for (int c0 = 0; c0 < NPAD; c0 += 16) {
+        for (int c0 = ehalf * 16; c0 < NPAD; c0 += 32) {
           if (c0 >= P.R) break;
           float v[16];
           tc_ld16(taddr + c0, v);
@@ -335,7 +336,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
         const int n_sub = 4 * P.tiles_total;
         const int B = P.B;
 #pragma unroll 1
-        for (int c0 = 0; c0 < NPAD; c0 += 16) {
+        for (int c0 = ehalf * 16; c0 < NPAD; c0 += 32) {
           if (c0 >= P.R) break;
           float v[16];
           tc_ld16(taddr + c0, v);
