@@ -142,7 +142,8 @@ moa_status moa_sa_append(moa_ctx *ctx, moa_state *st, const int32_t *tok, const 
  * Its scratch is a fixed array inside the library (4.5 MiB of device memory, held by every GPU on which
  * the library is loaded, until the process exits), so the call allocates and frees nothing. Inputs and
  * outputs are still the caller's: tok, the caches in st.
- *   Limits: sum(n_host) <= MOA_SA_STATIC_MAX_TOKENS, sum(n_host) * d_model * sizeof(T) <= 512 KiB and
+ *   Limits: sum(n_host) <= MOA_SA_STATIC_MAX_TOKENS, rows * d_model * sizeof(T) <= 512 KiB (rows = sum(n_host),
+ *   on bf16 plus that count rounded up to 16, 32, 64 or 128 for the low-order terms of the activations) and
  *   sum(n_host) * 2 * sa_hkv * head_dim * 4 <= 4 MiB; beyond them MOA_ERR_WORKSPACE is returned, nothing
  *   is launched, and moa_last_cuda_error() holds the limits in words.
  *   The first call on a device looks up the array's device address (a CUDA runtime query made with that

@@ -227,6 +227,10 @@ static moa_status launch_ws_any(cudaStream_t s, const WsParams& P, int npad, int
 
 static inline int npad_for(int R) { return R <= 16 ? 16 : R <= 32 ? 32 : R <= 64 ? 64 : R <= 128 ? 128 : 256; }
 
+// Up to 128 rows, bf16 activations travel between kernels as two terms (hi + lo): the low-order rows start at this
+// row offset of every X buffer (0: single term). Producers and the GEMM that consumes them derive it from the same R.
+static inline int lo_rows_of(size_t elt, int R) { return (elt == 2 && R > 0 && R <= 128) ? npad_for(R) : 0; }
+
 static bool fast_shape(const moa_ctx* ctx, int K, int nseg, const void* const* W) {
   if (!ctx->fast || K % WS_BK != 0) return false;
   for (int i = 0; i < nseg; ++i)
@@ -267,12 +271,14 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
     P.plane = out->plane;
     P.status = (int*)status_word;
     const int nblk = (R + 255) / 256;
+    const int lo = lo_rows_of(sizeof(T), R);
+    P.xsplit = lo > 0 ? 1 : 0;
     P.splits = pick_splits(tiles * nblk, P.kb_total, R, p.part_rows, ctx->sm_count);
     out->splits = P.splits;
     for (int r0 = 0; r0 < R; r0 += 256) {
       const int rows = imin(256, R - r0);
-      const int npad = npad_for(rows);
-      if (!encode_map(ctx, &P.tmX, (const bf16*)X + (size_t)r0 * K, rows, K, npad)) return MOA_ERR_CUDA;
+      const int npad = lo > 0 ? 2 * lo : npad_for(rows);
+      if (!encode_map(ctx, &P.tmX, (const bf16*)X + (size_t)r0 * K, lo > 0 ? lo + rows : rows, K, npad)) return MOA_ERR_CUDA;
       P.R = rows;
       P.out = part + (size_t)r0 * ntot;
       const int units = tiles * P.splits;
@@ -308,7 +314,7 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
     launch_pdl(attn_combine_kernel<DH>, dim3((nseq * P.rows_per_seq * P.hq + 7) / 8), dim3(256), 0, s, P.part_o, P.part_ml, P.n_parts,
-               nseq * P.rows_per_seq * P.hq, P.out);
+               nseq * P.rows_per_seq * P.hq, P.out, P.out_lo, P.hq);
     MOA_CHECK_LAUNCH();
   }
   return MOA_OK;
@@ -347,6 +353,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.part_o = (float*)(ws + p.att_o);
     P.part_ml = (float*)(ws + p.att_ml);
     P.out = (bf16*)out;
+    P.out_lo = lo_rows_of(sizeof(T), R);
     P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
     if (q32) return dh == 128 ? launch_attn_split<128, true>(s, P, nseq, nwarps) : launch_attn_split<64, true>(s, P, nseq, nwarps);
     return dh == 128 ? launch_attn_split<128, false>(s, P, nseq, nwarps) : launch_attn_split<64, false>(s, P, nseq, nwarps);
@@ -370,13 +377,13 @@ static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, co
   if (K % (RN_CLUSTER * 8) == 0 && K / RN_CLUSTER <= 256 * 8 * (RN_MAX_PER_THREAD / 4)) {
     launch_pdl(residual_norm_cluster_kernel<T>, dim3(dim3(RN_CLUSTER, R)), dim3(256), 0, s, 
         (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0, lo ? lo->plane : 0, K, (const T*)gain,
-        ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out);
+        ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out, lo_rows_of(sizeof(T), R));
     MOA_CHECK_LAUNCH();
     return MOA_OK;
   }
   launch_pdl(residual_norm_kernel<T>, dim3(R), dim3(256), 0, s, (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0,
                                             lo ? lo->plane : 0, K, (const T*)gain, ctx->c.rms_eps, (T*)(ws + p.xn),
-                                            (T*)hidden_out);
+                                            (T*)hidden_out, lo_rows_of(sizeof(T), R));
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -393,7 +400,8 @@ static moa_status mlp_block(cudaStream_t s, moa_ctx* ctx, const Workspace& p, ch
   MOA_TRY(linear<T>(ctx, s, xn, R, K, 2, W2, N2, ws, p, lo, status_word));
   const size_t total = (size_t)R * F;
   if (total) {
-    launch_pdl(silu_mul_split_kernel<T>, dim3(blocks_for(total / 8, 256)), dim3(256), 0, s, lo->part, lo->splits, lo->plane, F, h, total);
+    launch_pdl(silu_mul_split_kernel<T>, dim3(blocks_for(total / 8, 256)), dim3(256), 0, s, lo->part, lo->splits, lo->plane, F, h, total,
+               lo_rows_of(sizeof(T), R));
     MOA_CHECK_LAUNCH();
   }
   const void* W1[1] = {wdown};
@@ -425,7 +433,8 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     const int R = nt * S;
     const T* x = (const T*)h_stack + (size_t)t0 * S * D;
     // pre-norm and q, k, v projections of every (token, layer) row: rows of [q | k | v]
-    launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn);
+    launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn,
+               lo_rows_of(sizeof(T), R));
     MOA_CHECK_LAUNCH();
     const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
     const int N3[3] = {nq, nkv, nkv};
@@ -450,7 +459,8 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     launch_pdl(mean_layers_kernel<T>, dim3(dim3(nt, (D + 255) / 256)), dim3(256), 0, s, xres, S, D, kvf, kvo);
     MOA_CHECK_LAUNCH();
     // cross-attention keys / values of the new positions, appended to the cache
-    launch_pdl(rmsnorm_rows_kernel<float, T>, dim3(nt), dim3(256), 0, s, kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn);
+    launch_pdl(rmsnorm_rows_kernel<float, T>, dim3(nt), dim3(256), 0, s, kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn,
+               lo_rows_of(sizeof(T), nt));
     MOA_CHECK_LAUNCH();
     const int ckv = c.ca_hkv * dh;
     const void* W2[2] = {w.ca_wk, w.ca_wv};
@@ -478,7 +488,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
   for (int t0 = 0; t0 < total; t0 += p.rows_cap) {
     const int R = (total - t0) < p.rows_cap ? (total - t0) : p.rows_cap;
     launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, tok + t0, c.vocab, (const T*)w.sa_norm1, E,
-                                                c.rms_eps, nullptr, xn);
+                                                c.rms_eps, nullptr, xn, lo_rows_of(sizeof(T), R));
     MOA_CHECK_LAUNCH();
     const void* W2[2] = {w.sa_wk, w.sa_wv};
     const int N2[2] = {nkv, nkv};
@@ -526,8 +536,10 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.c_val = (float*)(ws + p.cval);
     P.c_id = (int*)(ws + p.cid);
     P.status = (int*)status_word;
-    const int npad = npad_for(R);
-    if (!encode_map(ctx, &P.tmX, xn, R, E, npad)) return MOA_ERR_CUDA;
+    const int lo = lo_rows_of(sizeof(T), R);
+    P.xsplit = lo > 0 ? 1 : 0;
+    const int npad = lo > 0 ? 2 * lo : npad_for(R);
+    if (!encode_map(ctx, &P.tmX, xn, lo > 0 ? lo + R : R, E, npad)) return MOA_ERR_CUDA;
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
     MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count)));
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
@@ -576,7 +588,8 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   LinOut lo;
 
   // ---- self-attention block ----
-  launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn);
+  launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn,
+             lo_rows_of(sizeof(T), R));
   MOA_CHECK_LAUNCH();
   const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh;
   {
@@ -1447,7 +1460,8 @@ moa_status moa_sa_append_static(moa_ctx* ctx, moa_state* st, const int32_t* tok,
     if ((long long)st->sa_len_host[b] + n_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
   const moa_config& c = ctx->c;
   const size_t kv_row_bytes = (size_t)2 * c.sa_hkv * c.head_dim * sizeof(float);
-  if (total > MOA_SA_STATIC_MAX_TOKENS || (size_t)total * c.d_model * ctx->elt > SA_STATIC_XN_BYTES ||
+  const size_t xn_rows = (size_t)total + lo_rows_of(ctx->elt, total);     // bf16: a second, low-order term per row
+  if (total > MOA_SA_STATIC_MAX_TOKENS || xn_rows * c.d_model * ctx->elt > SA_STATIC_XN_BYTES ||
       (size_t)total * kv_row_bytes > SA_STATIC_PART_BYTES) {
     snprintf(g_cuda_err, sizeof(g_cuda_err),
              "moa_sa_append_static: %d tokens of width %d exceed the fixed scratch (at most %d tokens, %zu bytes of "

@@ -34,6 +34,7 @@ struct AttnParams {
   int q_tiles;                           // query tiles per (seq, kv head)
   float* part_o; float* part_ml;         // [R*hq][n_parts][DH], [R*hq][n_parts][2]
   bf16* out;                             // [R, hq*DH]
+  int out_lo;                            // > 0: the low-order term of every output goes to row out_lo + r
   float scale_log2;                      // log2(e) / sqrt(DH)
 };
 
@@ -241,15 +242,19 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
       m_run[h] = mn;
     }
     float rs[2] = {0.f, 0.f};
-    uint32_t pf[AT_KB / 16][4];
+    uint32_t pf[AT_KB / 16][4], pl[AT_KB / 16][4];      // probabilities as hi (+ lo with QSPLIT) bf16 terms
 #pragma unroll
     for (int nt = 0; nt < AT_KB / 8; ++nt) {
       const float p0 = exp2f(s[nt][0] - msub[0]), p1 = exp2f(s[nt][1] - msub[0]);
       const float p2 = exp2f(s[nt][2] - msub[1]), p3 = exp2f(s[nt][3] - msub[1]);
       rs[0] += p0 + p1;
       rs[1] += p2 + p3;
-      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+      const bf16 h0 = __float2bfloat16_rn(p0), h1 = __float2bfloat16_rn(p1), h2 = __float2bfloat16_rn(p2),
+                 h3 = __float2bfloat16_rn(p3);
+      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(__bfloat162float(h2), __bfloat162float(h3));
+      pl[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0 - __bfloat162float(h0), p1 - __bfloat162float(h1));
+      pl[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2 - __bfloat162float(h2), p3 - __bfloat162float(h3));
     }
 #pragma unroll
     for (int h = 0; h < 2; ++h) l_run[h] = l_run[h] * corr[h] + rs[h];
@@ -268,6 +273,10 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
         ldsm_x4_t(sV + tile_off<DH>(key, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
         mma_bf16_16816(o[2 * n2], pf[kk], b0, b1);
         mma_bf16_16816(o[2 * n2 + 1], pf[kk], b2, b3);
+        if (QSPLIT) {
+          mma_bf16_16816(o[2 * n2], pl[kk], b0, b1);
+          mma_bf16_16816(o[2 * n2 + 1], pl[kk], b2, b3);
+        }
       }
     }
     __syncthreads();             // the stage may be overwritten by the next prefetch
@@ -289,9 +298,15 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     if (P.n_parts == 1) {
       const float inv = l_run[h] > 0.f ? 1.f / l_run[h] : 0.f;
       bf16* dst = P.out + ((size_t)row * P.hq + head) * DH;
+      bf16* dlo = P.out + ((size_t)(P.out_lo + row) * P.hq + head) * DH;
 #pragma unroll
-      for (int i = 0; i < DH / 8; ++i)
-        *reinterpret_cast<uint32_t*>(dst + i * 8 + tq * 2) = pack_bf16(o[i][2 * h] * inv, o[i][2 * h + 1] * inv);
+      for (int i = 0; i < DH / 8; ++i) {
+        const float a = o[i][2 * h] * inv, b = o[i][2 * h + 1] * inv;
+        const bf16 ha = __float2bfloat16_rn(a), hb = __float2bfloat16_rn(b);
+        *reinterpret_cast<uint32_t*>(dst + i * 8 + tq * 2) = pack_bf16(__bfloat162float(ha), __bfloat162float(hb));
+        if (P.out_lo > 0)
+          *reinterpret_cast<uint32_t*>(dlo + i * 8 + tq * 2) = pack_bf16(a - __bfloat162float(ha), b - __bfloat162float(hb));
+      }
     } else {
       const size_t pidx = ((size_t)row * P.hq + head) * P.n_parts + part;
       float* dst = P.part_o + pidx * DH;
@@ -312,7 +327,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
 template <int DH>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o,
                                                            const float* __restrict__ part_ml, int n_parts, int n_rh,
-                                                           bf16* __restrict__ out) {
+                                                           bf16* __restrict__ out, int out_lo, int hq) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -353,7 +368,12 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restri
   }
   const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll
-  for (int e = 0; e < DH / 32; ++e) out[(size_t)rh * DH + lane + 32 * e] = __float2bfloat16_rn(acc[e] * inv);
+  for (int e = 0; e < DH / 32; ++e) {
+    const float a = acc[e] * inv;
+    const bf16 h = __float2bfloat16_rn(a);
+    out[(size_t)rh * DH + lane + 32 * e] = h;
+    if (out_lo > 0) out[((size_t)out_lo * hq + rh) * DH + lane + 32 * e] = __float2bfloat16_rn(a - __bfloat162float(h));
+  }
 }
 
 }  // namespace moa

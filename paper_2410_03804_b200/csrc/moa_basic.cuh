@@ -30,12 +30,21 @@ template <> __device__ __forceinline__ void store8<bf16>(bf16* p, const float* v
                                             pack_bf16(v[6], v[7]));
 }
 
+// Row r, columns k..k+7 of an X buffer [rows, K]: bf16 buffers with lo_rows > 0 also get the low-order term.
+template <typename T> __device__ __forceinline__ void store8_x(T* xb, size_t K, int r, int k, int lo_rows, const float* v);
+template <> __device__ __forceinline__ void store8_x<float>(float* xb, size_t K, int r, int k, int, const float* v) {
+  store8<float>(xb + (size_t)r * K + k, v);
+}
+template <> __device__ __forceinline__ void store8_x<bf16>(bf16* xb, size_t K, int r, int k, int lo_rows, const float* v) {
+  xbuf_store8(xb, K, r, k, lo_rows, v);
+}
+
 constexpr int RN_CHUNKS = 8;     // 8-element chunks of a row one thread of a 256-thread block keeps in registers
 
 template <typename TIN, typename T>
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok,
                                                            int vocab, const T* __restrict__ gain, int K, float eps,
-                                                           float* __restrict__ res_out, T* __restrict__ y) {
+                                                           float* __restrict__ res_out, T* __restrict__ y, int lo_rows) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
@@ -76,7 +85,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict
     load8<T>(gain + c * 8, g8);
 #pragma unroll
     for (int i = 0; i < 8; ++i) o[i] = a[i] * rinv * g8[i];
-    store8<T>(y + (size_t)r * K + c * 8, o);
+    store8_x<T>(y, (size_t)K, r, c * 8, lo_rows, o);
   };
 #pragma unroll
   for (int j = 0; j < RN_CHUNKS; ++j) {
@@ -168,7 +177,8 @@ __device__ __forceinline__ float sum_splits(const float* p, size_t plane, int sp
 template <typename T>
 __global__ void __launch_bounds__(256) residual_norm_kernel(float* __restrict__ xres, const float* __restrict__ part,
                                                             int splits, size_t plane, int K, const T* __restrict__ gain,
-                                                            float eps, T* __restrict__ xn, T* __restrict__ hidden_out) {
+                                                            float eps, T* __restrict__ xn, T* __restrict__ hidden_out,
+                                                            int lo_rows) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
@@ -200,7 +210,7 @@ __global__ void __launch_bounds__(256) residual_norm_kernel(float* __restrict__ 
       load8<T>(gain + c * 8, g8);
 #pragma unroll
       for (int i = 0; i < 8; ++i) o[i] = v[i] * rinv * g8[i];
-      store8<T>(xn + (size_t)r * K + c * 8, o);
+      store8_x<T>(xn, (size_t)K, r, c * 8, lo_rows, o);
     }
   }
 }
@@ -215,7 +225,7 @@ template <typename T>
 __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
     residual_norm_cluster_kernel(float* __restrict__ xres, const float* __restrict__ part, int splits, size_t plane,
                                  int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
-                                 T* __restrict__ hidden_out) {
+                                 T* __restrict__ hidden_out, int lo_rows) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
@@ -274,7 +284,7 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
         load8<T>(gain + c0 + c * 8, g8);
 #pragma unroll
         for (int i = 0; i < 8; ++i) o[i] = v[j][i] * rinv * g8[i];
-        store8<T>(xn + idx, o);
+        store8_x<T>(xn, (size_t)K, r, c0 + c * 8, lo_rows, o);
       }
     }
   }
@@ -283,7 +293,7 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
 // h = silu(sum gate) * (sum up): a partial plane row holds [gate | up] (2F columns). One thread per 8 columns.
 template <typename T>
 __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
-                                      T* __restrict__ h, size_t total) {
+                                      T* __restrict__ h, size_t total, int lo_rows) {
   pdl_trigger();
   pdl_wait();
   const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
@@ -295,7 +305,7 @@ __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits
   load8_planes(part + r * 2 * F + F + c, splits, plane, u8);
 #pragma unroll
   for (int k = 0; k < 8; ++k) o[k] = g8[k] / (1.f + __expf(-g8[k])) * u8[k];
-  store8<T>(h + i, o);
+  store8_x<T>(h, (size_t)F, (int)r, c, lo_rows, o);
 }
 
 // y = T(sum of planes), flat. One thread per 8 elements.

@@ -42,6 +42,7 @@ struct WsParams {
   int kb_total;            // K / 64
   int splits;              // K splits per tile
   int mode;                // 0: fp32 partials, 1: LM-head partial top-B
+  int xsplit;              // activations carried as two bf16 terms: rows [0, R) hi, rows [NPAD/2, NPAD/2 + R) lo
   int ldo;                 // mode 0: columns of one partial plane
   float* out;              // mode 0: plane `split` starts at out + split * plane; row r, column c at [r * ldo + c]
   size_t plane;            // mode 0: elements between two partial planes
@@ -325,6 +326,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
           if (c0 >= P.R) break;
           float v[16];
           tc_ld16(taddr + c0, v);
+          if (P.xsplit) {                       // W x = W hi + W lo
+            float w2[16];
+            tc_ld16(taddr + NPAD / 2 + c0, w2);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += w2[i];
+          }
           if (valid) {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -340,6 +347,12 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
           if (c0 >= P.R) break;
           float v[16];
           tc_ld16(taddr + c0, v);
+          if (P.xsplit) {
+            float w2[16];
+            tc_ld16(taddr + NPAD / 2 + c0, w2);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += w2[i];
+          }
 #pragma unroll 1
           for (int i = 0; i < 16; ++i) {
             const int r = c0 + i;

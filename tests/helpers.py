@@ -28,12 +28,20 @@ def make_oracle(p: synth.Preset, weights_cpu: dict, cache_f64=True, store=None) 
     return O.Drafter(cfg_of(p), {k: np32(v) for k, v in weights_cpu.items()}, cache_f64=cache_f64, store=store)
 
 
+def split_regime(p: synth.Preset, rows: int = None) -> bool:
+    """bf16 forwards of up to 128 rows carry their activations as two bf16 terms (about 16 bits of mantissa),
+    so their decisions are taken at nearly the oracle's own precision."""
+    rows = p.batch * p.tree_topk if rows is None else rows
+    return p.dtype == "bf16" and rows <= 128
+
+
 def make_oracles(p: synth.Preset, weights_cpu: dict, cache_f64=True):
     """(values, decisions): the unrounded oracle that values are compared with, and the oracle whose
-    top-B decisions are compared -- the same object on the fp32 path, the bf16-storage mode on bf16."""
+    top-B decisions are compared. The same object on the fp32 path and on bf16 forwards of up to 128 rows
+    (activations carried at ~16 bits); the bf16-storage mode on larger bf16 forwards (plain 16-bit activations)."""
     w = {k: np32(v) for k, v in weights_cpu.items()}
     exact = O.Drafter(cfg_of(p), w, cache_f64=cache_f64)
-    if p.dtype == "f32":
+    if p.dtype == "f32" or split_regime(p):
         return exact, exact
     dec = O.Drafter(cfg_of(p), w, cache_f64=cache_f64, store="bf16")
     dec._cache = exact._cache          # share the widened weights
@@ -62,12 +70,17 @@ def assert_rows_close(got, want, tol, what=""):
 def tie_window(p: synth.Preset, z) -> float:
     """How close two of the oracle's log-probabilities must be for either order to count as correct.
 
-    fp32 path: 1e-3, as the task states. bf16 path: the value tolerance itself, 2e-2 * max|z|. Every
-    16-bit storage point between two matrix products adds rounding noise of relative size 2^-9, and
-    after the first few of the ~12 storage points two correct implementations' rounding decisions are
-    uncorrelated, so their logits differ by a few 1e-3 * max|z| whatever rounding points they share; a
+    fp32 path: 1e-3, as the task states. bf16 forwards of up to 128 rows: 1e-3 plus 2e-3 * max|z| -- weights,
+    cache entries and tree keys / values are stored in 16 bits whatever the arithmetic, which leaves the logits
+    about 1e-3 * max|z| away from the fp64 oracle's (measured: worst 1.1e-3 on configs 2 and 4, 1.7e-3 on the
+    reduced shapes). Larger bf16
+    forwards (plain 16-bit activations, compared with the oracle's bf16-storage mode): the value tolerance
+    itself, 2e-2 * max|z|: after ~12 storage roundings the two sides' rounding decisions are uncorrelated, so a
     swap of two tokens closer than the value tolerance is consistent with logits that pass it."""
-    return 1e-3 if p.dtype == "f32" else 2e-2 * float(np.max(np.abs(z)))
+    if p.dtype == "f32":
+        return 1e-3
+    scale = float(np.max(np.abs(z)))
+    return 1e-3 + 2e-3 * scale if split_regime(p) else 2e-2 * scale
 
 
 def check_topk(gpu_ids, gpu_lp, z, tol, window=1e-3, what=""):

@@ -3,8 +3,10 @@
 Tolerances (stated by the benchmark spec): hidden states and log-probabilities within
 max-abs 1e-4 (fp32 path) / 2e-2 (bf16 path) of the row's max |value|; token ids and tree structure
 bit-exact except where the oracle's competing log-probabilities differ by less than the tie window
-(1e-3 on the fp32 path; helpers.tie_window derives the bf16 one). On bf16 the top-B decisions are compared
-with the oracle in its bf16-storage mode, the values with the unrounded oracle walking the same tree.
+(1e-3 on the fp32 path; helpers.tie_window derives the bf16 ones). bf16 forwards of up to 128 rows carry their
+activations as two bf16 terms, so their top-B decisions are compared with the unrounded fp64 oracle directly;
+larger bf16 forwards (plain 16-bit activations) with the oracle in its bf16-storage mode, their values with the
+unrounded oracle walking the same tree.
 """
 import numpy as np
 import pytest
@@ -52,7 +54,7 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
     od = oracle_cycle(p, dec, h_stack, prompt, root, ca_cache, sa_cache, seqs=seqs)
     forced = {b: [([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in od["trees"][b][1]] for b in seqs}
     ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced, seqs=seqs)
-    stats = dict(rows=0, exact=0, worst_hidden=0.0)
+    stats = dict(rows=0, exact=0, worst_hidden=0.0, worst_logp=0.0)
     if ca_cache is None:
         n_tok = [h_stack.shape[0] // nb] * nb
         n = n_tok[0]
@@ -94,7 +96,9 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
                 # values against the unrounded oracle, decisions against the deciding oracle
                 zx = rx["z"]
                 lpx = zx - (zx.max() + np.log(np.exp(zx - zx.max()).sum()))
-                assert np.max(np.abs(lp[gr] - lpx[ids[gr]])) <= tol * np.max(np.abs(zx)), f"logp s{s} r{gr}"
+                lp_err = np.max(np.abs(lp[gr] - lpx[ids[gr]])) / np.max(np.abs(zx))
+                stats["worst_logp"] = max(stats["worst_logp"], float(lp_err))
+                assert lp_err <= tol, f"logp s{s} r{gr}"
                 stats["exact"] += H.check_topk(ids[gr], lp[gr], rd["z"], tol, H.tie_window(p, rd["z"]), f"topk s{s} r{gr}")
                 stats["rows"] += 1
                 f_ids[gr] = rd["ids"]
