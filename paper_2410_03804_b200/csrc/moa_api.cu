@@ -324,7 +324,7 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
 // themselves) with max_len positions at most on the host's count; segment B: tree slots masked per row.
 template <typename T>
 static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int dh, const T* q,
-                            const float* q32, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
+                            const float* q32, int q_splits, size_t q_plane, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
                             int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
                             int slots_ld, int nB, int n_slots, int rows_per_seq, T* out) {
   if (R <= 0) return MOA_OK;
@@ -332,7 +332,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     AttnParams P;
     memset(&P, 0, sizeof(P));
     const int nseq = R / rows_per_seq;
-    P.q = (const bf16*)q; P.q32 = q32; P.q_ld = q_ld;
+    P.q = (const bf16*)q; P.q32 = q32; P.q_splits = q_splits; P.q_plane = q_plane; P.q_ld = q_ld;
     P.hq = hq; P.hkv = hkv; P.group = hq / hkv;
     P.rows_per_seq = rows_per_seq;
     P.kA = (const bf16*)kA; P.vA = (const bf16*)vA; P.capA = capA; P.posA_ld = posA_ld;
@@ -445,7 +445,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
       MOA_CHECK_LAUNCH();
     }
     // attention over the S layer rows of the same token (full mask): "sequence" = token, cap = S
-    MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, nullptr, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld,
+    MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, nullptr, 1, 0, ld, R, c.lsa_hq, c.lsa_hkv, narrow + nq, narrow + nq + nkv, S, ld,
                          nullptr, S, S, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0, S, obuf));
     // out-projection + residual, MLP + residual
     const void* W1[1] = {w.lsa_wo};
@@ -611,7 +611,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     max_sa = imax(max_sa, st->sa_len_host[b]);
     max_ca = imax(max_ca, st->ca_len_host[b]);
   }
-  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
                        c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
                        step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
   {
@@ -629,14 +629,16 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
     const void* W1[1] = {w.ca_wq};
     const int N1[1] = {cq};
     MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
-    const size_t tot = (size_t)R * cq;
-    if (q32) launch_pdl(sum_cast_kernel<float>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, q32);
-    else launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
-    MOA_CHECK_LAUNCH();
+    if (!q32) {                              // fp32 path: queries in the storage type
+      const size_t tot = (size_t)R * cq;
+      launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
+      MOA_CHECK_LAUNCH();
+    }
   }
-  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, cq, R, c.ca_hq, c.ca_hkv, (const T*)st->ca_k, (const T*)st->ca_v,
-                       c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0,
-                       rows_per_seq, obuf));
+  // bf16 path: the attention kernel reads the projection's split planes itself (fp32 queries, two bf16 terms)
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32 ? lo.part : nullptr, lo.splits, lo.plane, cq, R, c.ca_hq, c.ca_hkv,
+                       (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr,
+                       (const T*)nullptr, 0, nullptr, 0, 0, 0, rows_per_seq, obuf));
   {
     const void* W1[1] = {w.ca_wo};
     const int N1[1] = {E};

@@ -22,7 +22,8 @@ constexpr int AT_KB = 64;        // keys per block
 
 struct AttnParams {
   const bf16* q; int q_ld;               // query row r, head h at q + r*q_ld + h*DH
-  const float* q32;                      // QSPLIT kernels: the same layout in fp32 (q is unused then)
+  const float* q32;                      // QSPLIT kernels: the same layout in fp32 (q is unused then), possibly as
+  int q_splits; size_t q_plane;          // q_splits split-K planes of a GEMM, q_plane elements apart, summed on load
   int hq, hkv, group;                    // group = hq / hkv
   int rows_per_seq;                      // query rows of one sequence (tree rows, or LSA layers)
   const bf16* kA; const bf16* vA; int capA; int posA_ld;   // segment A: (seq*capA + j)*posA_ld + g*DH
@@ -122,9 +123,8 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     if (QSPLIT) {
       uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
       if (valid) {
-        const float4* src = reinterpret_cast<const float4*>(P.q32 + (size_t)row * P.q_ld + head * DH + c * 8);
-        const float4 a = src[0], b = src[1];
-        const float x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        float x[8];
+        load8_planes(P.q32 + (size_t)row * P.q_ld + head * DH + c * 8, P.q_splits, P.q_plane, x);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const bf16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
