@@ -97,6 +97,7 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   p.kvn = take(((size_t)chunk_tok + xpad) * c.d_stack * elt);    // their normalised copy, T
   const int gmax = imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), hqmax = imax(c.sa_hq, c.ca_hq);
   p.att_units = (long long)c.tree_topk * gmax * 2 * 160 + 2ll * p.draft_rows * hqmax;
+  if (p.att_units < 10ll * p.draft_rows * hqmax) p.att_units = 10ll * p.draft_rows * hqmax;   // up to ten parts per (row, head)
   p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
   p.att_ml = take(elt == 2 ? (size_t)p.att_units * 2 * sizeof(float) : 256);           // their (max, sum)
   p.q32 = take(elt == 2 ? (size_t)p.draft_rows * hqmax * c.head_dim * sizeof(float) : 256);   // draft-step queries, fp32
@@ -296,12 +297,12 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
   return MOA_OK;
 }
 
-template <int DH, bool QSPLIT>
+template <int DH, bool QSPLIT, bool PSPLIT>
 static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nseq, int nwarps) {
   static bool attr_set = false;
   const int smem = (QSPLIT ? 2 : 1) * nwarps * 16 * DH * 2 + 4 * AT_KB * DH * 2;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<DH, QSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<DH, QSPLIT, PSPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (QSPLIT ? 2 : 1) * 8 * 16 * DH * 2 + 4 * AT_KB * DH * 2);
     if (e != cudaSuccess) {
       snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
@@ -310,7 +311,7 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
     attr_set = true;
   }
   dim3 grid(P.n_parts, P.hkv * P.q_tiles, nseq);
-  launch_pdl(attn_split_kernel<DH, QSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
+  launch_pdl(attn_split_kernel<DH, QSPLIT, PSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
     launch_pdl(attn_combine_kernel<DH>, dim3((nseq * P.rows_per_seq * P.hq + 7) / 8), dim3(256), 0, s, P.part_o, P.part_ml, P.n_parts,
@@ -355,8 +356,12 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.out = (bf16*)out;
     P.out_lo = lo_rows_of(sizeof(T), R);
     P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
-    if (q32) return dh == 128 ? launch_attn_split<128, true>(s, P, nseq, nwarps) : launch_attn_split<64, true>(s, P, nseq, nwarps);
-    return dh == 128 ? launch_attn_split<128, false>(s, P, nseq, nwarps) : launch_attn_split<64, false>(s, P, nseq, nwarps);
+    // fp32 queries are split into two bf16 terms; the probabilities too when the output itself carries two terms
+    if (q32 && P.out_lo > 0)
+      return dh == 128 ? launch_attn_split<128, true, true>(s, P, nseq, nwarps) : launch_attn_split<64, true, true>(s, P, nseq, nwarps);
+    if (q32)
+      return dh == 128 ? launch_attn_split<128, true, false>(s, P, nseq, nwarps) : launch_attn_split<64, true, false>(s, P, nseq, nwarps);
+    return dh == 128 ? launch_attn_split<128, false, false>(s, P, nseq, nwarps) : launch_attn_split<64, false, false>(s, P, nseq, nwarps);
   }
   dim3 grid(R, hq);
   if (dh == 128)

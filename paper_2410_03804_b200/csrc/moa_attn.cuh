@@ -70,7 +70,7 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 // that hi's 8-bit mantissa dropped); scores are Q_hi.K^T + Q_lo.K^T, so they carry the queries at about 16 bits
 // of mantissa while the cached keys stay in their 16-bit storage type. This keeps a peaked softmax (keys
 // with outlier channels) from amplifying the rounding of q.
-template <int DH, bool QSPLIT>
+template <int DH, bool QSPLIT, bool PSPLIT>
 __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   pdl_trigger();
   pdl_wait();
@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
       m_run[h] = mn;
     }
     float rs[2] = {0.f, 0.f};
-    uint32_t pf[AT_KB / 16][4], pl[AT_KB / 16][4];      // probabilities as hi (+ lo with QSPLIT) bf16 terms
+    uint32_t pf[AT_KB / 16][4], pl[AT_KB / 16][4];      // probabilities as hi (+ lo with PSPLIT) bf16 terms
 #pragma unroll
     for (int nt = 0; nt < AT_KB / 8; ++nt) {
       const float p0 = exp2f(s[nt][0] - msub[0]), p1 = exp2f(s[nt][1] - msub[0]);
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
         ldsm_x4_t(sV + tile_off<DH>(key, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
         mma_bf16_16816(o[2 * n2], pf[kk], b0, b1);
         mma_bf16_16816(o[2 * n2 + 1], pf[kk], b2, b3);
-        if (QSPLIT) {
+        if (PSPLIT) {
           mma_bf16_16816(o[2 * n2], pl[kk], b0, b1);
           mma_bf16_16816(o[2 * n2 + 1], pl[kk], b2, b3);
         }
