@@ -106,45 +106,59 @@ def measured_peaks():
 # ---------------------------------------------------------------------------------------------------
 # the CPU oracle, timed on a bounded sample (cpu_baseline leg and --impl reference)
 # ---------------------------------------------------------------------------------------------------
-def oracle_sample(p, rows: int = 2, lsa_tok: int = 1):
-    """Times `lsa_tok` LSA tokens and `rows` drafter forward rows of the workload on the host cores and
-    scales them to one drafting cycle. Returns (cycle_seconds_estimate, cores, description)."""
-    import numpy as np
-    import torch
-    from oracle import moa_oracle as O
-    from paper_2410_03804_b200 import synth
+class OracleSampler:
+    """The CPU oracle set up once on a workload (weights drawn and widened to fp64: set-up, like loading a
+    checkpoint), then timed on bounded samples: `lsa_tok` LSA tokens and `rows` drafter forward rows per sample,
+    scaled to one drafting cycle."""
 
-    cores = torch.get_num_threads()
-    w = synth.make_weights(p)
-    cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
-    dr = O.Drafter(cfg, {k: v.float().numpy() for k, v in w.items()})
-    for name in w:                       # widen the weights once: set-up, like loading a checkpoint
-        dr.w(name)
-    ctx = min(p.ctx, 2048)
-    caK, caV = synth.make_cache(synth.scaled(p, batch=1), "ca", ctx)
-    saK, saV = synth.make_cache(synth.scaled(p, batch=1), "sa", ctx)
-    caK, caV, saK, saV = [t[0].float().numpy().astype(np.float64) for t in (caK, caV, saK, saV)]
-    h = synth.make_h_stack(p, lsa_tok).float().numpy()
-    t0 = time.perf_counter()
-    dr.lsa_forward(h)
-    t_lsa = (time.perf_counter() - t0) / lsa_tok
-    toks = synth.make_root(synth.scaled(p, batch=rows)).tolist()
-    t0 = time.perf_counter()
-    for t in toks:
-        dr.forward_row(t, ctx, saK, saV, caK, caV, p.tree_topk)
-    t_row = (time.perf_counter() - t0) / rows
-    n_rows = p.batch * (1 + p.tree_topk * (p.tree_depth - 1))
-    cycle = p.batch * p.lsa_tokens * t_lsa + n_rows * t_row
-    what = (f"{lsa_tok} LSA token(s) ({t_lsa:.2f} s each) + {rows} drafter forward rows ({t_row:.2f} s each) of {p.name}"
-            f" with {ctx}-entry caches, scaled to one cycle = {p.batch * p.lsa_tokens} LSA tokens + {n_rows} rows;"
-            f" weights widened to fp64 beforehand")
-    return cycle, cores, what
+    def __init__(self, p):
+        import numpy as np
+        import torch
+        from oracle import moa_oracle as O
+        from paper_2410_03804_b200 import synth
+        self.p, self.np, self.synth = p, np, synth
+        self.cores = torch.get_num_threads()
+        w = synth.make_weights(p)
+        cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
+        self.dr = O.Drafter(cfg, {k: v.float().numpy() for k, v in w.items()})
+        for name in w:
+            self.dr.w(name)
+        self.ctx = min(p.ctx, 2048)
+        one = synth.scaled(p, batch=1)
+        caK, caV = synth.make_cache(one, "ca", self.ctx)
+        saK, saV = synth.make_cache(one, "sa", self.ctx)
+        self.caches = [t[0].float().numpy().astype(np.float64) for t in (caK, caV, saK, saV)]
+
+    def sample(self, rows: int = 2, lsa_tok: int = 1):
+        """Returns (cycle_seconds_estimate, cores, description)."""
+        p, synth = self.p, self.synth
+        caK, caV, saK, saV = self.caches
+        h = synth.make_h_stack(p, lsa_tok).float().numpy()
+        t0 = time.perf_counter()
+        self.dr.lsa_forward(h)
+        t_lsa = (time.perf_counter() - t0) / lsa_tok
+        toks = synth.make_root(synth.scaled(p, batch=rows)).tolist()
+        t0 = time.perf_counter()
+        for t in toks:
+            self.dr.forward_row(t, self.ctx, saK, saV, caK, caV, p.tree_topk)
+        t_row = (time.perf_counter() - t0) / rows
+        n_rows = p.batch * (1 + p.tree_topk * (p.tree_depth - 1))
+        cycle = p.batch * p.lsa_tokens * t_lsa + n_rows * t_row
+        what = (f"{lsa_tok} LSA token(s) ({t_lsa:.2f} s each) + {rows} drafter forward rows ({t_row:.2f} s each) of {p.name}"
+                f" with {self.ctx}-entry caches, scaled to one cycle = {p.batch * p.lsa_tokens} LSA tokens + {n_rows} rows;"
+                f" weights widened to fp64 beforehand")
+        return cycle, self.cores, what
+
+
+def oracle_sample(p, rows: int = 2, lsa_tok: int = 1):
+    return OracleSampler(p).sample(rows, lsa_tok)
 
 
 def run_reference(args, p):
+    sampler = OracleSampler(p)                       # set-up is not timed
     t_all = []
     for _ in range(args.warmup + args.steps):
-        cycle, cores, what = oracle_sample(p, rows=1, lsa_tok=1)
+        cycle, cores, what = sampler.sample(rows=1, lsa_tok=1)     # one bounded sample per step
         t_all.append(cycle)
     t = statistics.mean(t_all[args.warmup:]) if len(t_all) > args.warmup else t_all[-1]
     D, m = p.tree_depth, p.tree_keep
