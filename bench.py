@@ -345,13 +345,18 @@ def main():
     mask_host = torch.empty((nb, W, W), dtype=torch.uint8).pin_memory()
     lens = [p.ctx] * nb
 
-    def cycle(h, tok, root, show=False):
+    split_ev = []      # when filled by the caller: (before forwards, after forwards) event pairs of each cycle
+
+    def cycle(h, tok, root, show=False, mark=False):
         g.moa_state_set_len("ca", lens)
         g.moa_state_set_len("sa", lens)
         g.moa_lsa_forward(h, [A] * nb, want_kv=False)
         g.moa_sa_append(tok, [A] * nb)
         g.moa_tree_begin(root)
         res = None
+        if mark:
+            split_ev.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+            split_ev[-1][0].record()
         for s in range(D):
             R = nb if s == 0 else nb * B
             ids, lp, _ = g.moa_draft_step(out=(ids_buf[:R], lp_buf[:R], None))
@@ -360,6 +365,8 @@ def main():
                 sys.stderr.write(f"[phases, forward {s}] total {sum(u for _, u, _w in ph):.1f} us: " +
                                  " ".join(f"{k}:{u:.1f}({w_:.1f})" for k, u, w_ in ph) + "\n")
             res = g.moa_tree_expand(ids, lp, out=outs)
+        if mark:
+            split_ev[-1][1].record()
         return moa.moa_tree_attn_mask(res[1])
 
     def cycle_e2e():
@@ -434,6 +441,9 @@ def main():
     if args.fused_step and args.phases:
         cycle(h_dev, tok_dev, root_dev, show=True)
     lm_ms, lm_n = g.moa_profile_end()
+    # the D forwards alone (draft step + expansion), stream launches, events around them inside each cycle
+    timed(lambda: cycle(h_dev, tok_dev, root_dev, mark=True), args.steps)
+    fwd_us = statistics.mean(a.elapsed_time(b) for a, b in split_ev) * 1e3 / D
     clocks = sampler.stop()
     launches = launches_per_cycle * args.steps
     assert g.moa_state_status() == 0
@@ -467,6 +477,10 @@ def main():
                            "achieved_gbs": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9,
                            "frac_of_measured": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9 / peak,
                            "frac_of_8tbs": (D * ab["step"] + ab["lsa"]) / t_cycle / 1e9 / 8000.0},
+        "forward_roofline": {"what": "one drafter forward + tree expansion, mean over the cycle's forwards, stream launches",
+                             "us": fwd_us, "algorithmic_bytes": ab["step"], "achieved_gbs": ab["step"] / fwd_us / 1e3,
+                             "frac_of_measured": ab["step"] / fwd_us / 1e3 / peak,
+                             "frac_of_8tbs": ab["step"] / fwd_us / 1e3 / 8000.0},
         "replicas": "replicas only: no data-path collective" if world > 1 else None,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
