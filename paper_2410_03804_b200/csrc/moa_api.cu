@@ -1402,7 +1402,7 @@ moa_status moa_tree_expand(moa_ctx* ctx, moa_state* st, int32_t batch, const int
   const TreePtrs tp = tree_ptrs(st->tree, L);
   const int last = (st->step + 1 == c.tree_depth) ? 1 : 0;
   const size_t smem = ((size_t)(L.P > 256 ? L.P : 256) + L.P) * 4;
-  tree_expand_kernel<<<batch, 512, smem, (cudaStream_t)stream>>>(tp, c.tree_topk, c.tree_depth, L.P, c.tree_keep, st->step,
+  launch_pdl(tree_expand_kernel, dim3(batch), dim3(512), smem, (cudaStream_t)stream, tp, c.tree_topk, c.tree_depth, L.P, c.tree_keep, st->step,
                                                                  batch, c.max_batch * c.tree_topk, topk_id, topk_logp,
                                                                  last, out_tok, out_parent, out_depth, out_score, out_n);
   MOA_CHECK_LAUNCH();
