@@ -27,6 +27,11 @@ LSA or CA; the LLM's final RMSNorm gain precedes the LM head; the MLP listed
 probabilities are sums of fp32 log-probabilities. Ties break towards the
 smaller index everywhere.
 
+Target Layer Inference (Section 3.2): with n_tli = N > 0 the N last LLM decoder layers run on every drafted
+row between the CA block and the LM head, each over the LLM's own cache of that layer (positions <= t) plus
+the keys / values of the row's drafted ancestors; a Llama decoder layer (pre-RMSNorm, rotary embedding, GQA,
+SwiGLU, residuals) with weights "tli{l}_*", l = 0 the earliest of the N.
+
 Storage precision: with store="bf16" every tensor that the method keeps in
 the 16-bit storage type between two matrix products is rounded to bfloat16
 (round to nearest even) at that point -- normalised activations entering a
@@ -252,6 +257,35 @@ class Drafter:
         cc = x + linear(self.rnd(o).reshape(hq * dh), self.w("ca_wo"))
         return cc + self.mlp(self.rnd(rmsnorm(cc, self.w("ca_norm2"), c["rms_eps"])), "ca")
 
+    # ---- Target Layer Inference (Section 3.2): the last TLI frozen LLM decoder layers ----------
+    def tli_layers(self):
+        """Number of LLM decoder layers applied between the CA block and the LM head (TLI; 0 = none)."""
+        return int(self.c.get("n_tli", 0))
+
+    def tli_layer(self, l, x, pos, K, V):
+        """One frozen LLM decoder layer f^l_decoder on one drafted row (Section 3.2, the second line of the
+        drafter's equation; Algorithm 1, the loop over l): x [E] is o_hat^l, K, V [n, Hkv, dh] are the layer's
+        cached keys / values the row may see (positions <= t from the LLM, then its drafted ancestors), the row's
+        own key / value joins them. Llama-style reading as for the drafter's own blocks: pre-RMSNorm, rotary
+        embedding at the row's absolute position, GQA, SwiGLU, residuals. Returns (o_hat^{l+1}, k, v)."""
+        c = self.c
+        dh, hq, hkv = c["head_dim"], c["tli_hq"], c["tli_hkv"]
+        w = lambda n: self.w(f"tli{l}_{n}")
+        x = np.asarray(x, F64)
+        u = self.rnd(rmsnorm(x, w("norm1"), c["rms_eps"]))
+        q = self.rnd(rope(linear(u, w("wq")).reshape(hq, dh), pos, c["rope_theta"]))
+        k = self.rnd(rope(linear(u, w("wk")).reshape(hkv, dh), pos, c["rope_theta"]))
+        v = self.rnd(linear(u, w("wv")).reshape(hkv, dh))
+        Kf = np.concatenate([np.asarray(K, F64), k[None]], axis=0)
+        Vf = np.concatenate([np.asarray(V, F64), v[None]], axis=0)
+        o = np.zeros((hq, dh), F64)
+        for h in range(hq):
+            g = kv_head_of(h, hq, hkv)
+            o[h] = attend(q[h], Kf[:, g], Vf[:, g])
+        a = x + linear(self.rnd(o).reshape(hq * dh), w("wo"))
+        out = a + swiglu_mlp(self.rnd(rmsnorm(a, w("norm2"), c["rms_eps"])), w("wgate"), w("wup"), w("wdown"), self.rnd)
+        return out, k, v
+
     def head(self, o_hat, B):
         return lm_head_topk(o_hat, self.w("final_norm"), self.w("lm_head"), self.c["rms_eps"], B, self.rnd)
 
@@ -270,17 +304,22 @@ class Drafter:
                 np.stack(vs) if vs else np.zeros(shape, F64))
 
     # ---- one drafter forward for one row ----------------------------------
-    def forward_row(self, tok, pos, saK, saV, caK, caV, B):
-        """SA -> CA -> LM head for a token at position pos whose visible
-        self-attention keys/values (excluding itself) are saK, saV.
-        Returns dict(x, o_hat, ids, logp, k, v, z)."""
+    def forward_row(self, tok, pos, saK, saV, caK, caV, B, tliKV=None):
+        """SA -> CA -> (TLI decoder layers) -> LM head for a token at position pos whose visible
+        self-attention keys/values (excluding itself) are saK, saV; tliKV[l] = (K, V) visible to the row in
+        TLI layer l (the LLM's cache of that layer, then the row's drafted ancestors).
+        Returns dict(x, o_hat, ids, logp, k, v, z, tli_kv); o_hat is the input of the LM head."""
         e, q, k, v = self.sa_qkv(tok, pos)
         K = np.concatenate([np.asarray(saK, F64), k[None]], axis=0)
         V = np.concatenate([np.asarray(saV, F64), v[None]], axis=0)
         x = self.sa_block(e, q, K, V)
         o_hat = self.ca_block(x, caK, caV)
+        tli_kv = []
+        for l in range(self.tli_layers()):
+            o_hat, kl, vl = self.tli_layer(l, o_hat, pos, tliKV[l][0], tliKV[l][1])
+            tli_kv.append((kl, vl))
         ids, logp, z = self.head(o_hat, B)
-        return dict(x=x, o_hat=o_hat, ids=ids, logp=logp, k=k, v=v, z=z)
+        return dict(x=x, o_hat=o_hat, ids=ids, logp=logp, k=k, v=v, z=z, tli_kv=tli_kv)
 
 
 # --------------------------------------------------------------------------
@@ -362,7 +401,7 @@ def tree_mask(parent):
     return mask
 
 
-def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None):
+def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None, tliK=None, tliV=None):
     """Grow one sequence's draft tree with D drafter forwards.
 
     saK, saV [ctx, Hkv, dh]: self-attention prefix cache (positions 0..ctx-1);
@@ -370,6 +409,8 @@ def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None):
     prefix, its ancestors (root included) and itself.
     forced: optional list of per-step (ids, logp) to expand with instead of
     the oracle's own top-B (used to follow another implementation's choices).
+    tliK, tliV: per TLI layer, the LLM's cache of that layer over the same positions 0..ctx-1, [ctx, Hkv, dh];
+    a node's keys / values in those layers are kept for the cycle and seen by its descendants (Section 3.2).
     Returns (TreeState, steps) with steps[s] = list of forward_row dicts."""
     ctx = saK.shape[0]
     ts = TreeState(root_tok, B, D, m)
@@ -382,11 +423,14 @@ def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None):
             anc = [] if f < 0 else [-1] + ts.path_to(f)[:-1]
             Ks = [saK] + [node_kv[a][0][None] for a in anc]
             Vs = [saV] + [node_kv[a][1][None] for a in anc]
+            tli = [(np.concatenate([tliK[l]] + [node_kv[a][2][l][0][None] for a in anc], 0),
+                    np.concatenate([tliV[l]] + [node_kv[a][2][l][1][None] for a in anc], 0))
+                   for l in range(dr.tli_layers())]
             tok = ts.root_tok if f < 0 else ts.tok[f]
-            out = dr.forward_row(tok, ctx + s, np.concatenate(Ks, 0), np.concatenate(Vs, 0), caK, caV, B)
+            out = dr.forward_row(tok, ctx + s, np.concatenate(Ks, 0), np.concatenate(Vs, 0), caK, caV, B, tli)
             rows.append(out)
         for f, out in zip(ts.frontier, rows):
-            node_kv[f] = (out["k"], out["v"])
+            node_kv[f] = (out["k"], out["v"], out["tli_kv"])
         steps.append(rows)
         if forced is not None:
             ids, logp = forced[s]
@@ -400,7 +444,7 @@ def draft_tree(dr: Drafter, root_tok, saK, saV, caK, caV, B, D, m, forced=None):
 # --------------------------------------------------------------------------
 # independent loop-based paths used to pin the tree code by brute force
 # --------------------------------------------------------------------------
-def sequential_decode(dr: Drafter, prefix_toks, path_toks, caK, caV, B):
+def sequential_decode(dr: Drafter, prefix_toks, path_toks, caK, caV, B, tliK=None, tliV=None):
     """Plain causal decoding, token by token (Algorithm 1, the inner drafting loop with the
     tokens given): the self-attention cache grows by one entry per token and
     every token sees all earlier ones. Returns the forward_row dict of each
@@ -415,21 +459,24 @@ def sequential_decode(dr: Drafter, prefix_toks, path_toks, caK, caV, B):
         V = np.concatenate([V, v[None]], 0)
         pos += 1
     outs = []
+    tli = [(np.asarray(tliK[l], F64), np.asarray(tliV[l], F64)) for l in range(dr.tli_layers())]
     for t in path_toks:
-        out = dr.forward_row(t, pos, K, V, caK, caV, B)
+        out = dr.forward_row(t, pos, K, V, caK, caV, B, tli)
         K = np.concatenate([K, out["k"][None]], 0)
         V = np.concatenate([V, out["v"][None]], 0)
+        tli = [(np.concatenate([tli[l][0], out["tli_kv"][l][0][None]], 0),
+                np.concatenate([tli[l][1], out["tli_kv"][l][1][None]], 0)) for l in range(dr.tli_layers())]
         outs.append(out)
         pos += 1
     return outs
 
 
-def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft):
+def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft, tliK=None, tliV=None):
     """Chain drafting (Algorithm 1, inner loop) with greedy choice: K_draft
     tokens, each the most probable continuation. Returns (tokens, logps)."""
     toks, lps = [int(root_tok)], []
     for _ in range(K_draft):
-        out = sequential_decode(dr, prefix_toks, toks, caK, caV, 1)[-1]
+        out = sequential_decode(dr, prefix_toks, toks, caK, caV, 1, tliK, tliV)[-1]
         toks.append(int(out["ids"][0]))
         lps.append(float(out["logp"][0]))
     return toks[1:], lps
