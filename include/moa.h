@@ -7,8 +7,9 @@
  * causal / tree-masked self-attention over token embeddings and cross-attention into
  * keys and values derived from the LSA output (Section 3.1.2, Algorithm 1), the LM head
  * with log-softmax and the B most probable tokens (Eq. 1), and the EAGLE-2-style dynamic
- * draft tree with its ancestor mask (Section 2.2). Target Layer Inference is fixed at
- * TLI = 0 (Section 3.2): the drafter predicts the last decoder layer's activation.
+ * draft tree with its ancestor mask (Section 2.2). Target Layer Inference (Section 3.2)
+ * is off after moa_create (TLI = 0: the drafter predicts the last decoder layer's
+ * activation); moa_tli_configure turns it on for the last N <= MOA_MAX_TLI decoder layers.
  *
  * Conventions
  *  - Every pointer is DEVICE memory owned by the caller unless its name ends in _host or
@@ -35,6 +36,7 @@ extern "C" {
 #define MOA_MAX_BATCH 64      /* sequences per call */
 #define MOA_MAX_TOPK 16       /* tree breadth B */
 #define MOA_MAX_DEPTH 16      /* tree depth D */
+#define MOA_MAX_TLI 4         /* LLM decoder layers run by the drafter (Target Layer Inference) */
 
 typedef struct moa_ctx moa_ctx; /* opaque, host side */
 
@@ -99,6 +101,37 @@ typedef struct {
  * MOA_ERR_ARCH if the device is not compute capability 10.x: there is no fallback path. */
 moa_status moa_create(const moa_config *cfg, const moa_weights *w, moa_ctx **out);
 void moa_destroy(moa_ctx *ctx);
+
+/* Target Layer Inference (Section 3.2; Algorithm 1, the loop over the last N decoder layers): with TLI = N > 0
+ * the drafter's CA block predicts the input of LLM layer L+1-N, and moa_draft_step then runs the N last
+ * (frozen) LLM decoder layers on the drafted rows before the LM head. Layer l attends over the LLM's own
+ * key/value cache of that layer for the positions already decoded (0 .. sa_len[b]-1, the same positions as the
+ * drafter's self-attention prefix) and over the keys/values of the row's drafted ancestors and itself, which
+ * the library keeps in moa_state.tree for the duration of one tree and drops afterwards.
+ * A layer is a Llama decoder layer: RMSNorm(norm1) -> q,k,v projections -> rotary embedding (half-split
+ * pairing, base rope_theta) at the row's position -> grouped-query attention -> W_o, residual ->
+ * RMSNorm(norm2) -> SwiGLU MLP, residual. Width E = d_model, head size = moa_config.head_dim.
+ *   layers  HOST array [n_layers], layers[0] = the earliest of the N (LLM layer L+1-N); device pointers of T:
+ *           norm1 [E], wq [hq*dh,E], wk, wv [hkv*dh,E], wo [E,hq*dh], norm2 [E], wgate, wup [mlp,E], wdown [E,mlp]
+ *   k, v    device T [max_batch, max_ctx, hkv, head_dim] per layer: the LLM's cache of that layer (keys already
+ *           rotated), owned and filled by the caller, never written by the library
+ * Call it before moa_state_bytes: both sizes grow. n_layers = 0 (layers and caches may be NULL) turns it off
+ * again. With TLI on, MOA_OPT_FUSED_STEP does not apply to moa_draft_step (the launch chain is used).
+ * MOA_ERR_SHAPE for n_layers > MOA_MAX_TLI, hq % hkv != 0, mlp % 16 != 0. */
+typedef struct {
+  int32_t n_layers;  /* N = TLI, 0 .. MOA_MAX_TLI */
+  int32_t hq, hkv;   /* query / key-value heads of an LLM layer */
+  int32_t mlp;       /* its MLP width */
+  float rope_theta;  /* its rotary base; 0 disables the rotation */
+} moa_tli_config;
+typedef struct {
+  const void *norm1, *wq, *wk, *wv, *wo, *norm2, *wgate, *wup, *wdown;
+} moa_tli_layer;
+typedef struct {
+  const void *k[MOA_MAX_TLI], *v[MOA_MAX_TLI];
+} moa_tli_caches;
+moa_status moa_tli_configure(moa_ctx *ctx, const moa_tli_config *cfg, const moa_tli_layer *layers_host,
+                             const moa_tli_caches *caches);
 
 /* Options. MOA_OPT_FUSED_STEP (bf16 only): run moa_draft_step, and moa_lsa_forward passes of any size, as ONE
  * persistent cooperative kernel (phases separated by grid-wide barriers, weights prefetched across phases,
@@ -165,7 +198,8 @@ moa_status moa_tree_begin(moa_ctx *ctx, moa_state *st, const int32_t *root_tok, 
  * sees the prefix, its ancestors and itself.
  *   topk_id    int32 [R, B]  token ids, by (log-probability descending, id ascending)
  *   topk_logp  float [R, B]  their log-probabilities (logit - logsumexp over the vocabulary)
- *   hidden_out T [R, E] or NULL: the drafter's output activation (input of the LM head) */
+ *   hidden_out T [R, E] or NULL: the drafter's output activation (input of the LM head; with Target Layer
+ *              Inference on, the output of the last LLM decoder layer) */
 moa_status moa_draft_step(moa_ctx *ctx, moa_state *st, int32_t batch, int32_t *topk_id, float *topk_logp,
                           void *hidden_out, void *ws, size_t ws_bytes, void *stream);
 

@@ -18,7 +18,7 @@ using namespace moa;
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512, WMAP_MAX = 32 };
+enum { PROF_MAX = 512, WMAP_MAX = 64 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -40,6 +40,11 @@ struct moa_ctx {
   EncodeTiledFn encode;
   WeightMap wmap[WMAP_MAX];
   int n_wmap;
+  int n_wmap_base;     // maps of the drafter's own matrices; those of the Target-Layer-Inference layers follow
+  // Target Layer Inference (Section 3.2): the last N decoder layers of the LLM, off when tli.n_layers == 0
+  moa_tli_config tli;
+  moa_tli_layer tli_w[MOA_MAX_TLI];
+  moa_tli_caches tli_c;
   bool fast;           // weight-streaming tcgen05 GEMMs usable
   bool coop;           // cooperative launches available: the phase-machine kernels are used
   bool fused_step;     // moa_draft_step as one persistent kernel (moa_set_option)
@@ -65,7 +70,7 @@ struct Workspace {
 static inline int imax(int a, int b) { return a > b ? a : b; }
 static inline int imin(int a, int b) { return a < b ? a : b; }
 
-static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) {
+static Workspace plan_workspace(const moa_config& c, const moa_tli_config& t, size_t elt, int chunk_tok) {
   Workspace p;
   p.chunk_tok = chunk_tok;
   p.draft_rows = c.max_batch * c.tree_topk;
@@ -75,10 +80,12 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   const int qkv_lsa = (c.lsa_hq + 2 * c.lsa_hkv) * c.head_dim;
   const int qkv_sa = (c.sa_hq + 2 * c.sa_hkv) * c.head_dim;
   const int q_ca = imax(c.ca_hq * c.head_dim, 2 * c.ca_hkv * c.head_dim);
-  const int fmax = imax(c.lsa_mlp, imax(c.sa_mlp, c.ca_mlp));
-  p.wide = imax(imax(imax(qkv_lsa, qkv_sa), imax(q_ca, 2 * fmax)), dmax);
-  const int narrow = imax(imax(qkv_lsa, qkv_sa), imax(q_ca, fmax));
-  const int omax = imax(c.lsa_hq, imax(c.sa_hq, c.ca_hq)) * c.head_dim;
+  const bool tli = t.n_layers > 0;
+  const int qkv_tli = tli ? (t.hq + 2 * t.hkv) * c.head_dim : 0;
+  const int fmax = imax(imax(c.lsa_mlp, tli ? t.mlp : 0), imax(c.sa_mlp, c.ca_mlp));
+  p.wide = imax(imax(imax(qkv_lsa, imax(qkv_sa, qkv_tli)), imax(q_ca, 2 * fmax)), dmax);
+  const int narrow = imax(imax(qkv_lsa, imax(qkv_sa, qkv_tli)), imax(q_ca, fmax));
+  const int omax = imax(imax(c.lsa_hq, tli ? t.hq : 0), imax(c.sa_hq, c.ca_hq)) * c.head_dim;
   const size_t n_sub = (size_t)4 * ((c.vocab + WS_BM - 1) / WS_BM);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
@@ -95,7 +102,8 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
   p.cid = take(n_sub * p.draft_rows * c.tree_topk * sizeof(int));
   p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));   // LSA output rows, fp32
   p.kvn = take(((size_t)chunk_tok + xpad) * c.d_stack * elt);    // their normalised copy, T
-  const int gmax = imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), hqmax = imax(c.sa_hq, c.ca_hq);
+  const int gmax = imax(imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), tli ? t.hq / t.hkv : 0);
+  const int hqmax = imax(imax(c.sa_hq, c.ca_hq), tli ? t.hq : 0);
   p.att_units = (long long)c.tree_topk * gmax * 2 * 160 + 2ll * p.draft_rows * hqmax;
   if (p.att_units < 10ll * p.draft_rows * hqmax) p.att_units = 10ll * p.draft_rows * hqmax;   // up to ten parts per (row, head)
   p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
@@ -107,14 +115,14 @@ static Workspace plan_workspace(const moa_config& c, size_t elt, int chunk_tok) 
 }
 
 // Largest token chunk whose plan fits in ws_bytes (plan size is monotone in the chunk); 0 if none.
-static int chunk_from_bytes(const moa_config& c, size_t elt, size_t ws_bytes) {
-  if (plan_workspace(c, elt, 1).total > ws_bytes) return 0;
+static int chunk_from_bytes(const moa_config& c, const moa_tli_config& t, size_t elt, size_t ws_bytes) {
+  if (plan_workspace(c, t, elt, 1).total > ws_bytes) return 0;
   int lo = 1;
-  while (lo < (1 << 20) && plan_workspace(c, elt, lo * 2).total <= ws_bytes) lo *= 2;
+  while (lo < (1 << 20) && plan_workspace(c, t, elt, lo * 2).total <= ws_bytes) lo *= 2;
   int hi = lo * 2;
   while (lo + 1 < hi) {
     const int mid = lo + (hi - lo) / 2;
-    if (plan_workspace(c, elt, mid).total <= ws_bytes) lo = mid; else hi = mid;
+    if (plan_workspace(c, t, elt, mid).total <= ws_bytes) lo = mid; else hi = mid;
   }
   return lo;
 }
@@ -566,6 +574,57 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   return MOA_OK;
 }
 
+// One causal self-attention block over (a prefix cache, the row's drafted ancestors, itself) plus its MLP:
+// the drafter's SA block and every Target-Layer-Inference decoder layer have this shape (Section 3.1.2,
+// Section 3.2). On entry xn holds the block's normalised input and xres the residual stream; on exit the
+// MLP's down-projection is pending in `lo` (folded in by the next residual_norm).
+struct TreeAttnLayer {
+  const void *wq, *wk, *wv, *wo, *norm2, *wgate, *wup, *wdown;
+  int hq, hkv, mlp;
+  float theta;
+  const void *ck, *cv;     // prefix cache T [max_batch, max_ctx, hkv, dh]
+  void *tk, *tv;           // tree slots T [max_batch, NS, hkv, dh]
+};
+
+template <typename T>
+static moa_status tree_attn_layer(moa_ctx* ctx, moa_state* st, cudaStream_t s, char* ws, const Workspace& p, int R,
+                                  int rows_per_seq, int max_len, const int* row_anc, const TreeAttnLayer& a, LinOut* lo,
+                                  void* status_word) {
+  const moa_config& c = ctx->c;
+  const TreeLayout& L = ctx->tl;
+  const int step = st->step, B = c.tree_topk, D = c.tree_depth, E = c.d_model, dh = c.head_dim;
+  T* xn = (T*)(ws + p.xn);
+  T* narrow = (T*)(ws + p.narrow);
+  T* obuf = (T*)(ws + p.obuf);
+  // bf16 path: the queries stay in fp32 and are split into two bf16 terms by the attention kernel
+  float* q32 = sizeof(T) == 2 ? (float*)(ws + p.q32) : nullptr;
+  const int nq = a.hq * dh, nkv = a.hkv * dh;
+  {
+    const void* W3[3] = {a.wq, a.wk, a.wv};
+    const int N3[3] = {nq, nkv, nkv};
+    MOA_TRY(linear<T>(ctx, s, xn, R, E, 3, W3, N3, ws, p, lo, status_word));
+  }
+  RopeRows rr;
+  memset(&rr, 0, sizeof(rr));
+  rr.mode = 0;
+  rr.step = step;
+  rr.B = B;
+  rr.slots = L.NS;
+  launch_pdl(rope_store_kernel<T>, dim3(dim3(R, a.hq + 2 * a.hkv)), dim3(64), 0, s, lo->part, lo->splits, lo->plane, nq + 2 * nkv, 0, nq,
+             nq + nkv, a.hq, a.hkv, dh, a.theta, st->sa_len, rr, narrow, q32, (T*)a.tk, (T*)a.tv);
+  MOA_CHECK_LAUNCH();
+  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, a.hq, a.hkv, (const T*)a.ck, (const T*)a.cv, c.max_ctx, nkv,
+                       st->sa_len, 0, max_len, (const T*)a.tk, (const T*)a.tv, L.NS, row_anc, D, step + 1,
+                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
+  {
+    const void* W1[1] = {a.wo};
+    const int N1[1] = {E};
+    MOA_TRY(linear<T>(ctx, s, obuf, R, nq, 1, W1, N1, ws, p, lo, status_word));
+  }
+  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, lo, a.norm2, nullptr));
+  return mlp_block<T>(s, ctx, p, ws, R, E, a.mlp, a.wgate, a.wup, a.wdown, lo, status_word);
+}
+
 template <typename T>
 static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk_id, float* topk_logp,
                                void* hidden_out, char* ws, const Workspace& p, cudaStream_t s) {
@@ -582,50 +641,28 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   const int cur = step & 1;
   const int* row_tok = tp.row_tok + (size_t)cur * nbB;
   const int* row_anc = tp.row_anc + (size_t)cur * nbB * D;
-  T* tk = (T*)((char*)st->tree + L.tk);
-  T* tv = (T*)((char*)st->tree + L.tv);
   float* xres = (float*)(ws + p.xres);
   T* xn = (T*)(ws + p.xn);
   T* narrow = (T*)(ws + p.narrow);
   T* obuf = (T*)(ws + p.obuf);
-  // bf16 path: the queries of both attentions stay in fp32 and are split into two bf16 terms by the kernel
   float* q32 = sizeof(T) == 2 ? (float*)(ws + p.q32) : nullptr;
   LinOut lo;
-
-  // ---- self-attention block ----
-  launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn,
-             lo_rows_of(sizeof(T), R));
-  MOA_CHECK_LAUNCH();
-  const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh;
-  {
-    const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
-    const int N3[3] = {nq, nkv, nkv};
-    MOA_TRY(linear<T>(ctx, s, xn, R, E, 3, W3, N3, ws, p, &lo, status_word));
-  }
-  RopeRows rr;
-  memset(&rr, 0, sizeof(rr));
-  rr.mode = 0;
-  rr.step = step;
-  rr.B = B;
-  rr.slots = L.NS;
-  launch_pdl(rope_store_kernel<T>, dim3(dim3(R, c.sa_hq + 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq, nq + nkv, c.sa_hq, c.sa_hkv,
-                                         dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, tk, tv);
-  MOA_CHECK_LAUNCH();
   int max_sa = 0, max_ca = 0;
   for (int b = 0; b < batch; ++b) {
     max_sa = imax(max_sa, st->sa_len_host[b]);
     max_ca = imax(max_ca, st->ca_len_host[b]);
   }
-  MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, c.sa_hq, c.sa_hkv, (const T*)st->sa_k, (const T*)st->sa_v,
-                       c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
-                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
+
+  // ---- self-attention block ----
+  launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn,
+             lo_rows_of(sizeof(T), R));
+  MOA_CHECK_LAUNCH();
   {
-    const void* W1[1] = {w.sa_wo};
-    const int N1[1] = {E};
-    MOA_TRY(linear<T>(ctx, s, obuf, R, nq, 1, W1, N1, ws, p, &lo, status_word));
+    TreeAttnLayer a = {w.sa_wq, w.sa_wk, w.sa_wv, w.sa_wo, w.sa_norm2, w.sa_wgate, w.sa_wup, w.sa_wdown,
+                       c.sa_hq, c.sa_hkv, c.sa_mlp, c.sa_rope_theta, st->sa_k, st->sa_v,
+                       (char*)st->tree + L.tk, (char*)st->tree + L.tv};
+    MOA_TRY(tree_attn_layer<T>(ctx, st, s, ws, p, R, rows_per_seq, max_sa, row_anc, a, &lo, status_word));
   }
-  MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.sa_norm2, nullptr));
-  MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.sa_mlp, w.sa_wgate, w.sa_wup, w.sa_wdown, &lo, status_word));
 
   // ---- cross-attention block ----
   MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_normq, nullptr));
@@ -651,6 +688,16 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   }
   MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_norm2, nullptr));
   MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.ca_mlp, w.ca_wgate, w.ca_wup, w.ca_wdown, &lo, status_word));
+
+  // ---- Target Layer Inference: the last N decoder layers of the LLM on the drafted rows (Section 3.2) ----
+  for (int l = 0; l < ctx->tli.n_layers; ++l) {
+    const moa_tli_layer& t = ctx->tli_w[l];
+    MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, t.norm1, nullptr));
+    TreeAttnLayer a = {t.wq, t.wk, t.wv, t.wo, t.norm2, t.wgate, t.wup, t.wdown,
+                       ctx->tli.hq, ctx->tli.hkv, ctx->tli.mlp, ctx->tli.rope_theta, ctx->tli_c.k[l], ctx->tli_c.v[l],
+                       (char*)st->tree + L.tli_tk[l], (char*)st->tree + L.tli_tv[l]};
+    MOA_TRY(tree_attn_layer<T>(ctx, st, s, ws, p, R, rows_per_seq, max_sa, row_anc, a, &lo, status_word));
+  }
 
   // ---- LM head, log-softmax, top-B ----
   MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.final_norm, hidden_out));
@@ -1128,6 +1175,10 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
   ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
   ctx->last_n_ops = 0;
   ctx->fused_step = false;
+  ctx->n_wmap_base = 0;
+  memset(&ctx->tli, 0, sizeof(ctx->tli));
+  memset(ctx->tli_w, 0, sizeof(ctx->tli_w));
+  memset(&ctx->tli_c, 0, sizeof(ctx->tli_c));
   if (cfg->dtype == MOA_BF16) {
     // tensor maps of every weight matrix whose inner dimension the streaming GEMM can take
     void* fn = nullptr;
@@ -1164,8 +1215,65 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
       ++ctx->n_wmap;
     }
     ctx->fast = true;
+    ctx->n_wmap_base = ctx->n_wmap;
   }
   *out = ctx;
+  return MOA_OK;
+}
+
+moa_status moa_tli_configure(moa_ctx* ctx, const moa_tli_config* cfg, const moa_tli_layer* layers_host,
+                             const moa_tli_caches* caches) {
+  if (!ctx || !cfg) return MOA_ERR_NULL;
+  const moa_config& c = ctx->c;
+  const int n = cfg->n_layers;
+  if (n < 0 || n > MOA_MAX_TLI) return MOA_ERR_SHAPE;
+  if (n > 0) {
+    if (!layers_host || !caches) return MOA_ERR_NULL;
+    if (cfg->hq <= 0 || cfg->hkv <= 0 || cfg->hq % cfg->hkv != 0) return MOA_ERR_SHAPE;
+    if (cfg->mlp <= 0 || cfg->mlp % 16 != 0 || !(cfg->rope_theta >= 0.f)) return MOA_ERR_SHAPE;
+    for (int l = 0; l < n; ++l) {
+      const void* const* wp = (const void* const*)&layers_host[l];
+      for (size_t i = 0; i < sizeof(moa_tli_layer) / sizeof(void*); ++i) {
+        if (!wp[i]) return MOA_ERR_NULL;
+        if (!aligned16(wp[i])) return MOA_ERR_ALIGN;
+      }
+      if (!caches->k[l] || !caches->v[l]) return MOA_ERR_NULL;
+      if (!aligned16(caches->k[l]) || !aligned16(caches->v[l])) return MOA_ERR_ALIGN;
+    }
+  }
+  // tensor maps of the layers' matrices follow the drafter's own (bf16 path)
+  ctx->n_wmap = ctx->n_wmap_base;
+  if (n > 0 && ctx->fast) {
+    const int dh = c.head_dim, E = c.d_model;
+    for (int l = 0; l < n; ++l) {
+      const moa_tli_layer& t = layers_host[l];
+      struct { const void* p; int n, k; } mats[] = {
+          {t.wq, cfg->hq * dh, E}, {t.wk, cfg->hkv * dh, E}, {t.wv, cfg->hkv * dh, E}, {t.wo, E, cfg->hq * dh},
+          {t.wgate, cfg->mlp, E}, {t.wup, cfg->mlp, E}, {t.wdown, E, cfg->mlp}};
+      for (auto& m : mats) {
+        if (m.k % WS_BK != 0 || find_wmap(ctx, m.p)) continue;
+        if (ctx->n_wmap >= WMAP_MAX) return MOA_ERR_SHAPE;
+        WeightMap& wm = ctx->wmap[ctx->n_wmap];
+        wm.ptr = m.p;
+        wm.n = m.n;
+        wm.k = m.k;
+        if (!encode_map(ctx, &wm.tm, m.p, m.n, m.k, WS_BM)) {
+          ctx->n_wmap = ctx->n_wmap_base;
+          return MOA_ERR_CUDA;
+        }
+        ++ctx->n_wmap;
+      }
+    }
+  }
+  memset(&ctx->tli, 0, sizeof(ctx->tli));
+  memset(ctx->tli_w, 0, sizeof(ctx->tli_w));
+  memset(&ctx->tli_c, 0, sizeof(ctx->tli_c));
+  if (n > 0) {
+    ctx->tli = *cfg;
+    for (int l = 0; l < n; ++l) ctx->tli_w[l] = layers_host[l];
+    ctx->tli_c = *caches;
+  }
+  ctx->tl = make_tree_layout(c.max_batch, c.tree_topk, c.tree_depth, c.sa_hkv, c.head_dim, ctx->elt, n, n > 0 ? cfg->hkv : 0);
   return MOA_OK;
 }
 
@@ -1225,9 +1333,9 @@ moa_status moa_set_option(moa_ctx* ctx, int32_t option, int32_t value) {
 moa_status moa_profile_phases(moa_ctx* ctx, const void* ws, size_t ws_bytes, int32_t cap, double* us_out,
                               double* wait_us_out, int32_t* kind_out, int32_t* n_out, void* stream) {
   if (!ctx || !ws || !us_out || !kind_out || !n_out) return MOA_ERR_NULL;
-  const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
+  const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
-  const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
   unsigned long long t[2 * PM_MAX_OPS + 1];
   cudaError_t e = cudaMemcpyAsync(t, (const char*)ws + p.trace, sizeof(t), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
@@ -1249,7 +1357,7 @@ moa_status moa_state_bytes(const moa_ctx* ctx, int32_t lsa_chunk_tokens, size_t*
   if (!ctx) return MOA_ERR_NULL;
   if (lsa_chunk_tokens < 1) return MOA_ERR_SHAPE;
   if (tree_bytes) *tree_bytes = ctx->tl.total;
-  if (workspace_bytes) *workspace_bytes = plan_workspace(ctx->c, ctx->elt, lsa_chunk_tokens).total;
+  if (workspace_bytes) *workspace_bytes = plan_workspace(ctx->c, ctx->tli, ctx->elt, lsa_chunk_tokens).total;
   return MOA_OK;
 }
 
@@ -1307,9 +1415,9 @@ moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, con
   if (!aligned16(h_stack) || !aligned16(kv_out) || !aligned16(ws)) return MOA_ERR_ALIGN;
   for (int b = 0; b < batch; ++b)
     if ((long long)st->ca_len_host[b] + n_tok_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
-  const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
+  const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
-  const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
   moa_status r;
   // Passes with more than 256 (token, layer) rows run as one persistent kernel with tensor-core GEMMs whose
   // epilogues are fused (dense regime); smaller ones take the weight-streaming kernels launch by launch.
@@ -1347,9 +1455,9 @@ moa_status moa_sa_append(moa_ctx* ctx, moa_state* st, const int32_t* tok, const 
   if (!aligned16(ws)) return MOA_ERR_ALIGN;
   for (int b = 0; b < batch; ++b)
     if ((long long)st->sa_len_host[b] + n_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
-  const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
+  const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
-  const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
   moa_status r = ctx->c.dtype == MOA_F32 ? sa_append_t<float>(ctx, st, tok, split, (char*)ws, p, (cudaStream_t)stream)
                                          : sa_append_t<bf16>(ctx, st, tok, split, (char*)ws, p, (cudaStream_t)stream);
   if (r == MOA_OK)
@@ -1376,13 +1484,13 @@ moa_status moa_draft_step(moa_ctx* ctx, moa_state* st, int32_t batch, int32_t* t
   if (!topk_id || !topk_logp || !ws) return MOA_ERR_NULL;
   if (!aligned16(topk_id) || !aligned16(topk_logp) || !aligned16(hidden_out) || !aligned16(ws)) return MOA_ERR_ALIGN;
   if (st->step < 0 || st->step >= ctx->c.tree_depth) return MOA_ERR_STATE;
-  const int chunk = chunk_from_bytes(ctx->c, ctx->elt, ws_bytes);
+  const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
-  const Workspace p = plan_workspace(ctx->c, ctx->elt, chunk);
+  const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
   // The single-kernel forward exists and is parity-tested, but with few rows the chain of separate launches is
   // the faster of the two on B200 as measured (421 us against 620 us per forward at the Llama-3-8B shape), so the
   // fused kernel is taken only on request.
-  if (ctx->fused_step && pm_usable(ctx))
+  if (ctx->fused_step && ctx->tli.n_layers == 0 && pm_usable(ctx))
     return draft_step_pm(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream);
   return ctx->c.dtype == MOA_F32
              ? draft_step_t<float>(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream)

@@ -18,10 +18,13 @@ struct TreeLayout {
   size_t pool_tok, pool_parent, pool_depth;   // int[nb*P]
   size_t pool_score;       // float[nb*P]
   size_t tk, tv;           // T[nb][NS][hkv][dh]
+  int n_tli;               // decoder layers of the LLM run on the drafted rows (Section 3.2), 0..4
+  size_t tli_tk[4], tli_tv[4];   // per such layer T[nb][NS][tli_hkv][dh]: the drafted rows' keys / values in it
   size_t total;
 };
 
-__host__ inline TreeLayout make_tree_layout(int nb, int B, int D, int hkv, int dh, size_t elt) {
+__host__ inline TreeLayout make_tree_layout(int nb, int B, int D, int hkv, int dh, size_t elt, int n_tli = 0,
+                                            int tli_hkv = 0) {
   TreeLayout L;
   L.nb = nb; L.B = B; L.D = D;
   L.P = B + (D - 1) * B * B;
@@ -40,6 +43,14 @@ __host__ inline TreeLayout make_tree_layout(int nb, int B, int D, int hkv, int d
   L.pool_score = take((size_t)nb * L.P * sizeof(float));
   L.tk = take((size_t)nb * L.NS * hkv * dh * elt);
   L.tv = take((size_t)nb * L.NS * hkv * dh * elt);
+  L.n_tli = n_tli;
+  for (int l = 0; l < 4; ++l) {
+    L.tli_tk[l] = L.tli_tv[l] = 0;
+    if (l < n_tli) {
+      L.tli_tk[l] = take((size_t)nb * L.NS * tli_hkv * dh * elt);
+      L.tli_tv[l] = take((size_t)nb * L.NS * tli_hkv * dh * elt);
+    }
+  }
   L.total = o;
   return L;
 }

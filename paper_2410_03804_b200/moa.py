@@ -19,7 +19,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
                 "ERR_STATE", "ERR_ARCH", "ERR_CUDA", "ERR_TIMEOUT"]
 MOA_OK = 0
 
-EXPORTS = ["moa_create", "moa_destroy", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
+EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
@@ -42,6 +42,23 @@ WEIGHT_FIELDS = ["embed", "lm_head", "final_norm",
 
 class MoaWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in WEIGHT_FIELDS]
+
+
+MOA_MAX_TLI = 4
+TLI_LAYER_FIELDS = ["norm1", "wq", "wk", "wv", "wo", "norm2", "wgate", "wup", "wdown"]
+
+
+class MoaTliConfig(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("hq", C.c_int32), ("hkv", C.c_int32), ("mlp", C.c_int32),
+                ("rope_theta", C.c_float)]
+
+
+class MoaTliLayer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in TLI_LAYER_FIELDS]
+
+
+class MoaTliCaches(C.Structure):
+    _fields_ = [("k", C.c_void_p * MOA_MAX_TLI), ("v", C.c_void_p * MOA_MAX_TLI)]
 
 
 class MoaState(C.Structure):
@@ -85,6 +102,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_status_str.restype = C.c_char_p
     lib.moa_last_cuda_error.argtypes = []
     lib.moa_last_cuda_error.restype = C.c_char_p
+    lib.moa_tli_configure.argtypes = [vp, C.POINTER(MoaTliConfig), vp, C.POINTER(MoaTliCaches)]
     lib.moa_state_set_len.argtypes = [vp, C.POINTER(MoaState), i32, vp, i32, vp]
     lib.moa_lsa_forward.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, vp, sz, vp]
     lib.moa_sa_append.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, sz, vp]
@@ -145,7 +163,9 @@ class MoA:
     """A drafter context plus one decoding state on the current CUDA device.
 
     weights: dict name -> CUDA tensor (dtype float32 or bfloat16, as cfg['dtype'] says).
-    cfg keys: the fields of moa_config except dtype/max_* (given separately)."""
+    cfg keys: the fields of moa_config except dtype/max_* (given separately). Target Layer Inference: with
+    cfg['n_tli'] = N > 0 (plus 'tli_hq', 'tli_hkv', 'tli_mlp') the weights also hold 'tli{l}_{norm1,wq,...}' for
+    l < N, and the LLM's caches of those layers are the tensors tli_k[l], tli_v[l] (fill_tli_cache)."""
 
     def __init__(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int, lsa_chunk_tokens: int = 8,
                  fused_step: bool = False):
@@ -176,6 +196,10 @@ class MoA:
         if fused_step:
             _check(self.lib.moa_set_option(self.h, 1, 1), "moa_set_option")
         self.device = weights["embed"].device
+        self.n_tli = int(cfg.get("n_tli", 0))
+        self.tli_k, self.tli_v = [], []
+        if self.n_tli > 0:
+            self.moa_tli_configure(cfg, weights, max_batch, max_ctx)
         tb, wb = C.c_size_t(), C.c_size_t()
         _check(self.lib.moa_state_bytes(self.h, int(lsa_chunk_tokens), C.byref(tb), C.byref(wb)), "moa_state_bytes")
         self.tree_bytes, self.ws_bytes = tb.value, wb.value
@@ -210,6 +234,27 @@ class MoA:
             pass
 
     # ---- the C-ABI calls, same names -------------------------------------------------------
+    def moa_tli_configure(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int):
+        """Turns Target Layer Inference on: binds the N decoder layers' weights and allocates their caches."""
+        n = int(cfg["n_tli"])
+        tc = MoaTliConfig(n, int(cfg["tli_hq"]), int(cfg["tli_hkv"]), int(cfg["tli_mlp"]),
+                          float(cfg.get("rope_theta", 500000.0)))
+        layers = (MoaTliLayer * n)()
+        for l in range(n):
+            for f in TLI_LAYER_FIELDS:
+                t = weights[f"tli{l}_{f}"]
+                assert t.is_cuda and t.dtype == self.dtype and t.is_contiguous(), (l, f)
+                self.weights[f"tli{l}_{f}"] = t
+                setattr(layers[l], f, t.data_ptr())
+        caches = MoaTliCaches()
+        shape = (max_batch, max_ctx, tc.hkv, self.cfg.head_dim)
+        self.tli_k = [torch.zeros(shape, dtype=self.dtype, device=self.device) for _ in range(n)]
+        self.tli_v = [torch.zeros(shape, dtype=self.dtype, device=self.device) for _ in range(n)]
+        for l in range(n):
+            caches.k[l], caches.v[l] = self.tli_k[l].data_ptr(), self.tli_v[l].data_ptr()
+        _check(self.lib.moa_tli_configure(self.h, C.byref(tc), C.cast(layers, C.c_void_p), C.byref(caches)),
+               "moa_tli_configure")
+
     def moa_state_set_len(self, which: str, lens, stream=None):
         lens = [int(v) for v in lens]
         _check(self.lib.moa_state_set_len(self.h, C.byref(self.st), 0 if which == "ca" else 1, _host_i32(lens),
@@ -316,3 +361,10 @@ class MoA:
         ck[:b, :n].copy_(k)
         cv[:b, :n].copy_(v)
         self.moa_state_set_len(which, [n] * b)
+
+    def fill_tli_cache(self, layer: int, k: torch.Tensor, v: torch.Tensor):
+        """Copies the LLM's cache of one Target-Layer-Inference layer [batch, n, hkv, dh] in (positions 0..n-1;
+        the valid length is the self-attention prefix length)."""
+        b, n = k.shape[0], k.shape[1]
+        self.tli_k[layer][:b, :n].copy_(k)
+        self.tli_v[layer][:b, :n].copy_(v)

@@ -51,6 +51,11 @@ class Preset:
     stack_std_ramp: bool  # std of stacked activation l is 0.5 + l/16 instead of 1
     rms_eps: float = 1e-5
     rope_theta: float = 500000.0
+    # Target Layer Inference (Section 3.2): the last n_tli decoder layers of the LLM run on the drafted rows
+    n_tli: int = 0
+    tli_hq: int = 0
+    tli_hkv: int = 0
+    tli_mlp: int = 0
 
     @property
     def torch_dtype(self) -> torch.dtype:
@@ -136,6 +141,41 @@ def make_weights(p: Preset, only=None) -> dict:
         w = _randn(p, 100 + i, shape, std=0.02, mean=1.0 if is_gain else 0.0)
         out[name] = w.to(p.torch_dtype)
     return out
+
+
+TLI_LAYER_NAMES = ["norm1", "wq", "wk", "wv", "wo", "norm2", "wgate", "wup", "wdown"]
+
+
+def tli_weight_shapes(p: Preset) -> dict:
+    """Shapes of the n_tli LLM decoder layers' weights, named tli{l}_{name}, l = 0 the earliest layer."""
+    E, dh = p.d_model, p.head_dim
+    one = {"norm1": (E,), "wq": (p.tli_hq * dh, E), "wk": (p.tli_hkv * dh, E), "wv": (p.tli_hkv * dh, E),
+           "wo": (E, p.tli_hq * dh), "norm2": (E,), "wgate": (p.tli_mlp, E), "wup": (p.tli_mlp, E),
+           "wdown": (E, p.tli_mlp)}
+    return {f"tli{l}_{n}": one[n] for l in range(p.n_tli) for n in TLI_LAYER_NAMES}
+
+
+def make_tli_weights(p: Preset) -> dict:
+    """Random decoder-layer weights with the distributions of make_weights (tensor indices 200 + ...)."""
+    out = {}
+    for i, (name, shape) in enumerate(tli_weight_shapes(p).items()):
+        is_gain = len(shape) == 1
+        out[name] = _randn(p, 200 + i, shape, std=0.02, mean=1.0 if is_gain else 0.0).to(p.torch_dtype)
+    return out
+
+
+def make_tli_cache(p: Preset, layer: int, ctx: int | None = None) -> tuple[torch.Tensor, torch.Tensor]:
+    """Synthetic LLM K and V cache of one Target-Layer-Inference layer [batch, ctx, tli_hkv, dh] ~ N(0,1)
+    (keys treated as already rotated; the cache_outliers rule of make_cache applies)."""
+    ctx = p.ctx if ctx is None else ctx
+    outs = []
+    for j in range(2):
+        x = _randn(p, 300 + 10 * layer + j, (p.batch, ctx, p.tli_hkv * p.head_dim))
+        if p.cache_outliers:
+            ch = _outlier_channels(p, 305 + 10 * layer + j, p.tli_hkv * p.head_dim)
+            x[:, :, ch] *= 20.0
+        outs.append(x.view(p.batch, ctx, p.tli_hkv, p.head_dim).to(p.torch_dtype))
+    return outs[0], outs[1]
 
 
 def _outlier_channels(p: Preset, tensor_index: int, width: int) -> torch.Tensor:

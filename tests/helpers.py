@@ -7,7 +7,7 @@ from paper_2410_03804_b200 import synth
 
 CFG_KEYS = ("d_model", "n_stack", "d_stack", "vocab", "head_dim", "lsa_hq", "lsa_hkv", "lsa_mlp", "sa_hq", "sa_hkv",
             "sa_mlp", "ca_hq", "ca_hkv", "ca_mlp", "tree_topk", "tree_depth", "tree_keep", "rms_eps", "rope_theta",
-            "dtype")
+            "dtype", "n_tli", "tli_hq", "tli_hkv", "tli_mlp")
 
 
 def cfg_of(p: synth.Preset) -> dict:

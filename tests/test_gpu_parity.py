@@ -19,7 +19,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def oracle_cycle(p, dr, h_stack, prompt, root, ca_cache, sa_cache, forced=None, seqs=None):
+def oracle_cycle(p, dr, h_stack, prompt, root, ca_cache, sa_cache, forced=None, seqs=None, tli_cache=None):
     """The oracle's side of one drafting cycle, for the sequences listed in seqs (default: all).
     forced[b] = per-step (ids, logp) to expand with. Per-sequence results are dicts keyed by b."""
     nb = p.batch
@@ -38,11 +38,13 @@ def oracle_cycle(p, dr, h_stack, prompt, root, ca_cache, sa_cache, forced=None, 
             out["saK"][b], out["saV"][b] = H.np32(sa_cache[0][b]), H.np32(sa_cache[1][b])
         out["trees"][b] = O.draft_tree(dr, int(root[b]), out["saK"][b], out["saV"][b], out["caK"][b], out["caV"][b],
                                        p.tree_topk, p.tree_depth, p.tree_keep,
-                                       forced=None if forced is None else forced[b])
+                                       forced=None if forced is None else forced[b],
+                                       tliK=None if tli_cache is None else [H.np32(k[b]) for k, _ in tli_cache],
+                                       tliV=None if tli_cache is None else [H.np32(v[b]) for _, v in tli_cache])
     return out
 
 
-def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None, seqs=None):
+def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None, seqs=None, tli_cache=None):
     """One drafting cycle on both sides. The tree follows the deciding oracle's top-B (teacher forcing);
     values are compared with the unrounded oracle walking the same tree. With seqs given, the oracle runs
     only on those sequences of the batch (sampled outputs); the others expand with the GPU's own lists."""
@@ -51,9 +53,10 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
     nb = p.batch
     B, D = p.tree_topk, p.tree_depth
     seqs = list(range(nb)) if seqs is None else list(seqs)
-    od = oracle_cycle(p, dec, h_stack, prompt, root, ca_cache, sa_cache, seqs=seqs)
+    od = oracle_cycle(p, dec, h_stack, prompt, root, ca_cache, sa_cache, seqs=seqs, tli_cache=tli_cache)
     forced = {b: [([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in od["trees"][b][1]] for b in seqs}
-    ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced, seqs=seqs)
+    ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced, seqs=seqs,
+                                              tli_cache=tli_cache)
     stats = dict(rows=0, exact=0, worst_hidden=0.0, worst_logp=0.0)
     if ca_cache is None:
         n_tok = [h_stack.shape[0] // nb] * nb
@@ -79,6 +82,8 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
         assert g.sa_len[:nb].tolist() == [n] * nb
     else:
         g.fill_cache("sa", sa_cache[0].cuda(), sa_cache[1].cuda())
+    for l, (k, v) in enumerate(tli_cache or []):
+        g.fill_tli_cache(l, k.cuda(), v.cuda())
     g.moa_tree_begin(root.cuda())
     outs = None
     for s in range(D):
@@ -173,6 +178,33 @@ def test_reduced_llama_shape(dtype, batch, fused):
     stats = run_cycle(p, g, H.make_oracles(p, w), synth.make_h_stack(p, p.lsa_tokens * batch),
                       synth.make_tokens(p, p.ctx), synth.make_root(p))
     assert stats["rows"] == batch * (1 + 2 * 5)
+
+
+@pytest.mark.parametrize("dtype,batch,n_tli", [("bf16", 2, 2), ("f32", 2, 1), ("bf16", 1, 4)])
+def test_target_layer_inference_reduced_llama_shape(dtype, batch, n_tli):
+    """Target Layer Inference (Section 3.2): the last n_tli LLM decoder layers (Llama-3-8B head layout, reduced
+    widths) run on the drafted rows over synthetic LLM caches of those layers plus the drafted ancestors."""
+    p = synth.scaled(synth.PRESETS["c2"], d_model=512, d_stack=512, n_stack=6, vocab=4099, lsa_hq=4, lsa_hkv=2, lsa_mlp=768,
+                     sa_hq=4, sa_hkv=2, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=896, ctx=150, batch=batch, tree_topk=4,
+                     tree_depth=4, tree_keep=20, dtype=dtype, lsa_tokens=7, n_tli=n_tli, tli_hq=8, tli_hkv=2,
+                     tli_mlp=1408)
+    w = synth.make_weights(p)
+    w.update(synth.make_tli_weights(p))
+    g = H.make_gpu(p, w, max_ctx=p.ctx + 16, lsa_chunk_tokens=16)
+    tli_cache = [synth.make_tli_cache(p, l) for l in range(n_tli)]
+    stats = run_cycle(p, g, H.make_oracles(p, w), synth.make_h_stack(p, p.lsa_tokens * batch),
+                      synth.make_tokens(p, p.ctx), synth.make_root(p), tli_cache=tli_cache)
+    assert stats["rows"] == batch * (1 + 3 * 4)
+    # the layers are really in the path: without them the drafter's output differs
+    g0 = H.make_gpu(synth.scaled(p, n_tli=0), synth.make_weights(p), max_ctx=p.ctx + 16, lsa_chunk_tokens=16)
+    g0.moa_sa_append(synth.make_tokens(p, p.ctx).reshape(-1).cuda(), [p.ctx] * batch)
+    g0.moa_lsa_forward(synth.make_h_stack(p, p.lsa_tokens * batch).cuda(), [p.lsa_tokens] * batch)
+    g0.moa_tree_begin(synth.make_root(p).cuda())
+    _, _, h0 = g0.moa_draft_step(want_hidden=True)
+    g.moa_tree_begin(synth.make_root(p).cuda())
+    _, _, h1 = g.moa_draft_step(want_hidden=True)
+    torch.cuda.synchronize()
+    assert not torch.allclose(h0.float(), h1.float(), rtol=0, atol=1e-2 * float(h0.float().abs().max()))
 
 
 def test_maximum_rows_per_step_256():
