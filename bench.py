@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 CFG_KEYS = ("d_model", "n_stack", "d_stack", "vocab", "head_dim", "lsa_hq", "lsa_hkv", "lsa_mlp", "sa_hq", "sa_hkv",
             "sa_mlp", "ca_hq", "ca_hkv", "ca_mlp", "tree_topk", "tree_depth", "tree_keep", "rms_eps", "rope_theta",
-            "dtype")
+            "dtype", "n_tli", "tli_hq", "tli_hkv", "tli_mlp")
 
 
 def algorithmic_bytes(p) -> dict:
@@ -38,10 +38,13 @@ def algorithmic_bytes(p) -> dict:
     ca_w = p.ca_hq * dh * E + E * p.ca_hq * dh + 3 * E * p.ca_mlp
     lm = p.vocab * E
     caches = p.batch * p.ctx * 2 * (p.sa_hkv + p.ca_hkv) * dh
+    # Target Layer Inference: each LLM decoder layer's weights and its cache, once per forward
+    tli = p.n_tli * ((p.tli_hq + 2 * p.tli_hkv) * dh * E + E * p.tli_hq * dh + 3 * E * p.tli_mlp
+                     + p.batch * p.ctx * 2 * p.tli_hkv * dh)
     lsa_w = ((p.lsa_hq + 2 * p.lsa_hkv) * dh * p.d_stack + p.d_stack * p.lsa_hq * dh + 3 * p.d_stack * p.lsa_mlp
              + 2 * p.ca_hkv * dh * p.d_stack)
     lsa_in = p.batch * p.lsa_tokens * p.n_stack * p.d_stack
-    return dict(step=(sa_w + ca_w + lm + caches) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
+    return dict(step=(sa_w + ca_w + lm + caches + tli) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (wstream_gemm_kernel<16>, mode 1) from the ncu
@@ -119,6 +122,7 @@ class OracleSampler:
         self.p, self.np, self.synth = p, np, synth
         self.cores = torch.get_num_threads()
         w = synth.make_weights(p)
+        w.update(synth.make_tli_weights(p))
         cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
         self.dr = O.Drafter(cfg, {k: v.float().numpy() for k, v in w.items()})
         for name in w:
@@ -128,6 +132,8 @@ class OracleSampler:
         caK, caV = synth.make_cache(one, "ca", self.ctx)
         saK, saV = synth.make_cache(one, "sa", self.ctx)
         self.caches = [t[0].float().numpy().astype(np.float64) for t in (caK, caV, saK, saV)]
+        self.tli = [tuple(t[0].float().numpy().astype(np.float64) for t in synth.make_tli_cache(one, l, self.ctx))
+                    for l in range(p.n_tli)]
 
     def sample(self, rows: int = 2, lsa_tok: int = 1):
         """Returns (cycle_seconds_estimate, cores, description)."""
@@ -140,7 +146,7 @@ class OracleSampler:
         toks = synth.make_root(synth.scaled(p, batch=rows)).tolist()
         t0 = time.perf_counter()
         for t in toks:
-            self.dr.forward_row(t, self.ctx, saK, saV, caK, caV, p.tree_topk)
+            self.dr.forward_row(t, self.ctx, saK, saV, caK, caV, p.tree_topk, self.tli)
         t_row = (time.perf_counter() - t0) / rows
         n_rows = p.batch * (1 + p.tree_topk * (p.tree_depth - 1))
         cycle = p.batch * p.lsa_tokens * t_lsa + n_rows * t_row
@@ -176,7 +182,7 @@ def run_reference(args, p):
 def workload_config(p):
     return {"workload": f"{p.name}: Llama-3-shaped MoA drafter, one drafting cycle = LSA on {p.lsa_tokens} tokens/seq + "
                         f"SA append + {p.tree_depth} drafter forwards (tree top-{p.tree_topk}, keep {p.tree_keep}) + mask",
-            "batch": p.batch, "context": p.ctx, "d_model": p.d_model, "vocab": p.vocab, "n_stack": p.n_stack,
+            "tli": p.n_tli, "batch": p.batch, "context": p.ctx, "d_model": p.d_model, "vocab": p.vocab, "n_stack": p.n_stack,
             "l2": "inputs larger than L2 (weights streamed per step exceed 126 MB)" if p.name != "c1" else "L2-resident"}
 
 
@@ -289,12 +295,17 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch every cycle on the stream instead of replaying a CUDA graph")
     ap.add_argument("--fused-step", action="store_true",
                     help="every forward as one persistent kernel (MOA_OPT_FUSED_STEP); implies --no-graph")
+    ap.add_argument("--tli", type=int, default=0,
+                    help="Target Layer Inference: run the last N Llama-shaped decoder layers in every forward (default 0, "
+                         "the headline configuration)")
     ap.add_argument("--phases", action="store_true", help="with --fused-step or --workload c3: print per-phase times to stderr")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     from paper_2410_03804_b200 import synth
     p = synth.PRESETS[args.workload]
+    if args.tli > 0:          # the LLM's own layer shape: the drafter's SA head layout, MLP 3.5 x E
+        p = synth.scaled(p, n_tli=args.tli, tli_hq=p.sa_hq, tli_hkv=p.sa_hkv, tli_mlp=p.d_model * 7 // 2)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -321,6 +332,7 @@ def main():
         args.no_graph = True
     # Replicas only: the path does not shard (one sequence batch per GPU, no data-path collective).
     w = {k: v.to(dev) for k, v in synth.make_weights(p).items()}
+    w.update({k: v.to(dev) for k, v in synth.make_tli_weights(p).items()})
     cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
     max_ctx = p.ctx + 64
     g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens, fused_step=args.fused_step)
@@ -328,6 +340,9 @@ def main():
     saK, saV = synth.make_cache(p, "sa")
     g.fill_cache("ca", caK.to(dev), caV.to(dev))
     g.fill_cache("sa", saK.to(dev), saV.to(dev))
+    for l in range(p.n_tli):
+        tk, tv = synth.make_tli_cache(p, l)
+        g.fill_tli_cache(l, tk.to(dev), tv.to(dev))
     del caK, caV, saK, saV
     nb, A, D, B, m = p.batch, p.lsa_tokens, p.tree_depth, p.tree_topk, p.tree_keep
     h_host = synth.make_h_stack(p, nb * A).pin_memory()

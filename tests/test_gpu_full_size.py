@@ -26,7 +26,7 @@ def llama8b():
     g.close()
 
 
-def _given_caches_cycle(p, g, oracles, seqs=None):
+def _given_caches_cycle(p, g, oracles, seqs=None, tli_cache=None):
     """LSA on the cycle's new tokens (checked against the oracle on sampled sequences), then a teacher-forced
     tree over the synthetic caches."""
     tol = H.tol_of(p)
@@ -35,7 +35,8 @@ def _given_caches_cycle(p, g, oracles, seqs=None):
     seqs = list(range(nb)) if seqs is None else seqs
     caK, caV = synth.make_cache(p, "ca")
     saK, saV = synth.make_cache(p, "sa")
-    stats = run_cycle(p, g, oracles, None, None, synth.make_root(p), ca_cache=(caK, caV), sa_cache=(saK, saV), seqs=seqs)
+    stats = run_cycle(p, g, oracles, None, None, synth.make_root(p), ca_cache=(caK, caV), sa_cache=(saK, saV), seqs=seqs,
+                      tli_cache=tli_cache)
     # the cycle's LSA step on top of the filled cache: appended CA rows against the oracle
     h = synth.make_h_stack(p, nb * A)
     kv = g.moa_lsa_forward(h.cuda(), [A] * nb)
@@ -68,6 +69,18 @@ def test_c2_llama8b_fused_single_kernel_forward():
     w = synth.make_weights(p)
     g = H.make_gpu(p, w, max_ctx=p.ctx + 64, lsa_chunk_tokens=p.lsa_tokens, fused_step=True)
     stats = _given_caches_cycle(p, g, H.make_oracles(p, w))
+    assert stats["rows"] == 1 + 5 * 10
+    g.close()
+
+
+def test_c2_llama8b_target_layer_inference_one_layer():
+    """Config 2 with Target Layer Inference N = 1 (Section 3.2): one full-size Llama-3-8B decoder layer (32/8
+    heads x 128, MLP 14336) over a 2048-entry synthetic LLM cache runs on every drafted row; all 51 rows checked."""
+    p = synth.scaled(synth.PRESETS["c2"], n_tli=1, tli_hq=32, tli_hkv=8, tli_mlp=14336)
+    w = synth.make_weights(p)
+    w.update(synth.make_tli_weights(p))
+    g = H.make_gpu(p, w, max_ctx=p.ctx + 64, lsa_chunk_tokens=p.lsa_tokens)
+    stats = _given_caches_cycle(p, g, H.make_oracles(p, w), tli_cache=[synth.make_tli_cache(p, 0)])
     assert stats["rows"] == 1 + 5 * 10
     g.close()
 
