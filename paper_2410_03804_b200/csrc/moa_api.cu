@@ -62,7 +62,7 @@ struct moa_ctx {
 // workspace carving (same arithmetic in moa_state_bytes and in the calls)
 // ---------------------------------------------------------------------------------------------
 struct Workspace {
-  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, kvf, kvn, att_o, att_ml, q32, trace, total;
+  size_t xres, xn, part, narrow, obuf, logits, pmax, psum, cval, cid, mrg_ms, mrg_val, mrg_id, kvf, kvn, att_o, att_ml, q32, trace, total;
   int rows_cap, draft_rows, chunk_tok, part_rows, wide;
   long long att_units;   // (row, head, part) triples the split-attention partial buffers hold
 };
@@ -100,6 +100,9 @@ static Workspace plan_workspace(const moa_config& c, const moa_tli_config& t, si
   p.psum = take(n_sub * p.draft_rows * sizeof(float));
   p.cval = take(n_sub * p.draft_rows * c.tree_topk * sizeof(float));
   p.cid = take(n_sub * p.draft_rows * c.tree_topk * sizeof(int));
+  p.mrg_ms = take((size_t)p.draft_rows * MERGE_MAXCHUNKS * 2 * sizeof(float));     // LM-head merge, level-1 results
+  p.mrg_val = take((size_t)p.draft_rows * MERGE_MAXCHUNKS * MERGE_MAXB * sizeof(float));
+  p.mrg_id = take((size_t)p.draft_rows * MERGE_MAXCHUNKS * MERGE_MAXB * sizeof(int));
   p.kvf = take((size_t)chunk_tok * c.d_stack * sizeof(float));   // LSA output rows, fp32
   p.kvn = take(((size_t)chunk_tok + xpad) * c.d_stack * elt);    // their normalised copy, T
   const int gmax = imax(imax(c.sa_hq / c.sa_hkv, c.ca_hq / c.ca_hkv), tli ? t.hq / t.hkv : 0);
@@ -532,7 +535,7 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   const bool timed = ctx->prof_on && ctx->prof_n < PROF_MAX;
   if (sizeof(T) == 2) {
     if (R > 256 || !fast_shape(ctx, E, 1, W1)) return MOA_ERR_SHAPE;   // validated at moa_create
-    if (4 * ((V + WS_BM - 1) / WS_BM) > MERGE_OWN * MERGE_THREADS) return MOA_ERR_SHAPE;
+    if (4 * ((V + WS_BM - 1) / WS_BM) > MERGE_CHUNK * MERGE_MAXCHUNKS) return MOA_ERR_SHAPE;
     WsParams P;
     memset(&P, 0, sizeof(P));
     P.n_seg = 1;
@@ -556,8 +559,14 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
     MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count)));
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
-    launch_pdl(lm_merge_kernel, dim3(R), dim3(MERGE_THREADS), 0, s, P.p_max, P.p_sum, P.c_val, P.c_id, 4 * P.tiles_total, R, B, topk_id,
-                                                topk_logp);
+    MergeScratch sc;
+    sc.ms = (float*)(ws + p.mrg_ms);
+    sc.val = (float*)(ws + p.mrg_val);
+    sc.id = (int*)(ws + p.mrg_id);
+    sc.count = (int*)status_word + TREE_STATUS_WORDS;      // per-row arrival counters behind the status words
+    const int n_sub = 4 * P.tiles_total;
+    launch_pdl(lm_merge_kernel, dim3((n_sub + MERGE_CHUNK - 1) / MERGE_CHUNK, R), dim3(MERGE_THREADS), 0, s, P.p_max, P.p_sum,
+               P.c_val, P.c_id, n_sub, R, B, sc, topk_id, topk_logp);
     MOA_CHECK_LAUNCH();
     return MOA_OK;
   }

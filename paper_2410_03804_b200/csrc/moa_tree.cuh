@@ -6,10 +6,14 @@
 
 namespace moa {
 
+constexpr int TREE_STATUS_WORDS = 8;      // status word, barrier words of the fused kernels
+constexpr int TREE_ROW_COUNTERS = 256;    // per draft-row arrival counters of the LM-head merge (zero between launches)
+
 // Byte offsets inside the caller-owned tree blob.
 struct TreeLayout {
   int nb, B, D, P, NS;     // sequences, breadth, depth, pool size per sequence, tree K/V slots per sequence
-  size_t status;           // int[8]: [0] status word, [4..6] grid-barrier counter, abort word, exit counter
+  size_t status;           // int[8 + 256]: [0] status word, [4..6] grid-barrier counter, abort word, exit counter,
+                           // [8..] the LM-head merge's per-row arrival counters
   size_t flags;            // int[256 * 32]: per-CTA grid-barrier flags of the fused kernels, one 128-byte line each
   size_t root_tok;         // int[nb]
   size_t frontier;         // int[nb*B]        pool index of each frontier node (-1: the root)
@@ -31,7 +35,7 @@ __host__ inline TreeLayout make_tree_layout(int nb, int B, int D, int hkv, int d
   L.NS = 1 + B * (D - 1);
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
-  L.status = take(8 * sizeof(int));
+  L.status = take((TREE_STATUS_WORDS + TREE_ROW_COUNTERS) * sizeof(int));
   L.flags = take((size_t)256 * 32 * sizeof(int));
   L.root_tok = take((size_t)nb * sizeof(int));
   L.frontier = take((size_t)nb * B * sizeof(int));

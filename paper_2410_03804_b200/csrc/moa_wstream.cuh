@@ -404,20 +404,28 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 }
 
 // ---------------------------------------------------------------------------------------------
-// LM-head merge: one block per activation row combines the per-slice partials into logsumexp and
-// the global top-B, ordered by (log-probability descending, id ascending). Built for few dependent
-// memory round trips (the kernel is latency-bound):
-//   1. every thread loads (max, sum exp, best value, best id) of the <= MERGE_OWN slices it owns, coalesced;
-//   2. logsumexp from the (max, sum exp) pairs;
-//   3. threshold = the B-th best slice head (each slice list is sorted, so its head is its best): B rounds
-//      of "best ranking strictly after the previous pick", per warp over registers, then over the warp lists;
-//   4. only slices whose head ranks at or before the threshold can contribute (at most B of them): their
-//      owners load the whole B-entry list at once and keep what passes the threshold (at most B*B survivors);
-//   5. the survivors are ranked by counting.
+// LM-head merge: combines the per-slice partials of one activation row into logsumexp and the global top-B,
+// ordered by (log-probability descending, id ascending). The kernel is latency-bound (a few MB, many
+// dependent steps), so a row is spread over several CTAs and the steps are kept few:
+//   level 1, CTA (chunk, row): MERGE_CHUNK slices of the row.
+//     1. every thread loads (max, sum exp, best value, best id) of the <= MERGE_OWN slices it owns;
+//     2. the chunk's (max, sum exp);
+//     3. threshold = the B-th best slice head of the chunk (each slice list is sorted, so its head is its
+//        best): B rounds of "best ranking strictly after the previous pick", per warp over registers, then
+//        over the warp lists;
+//     4. only slices whose head ranks at or before the threshold can contribute (at most B of them): their
+//        owners load the whole B-entry list and keep what passes the threshold (at most B*B survivors),
+//        which are ranked by counting: the chunk's sorted top-B goes to global scratch;
+//   level 2, the LAST CTA of the row to finish (one atomic arrival per CTA on the row's counter, which the
+//     last one sets back to zero): logsumexp over the chunks, rank by counting over the chunks' B entries each.
+// The global top-B is a subset of the union of the chunks' top-B lists, so the result is exact.
 // ---------------------------------------------------------------------------------------------
-constexpr int MERGE_THREADS = 1024;
+constexpr int MERGE_THREADS = 256;
 constexpr int MERGE_MAXB = 16;
-constexpr int MERGE_OWN = 8;          // slices per thread: up to 8192 slices = 262144 vocabulary rows
+constexpr int MERGE_OWN = 2;                                // slices per thread
+constexpr int MERGE_CHUNK = MERGE_THREADS * MERGE_OWN;      // slices per CTA
+constexpr int MERGE_MAXCHUNKS = 16;                         // up to 8192 slices = 262144 vocabulary rows
+constexpr int MERGE_WARPS = MERGE_THREADS / 32;
 
 __device__ __forceinline__ void warp_best(float& bv, int& bi) {
 #pragma unroll
@@ -428,40 +436,51 @@ __device__ __forceinline__ void warp_best(float& bv, int& bi) {
   }
 }
 
+struct MergeScratch {      // level-1 results, [R][n_chunks] each
+  float* ms;               // (max, sum exp) pairs
+  float* val;              // [B] sorted values
+  int* id;                 // [B] their ids
+  int* count;              // [R] arrival counters: zero before the first launch, left at zero by every launch
+};
+
 __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __restrict__ p_max,
                                                                  const float* __restrict__ p_sum,
                                                                  const float* __restrict__ c_val,
                                                                  const int* __restrict__ c_id, int n_sub, int R, int B,
-                                                                 int* __restrict__ ids, float* __restrict__ logp) {
+                                                                 MergeScratch sc, int* __restrict__ ids,
+                                                                 float* __restrict__ logp) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[33];
-  __shared__ float w_val[32][MERGE_MAXB];
-  __shared__ int w_id[32][MERGE_MAXB];
+  __shared__ float w_val[MERGE_WARPS][MERGE_MAXB];
+  __shared__ int w_id[MERGE_WARPS][MERGE_MAXB];
   __shared__ float t_val;
   __shared__ int t_id;
   __shared__ float s_val[MERGE_MAXB * MERGE_MAXB];
   __shared__ int s_id[MERGE_MAXB * MERGE_MAXB];
   __shared__ int n_surv;
-  const int r = blockIdx.x;
+  __shared__ int is_last;
+  __shared__ float lse_sh;
+  const int chunk = blockIdx.x, n_chunks = gridDim.x, r = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int NONE = 0x7fffffff;
   const size_t row = (size_t)r * n_sub;
+  const size_t slot = (size_t)r * n_chunks + chunk;
   if (tid == 0) n_surv = 0;
-  if (tid < B) { ids[(size_t)r * B + tid] = -1; logp[(size_t)r * B + tid] = -INFINITY; }
+  if (tid < B) { sc.val[slot * B + tid] = -INFINITY; sc.id[slot * B + tid] = NONE; }
   // 1. this thread's slices
   float hv[MERGE_OWN], pm[MERGE_OWN], ps[MERGE_OWN];
   int hi[MERGE_OWN];
 #pragma unroll
   for (int j = 0; j < MERGE_OWN; ++j) {
-    const int s = tid + j * MERGE_THREADS;
+    const int s = chunk * MERGE_CHUNK + tid + j * MERGE_THREADS;
     const bool in = s < n_sub;
     pm[j] = in ? p_max[row + s] : -INFINITY;
     ps[j] = in ? p_sum[row + s] : 0.f;
     hv[j] = in ? c_val[(row + s) * B] : -INFINITY;
     hi[j] = in ? c_id[(row + s) * B] : NONE;
   }
-  // 2. logsumexp
+  // 2. the chunk's (max, sum exp)
   float m = -INFINITY;
 #pragma unroll
   for (int j = 0; j < MERGE_OWN; ++j) m = fmaxf(m, pm[j]);
@@ -471,7 +490,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   for (int j = 0; j < MERGE_OWN; ++j)
     if (pm[j] > -INFINITY) se += ps[j] * __expf(pm[j] - m);
   se = block_sum(se, red);
-  const float lse = m + logf(se);
+  if (tid == 0) { sc.ms[slot * 2] = m; sc.ms[slot * 2 + 1] = se; }
   // 3a. per warp: the B best heads among this warp's slices
   float pv = INFINITY;
   int pi = -1;
@@ -487,14 +506,14 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
     if (lane == 0) { w_val[wid][round] = bv; w_id[wid][round] = bi; }
   }
   __syncthreads();
-  // 3b. warp 0: the B-th best over the 32 sorted warp lists
+  // 3b. warp 0: the B-th best over the sorted warp lists
   if (wid == 0) {
     float qv = INFINITY;
     int qi = -1;
     int cur = 0;                                  // this lane's list is sorted: a cursor is enough
     for (int round = 0; round < B; ++round) {
-      float bv = cur < B ? w_val[lane][cur] : -INFINITY;
-      int bi = cur < B ? w_id[lane][cur] : NONE;
+      float bv = (lane < MERGE_WARPS && cur < B) ? w_val[lane][cur] : -INFINITY;
+      int bi = (lane < MERGE_WARPS && cur < B) ? w_id[lane][cur] : NONE;
       const float mv = bv;
       const int mi = bi;
       warp_best(bv, bi);
@@ -510,7 +529,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
   // 4. survivors: whole lists of the slices whose head passes, loaded at once
 #pragma unroll
   for (int j = 0; j < MERGE_OWN; ++j) {
-    const int s = tid + j * MERGE_THREADS;
+    const int s = chunk * MERGE_CHUNK + tid + j * MERGE_THREADS;
     if (s >= n_sub || hi[j] == NONE || ranks_before(tv, ti, hv[j], hi[j])) continue;
     float lv[MERGE_MAXB];
     int li[MERGE_MAXB];
@@ -527,16 +546,50 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
     }
   }
   __syncthreads();
-  // 5. rank by counting
-  const int ns = n_surv < MERGE_MAXB * MERGE_MAXB ? n_surv : MERGE_MAXB * MERGE_MAXB;
-  if (tid < ns) {
+  {
+    const int ns = n_surv < MERGE_MAXB * MERGE_MAXB ? n_surv : MERGE_MAXB * MERGE_MAXB;
+    if (tid < ns) {
+      const float v = s_val[tid];
+      const int id = s_id[tid];
+      int rank = 0;
+      for (int j = 0; j < ns; ++j) rank += ranks_before(s_val[j], s_id[j], v, id) ? 1 : 0;
+      if (rank < B) { sc.val[slot * B + rank] = v; sc.id[slot * B + rank] = id; }
+    }
+  }
+  // ---- arrival: the row's last CTA does level 2 ----
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int seen = atomicAdd(sc.count + r, 1);
+    is_last = seen == n_chunks - 1 ? 1 : 0;
+    if (is_last) sc.count[r] = 0;            // every CTA of the row has arrived: nobody touches it again
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  if (tid < B) { ids[(size_t)r * B + tid] = -1; logp[(size_t)r * B + tid] = -INFINITY; }
+  if (wid == 0) {
+    const bool in = lane < n_chunks;         // n_chunks <= MERGE_MAXCHUNKS <= 32
+    const float cm = in ? __ldcg(sc.ms + ((size_t)r * n_chunks + lane) * 2) : -INFINITY;
+    const float cs = in ? __ldcg(sc.ms + ((size_t)r * n_chunks + lane) * 2 + 1) : 0.f;
+    const float M = warp_max(cm);
+    const float S = warp_sum(cm > -INFINITY ? cs * __expf(cm - M) : 0.f);
+    if (lane == 0) lse_sh = M + logf(S);
+  }
+  const int nc = n_chunks * B;               // <= 256 candidates, sorted within each chunk
+  if (tid < nc) {
+    s_val[tid] = __ldcg(sc.val + (size_t)r * n_chunks * B + tid);
+    s_id[tid] = __ldcg(sc.id + (size_t)r * n_chunks * B + tid);
+  }
+  __syncthreads();
+  if (tid < nc && s_id[tid] != NONE) {
     const float v = s_val[tid];
     const int id = s_id[tid];
     int rank = 0;
-    for (int j = 0; j < ns; ++j) rank += ranks_before(s_val[j], s_id[j], v, id) ? 1 : 0;
+    for (int j = 0; j < nc; ++j) rank += ranks_before(s_val[j], s_id[j], v, id) ? 1 : 0;
     if (rank < B) {
       ids[(size_t)r * B + rank] = id;
-      logp[(size_t)r * B + rank] = v - lse;
+      logp[(size_t)r * B + rank] = v - lse_sh;
     }
   }
 }
