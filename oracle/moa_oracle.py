@@ -389,6 +389,34 @@ def tree_finalize(ts: TreeState):
             np.array(depth, np.int64), np.array(score, np.float32))
 
 
+def verify_greedy(tok, parent, target_logits):
+    """Greedy (exact-match) verification of a kept draft tree (Section 2.2, step 2 with Tree Attention;
+    Algorithm 1, the "identify K' verified tokens" step).
+
+    tok, parent [n]: the kept tree, slot 0 = the root (last verified token), parent[0] = -1, parent[i] < i; an
+    entry parent[i] < 0 at i > 0 marks an unused slot. target_logits [n, V]: the LLM's logits at every slot,
+    row i scoring the token that follows slot i's token on its root path (one LLM pass with the tree mask).
+    The LLM's choice at a slot is the arg-max (ties: smallest id). Starting at the root, the child carrying
+    the chosen token is accepted and the walk continues from it; at the first slot with no such child
+    everything else is discarded. Returns (slots, next_tok, choice): the accepted slots (root first, so
+    K' = len(slots) - 1), the LLM's choice at the last accepted slot (the next cycle's root) and every
+    slot's choice."""
+    tok = [int(t) for t in tok]
+    parent = [int(q) for q in parent]
+    z = np.asarray(target_logits, F64)
+    n = len(tok)
+    choice = [int(np.lexsort((np.arange(z.shape[1]), -z[i]))[0]) for i in range(n)]
+    slots = [0]
+    cur = 0
+    while True:
+        nxt = [c for c in range(1, n) if parent[c] == cur and tok[c] == choice[cur]]
+        if not nxt:
+            break
+        cur = nxt[0]
+        slots.append(cur)
+    return slots, choice[cur], choice
+
+
 def tree_mask(parent):
     """mask[i][j] = 1 iff j == i or j is an ancestor of i. parent[0] = -1."""
     n = len(parent)

@@ -524,3 +524,72 @@ def test_fp32_inputs_agree_with_fp64():
     a = O.Drafter(c, w).lsa_forward(H)
     b = O.Drafter(c, w32).lsa_forward(H.astype(np.float32))
     assert np.max(np.abs(a - b)) < 1e-5 * np.max(np.abs(a))
+
+
+# ------------------------------------------------------------------ verification (greedy acceptance)
+def _random_tree(rng, n, vocab, width=3):
+    """A random kept tree: parent[i] < i, sibling tokens distinct."""
+    tok, parent = [int(rng.integers(vocab))], [-1]
+    for i in range(1, n):
+        for _ in range(100):
+            q = int(rng.integers(0, i))
+            t = int(rng.integers(vocab))
+            sibs = [tok[c] for c in range(1, i) if parent[c] == q]
+            if t not in sibs and len(sibs) < width:
+                break
+        tok.append(t)
+        parent.append(q)
+    return tok, parent
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_verify_greedy_equals_token_by_token_greedy_decoding(seed):
+    """Brute force (Section 2.2, step 2: discard everything after the first mismatch): with an LLM that is a
+    deterministic function of the token path, the accepted tokens are the longest prefix of the LLM's own greedy
+    continuation that exists in the tree as a root path, and the bonus token is the continuation's next token."""
+    rng = np.random.default_rng(seed)
+    vocab, n = 5, 30
+    tok, parent = _random_tree(rng, n, vocab)
+    table = {}
+    def llm_logits(path):                     # a fixed random logit row per token path
+        if path not in table:
+            table[path] = np.random.default_rng(hash(path) % (2 ** 32)).standard_normal(vocab)
+        return table[path]
+    def path_of(i):
+        p = []
+        while i >= 0:
+            p.append(tok[i]); i = parent[i]
+        return tuple(reversed(p))
+    logits = np.stack([llm_logits(path_of(i)) for i in range(n)])
+    slots, nxt, choice = O.verify_greedy(tok, parent, logits)
+    # token-by-token greedy decoding from the root, no tree involved
+    seq = [tok[0]]
+    paths = {path_of(i) for i in range(n)}
+    while True:
+        g = int(np.argmax(llm_logits(tuple(seq))))
+        if tuple(seq + [g]) in paths:
+            seq.append(g)
+        else:
+            bonus = g
+            break
+    assert [tok[i] for i in slots] == seq
+    assert nxt == bonus
+    assert slots[0] == 0 and all(parent[b] == a for a, b in zip(slots, slots[1:]))
+    assert choice == [int(np.argmax(r)) for r in logits]
+
+
+def test_verify_greedy_special_cases():
+    """A chain whose every token is the LLM's choice is accepted whole; a wrong first token rejects everything;
+    ties go to the smaller token id; unused slots (parent < 0) never match."""
+    V = 6
+    tok, parent = [2, 4, 1, 3], [-1, 0, 1, 2]
+    z = np.full((4, V), -1.0)
+    z[0, 4] = z[1, 1] = z[2, 3] = z[3, 5] = 2.0
+    slots, nxt, _ = O.verify_greedy(tok, parent, z)
+    assert slots == [0, 1, 2, 3] and nxt == 5
+    z2 = z.copy(); z2[0, 4] = -1.0; z2[0, 0] = 3.0
+    assert O.verify_greedy(tok, parent, z2)[:2] == ([0], 0)
+    z3 = z.copy(); z3[0, 1] = 2.0                       # tie between ids 1 and 4 at the root: id 1 wins, no child has it
+    assert O.verify_greedy(tok, parent, z3)[:2] == ([0], 1)
+    tok5, parent5 = [2, 4, 4], [-1, -1, 0]              # slot 1 unused; slot 2 is the real child
+    assert O.verify_greedy(tok5, parent5, z[:3])[0] == [0, 2]
