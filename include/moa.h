@@ -219,6 +219,24 @@ moa_status moa_tree_expand(moa_ctx *ctx, moa_state *st, int32_t batch, const int
  * packed = 0: uint8 [batch, n, n]; packed = 1: uint64 [batch, n, ceil(n/64)], bit j%64 of word j/64. */
 moa_status moa_tree_attn_mask(const int32_t *parent, int32_t batch, int32_t n, void *mask_out, int32_t packed, void *stream);
 
+/* Greedy verification of the kept tree (Section 2.2, step 2: exact matching, everything after the first mismatch
+ * is discarded; Algorithm 1, the step that identifies the K' verified tokens and the LLM's next token y').
+ * The LLM itself is not part of the library: the caller runs it once over the kept tree with the mask of
+ * moa_tree_attn_mask and passes its logits.
+ *   tok, parent    device int32 [batch, n]: the kept tree as moa_tree_expand wrote it (slot 0 = root, parent[0] = -1,
+ *                  parent[i] < i, parent[i] < 0 at i > 0 = unused slot)
+ *   target_logits  device [batch, n, vocab] of logits_dtype (moa_dtype): row (b, i) scores the token FOLLOWING slot i
+ *   choice         device int32 [batch, n] out: arg-max of every row, ties to the smallest id (the row of an
+ *                  unused slot is read like any other)
+ *   acc_slot, acc_tok  device int32 [batch, cap] out: slots and tokens of the accepted path, root first, -1 behind it
+ *   acc_len        device int32 [batch] out: 1 + K' (root included), at most cap
+ *   next_tok       device int32 [batch] out: the LLM's choice at the last accepted slot = the next cycle's root
+ * cap >= 1 bounds the path length (tree_depth + 1 covers every tree of this library). To carry the accepted
+ * tokens into the drafter's self-attention prefix, pass acc_tok's first acc_len entries to moa_sa_append. */
+moa_status moa_verify_greedy(const int32_t *tok, const int32_t *parent, int32_t batch, int32_t n, const void *target_logits,
+                             int32_t logits_dtype, int32_t vocab, int32_t cap, int32_t *choice, int32_t *acc_slot,
+                             int32_t *acc_tok, int32_t *acc_len, int32_t *next_tok, void *stream);
+
 /* Reads back the device status word kept in st->tree (0 = no device-side problem seen). Synchronises the stream. */
 moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
 

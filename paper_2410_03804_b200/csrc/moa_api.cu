@@ -11,6 +11,7 @@
 #include "moa_basic.cuh"
 #include "moa_phases.cuh"
 #include "moa_tree.cuh"
+#include "moa_verify.cuh"
 #include "moa_wstream.cuh"
 
 using namespace moa;
@@ -1608,6 +1609,25 @@ moa_status moa_sa_append_static(moa_ctx* ctx, moa_state* st, const int32_t* tok,
   if (r == MOA_OK)
     for (int b = 0; b < batch; ++b) st->sa_len_host[b] += n_host[b];
   return r;
+}
+
+moa_status moa_verify_greedy(const int32_t* tok, const int32_t* parent, int32_t batch, int32_t n, const void* target_logits,
+                             int32_t logits_dtype, int32_t vocab, int32_t cap, int32_t* choice, int32_t* acc_slot,
+                             int32_t* acc_tok, int32_t* acc_len, int32_t* next_tok, void* stream) {
+  if (!tok || !parent || !target_logits || !choice || !acc_slot || !acc_tok || !acc_len || !next_tok) return MOA_ERR_NULL;
+  if (batch <= 0 || batch > MOA_MAX_BATCH || n <= 0 || vocab <= 0 || cap <= 0) return MOA_ERR_SHAPE;
+  if (logits_dtype != MOA_F32 && logits_dtype != MOA_BF16) return MOA_ERR_DTYPE;
+  if ((long long)batch * n > 0x7fffffffll) return MOA_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (logits_dtype == MOA_F32)
+    launch_pdl(argmax_rows_kernel<float>, dim3(batch * n), dim3(512), 0, s, (const float*)target_logits, vocab, choice);
+  else
+    launch_pdl(argmax_rows_kernel<bf16>, dim3(batch * n), dim3(512), 0, s, (const bf16*)target_logits, vocab, choice);
+  MOA_CHECK_LAUNCH();
+  launch_pdl(verify_walk_kernel, dim3((batch + 63) / 64), dim3(64), 0, s, tok, parent, (const int*)choice, batch, n, cap, acc_slot,
+             acc_tok, acc_len, next_tok);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
 }
 
 moa_status moa_state_status(moa_ctx* ctx, moa_state* st, void* stream) {

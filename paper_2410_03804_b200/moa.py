@@ -21,7 +21,7 @@ MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
-           "moa_tree_expand", "moa_tree_attn_mask", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
+           "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
 
 
@@ -111,6 +111,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_draft_step.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, sz, vp]
     lib.moa_tree_expand.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moa_tree_attn_mask.argtypes = [vp, i32, i32, vp, i32, vp]
+    lib.moa_verify_greedy.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.moa_state_status.argtypes = [vp, C.POINTER(MoaState), vp]
     lib.moa_profile_begin.argtypes = [vp]
     lib.moa_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
@@ -157,6 +158,27 @@ def moa_tree_attn_mask(parent: torch.Tensor, packed: bool = False, stream=None) 
                                            1 if packed else 0, _stream(stream))
     _check(st, "moa_tree_attn_mask")
     return out
+
+
+def moa_verify_greedy(tok: torch.Tensor, parent: torch.Tensor, target_logits: torch.Tensor, cap: int, stream=None):
+    """tok, parent: cuda int32 [batch, n] (the kept tree); target_logits: cuda float32 / bfloat16 [batch, n, V].
+    Returns (choice [batch, n], acc_slot [batch, cap], acc_tok [batch, cap], acc_len [batch], next_tok [batch])."""
+    assert tok.is_cuda and tok.dtype == torch.int32 and tok.is_contiguous() and tok.dim() == 2
+    assert parent.is_cuda and parent.dtype == torch.int32 and parent.is_contiguous() and parent.shape == tok.shape
+    assert target_logits.is_cuda and target_logits.is_contiguous() and target_logits.shape[:2] == tok.shape
+    assert target_logits.dtype in (torch.float32, torch.bfloat16)
+    b, n = tok.shape
+    dev = tok.device
+    choice = torch.empty((b, n), dtype=torch.int32, device=dev)
+    acc_slot = torch.empty((b, cap), dtype=torch.int32, device=dev)
+    acc_tok = torch.empty((b, cap), dtype=torch.int32, device=dev)
+    acc_len = torch.empty((b,), dtype=torch.int32, device=dev)
+    next_tok = torch.empty((b,), dtype=torch.int32, device=dev)
+    _check(load_library().moa_verify_greedy(_ptr(tok), _ptr(parent), b, n, _ptr(target_logits),
+                                            0 if target_logits.dtype == torch.float32 else 1, target_logits.shape[2],
+                                            int(cap), _ptr(choice), _ptr(acc_slot), _ptr(acc_tok), _ptr(acc_len),
+                                            _ptr(next_tok), _stream(stream)), "moa_verify_greedy")
+    return choice, acc_slot, acc_tok, acc_len, next_tok
 
 
 class MoA:
