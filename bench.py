@@ -459,6 +459,21 @@ def main():
     # the D forwards alone (draft step + expansion), stream launches, events around them inside each cycle
     timed(lambda: cycle(h_dev, tok_dev, root_dev, mark=True), args.steps)
     fwd_us = statistics.mean(a.elapsed_time(b) for a, b in split_ev) * 1e3 / D
+    # verification bookkeeping (moa_verify_greedy) on the last cycle's kept tree with seeded synthetic LLM logits:
+    # timed on its own, not part of the step
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(synth.SEED_BASE + 77)
+    vz = torch.randn((nb, W, p.vocab), generator=gen, device=dev, dtype=torch.float32).to(p.torch_dtype)
+    vout = moa.moa_verify_greedy(outs[0], outs[1], vz, D + 1)
+    torch.cuda.synchronize()
+    vgraph = torch.cuda.CUDAGraph()               # `steps` calls recorded once: the calls are shorter than a Python call
+    with torch.cuda.graph(vgraph):
+        for _ in range(args.steps):
+            moa.moa_verify_greedy(outs[0], outs[1], vz, D + 1, out=vout)
+    vgraph.replay()
+    ms_verify = timed(vgraph.replay, 1) / args.steps
+    vbytes = vz.numel() * vz.element_size()
+    del vz
     clocks = sampler.stop()
     launches = launches_per_cycle * args.steps
     assert g.moa_state_status() == 0
@@ -496,6 +511,11 @@ def main():
                              "us": fwd_us, "algorithmic_bytes": ab["step"], "achieved_gbs": ab["step"] / fwd_us / 1e3,
                              "frac_of_measured": ab["step"] / fwd_us / 1e3 / peak,
                              "frac_of_8tbs": ab["step"] / fwd_us / 1e3 / 8000.0},
+        "verify": {"what": f"moa_verify_greedy on [{nb}, {W}, {p.vocab}] {p.dtype} logits (arg-max + accepted-path walk), "
+                           "back-to-back calls replayed from a CUDA graph, not part of the step",
+                   "us": ms_verify * 1e3, "bytes": vbytes, "achieved_gbs": vbytes / ms_verify / 1e6,
+                   "frac_of_measured": vbytes / ms_verify / 1e6 / peak,
+                   "l2": "logits larger than L2" if vbytes > 126e6 else "logits fit in L2: not an HBM figure"},
         "replicas": "replicas only: no data-path collective" if world > 1 else None,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

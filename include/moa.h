@@ -231,7 +231,7 @@ moa_status moa_tree_attn_mask(const int32_t *parent, int32_t batch, int32_t n, v
  *   acc_slot, acc_tok  device int32 [batch, cap] out: slots and tokens of the accepted path, root first, -1 behind it
  *   acc_len        device int32 [batch] out: 1 + K' (root included), at most cap
  *   next_tok       device int32 [batch] out: the LLM's choice at the last accepted slot = the next cycle's root
- * cap >= 1 bounds the path length (tree_depth + 1 covers every tree of this library). To carry the accepted
+ * cap >= 1 bounds the path length (tree_depth + 1 covers every tree of this library). batch * n <= 65535. To carry the accepted
  * tokens into the drafter's self-attention prefix, pass acc_tok's first acc_len entries to moa_sa_append. */
 moa_status moa_verify_greedy(const int32_t *tok, const int32_t *parent, int32_t batch, int32_t n, const void *target_logits,
                              int32_t logits_dtype, int32_t vocab, int32_t cap, int32_t *choice, int32_t *acc_slot,

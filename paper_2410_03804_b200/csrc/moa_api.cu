@@ -1617,14 +1617,25 @@ moa_status moa_verify_greedy(const int32_t* tok, const int32_t* parent, int32_t 
   if (!tok || !parent || !target_logits || !choice || !acc_slot || !acc_tok || !acc_len || !next_tok) return MOA_ERR_NULL;
   if (batch <= 0 || batch > MOA_MAX_BATCH || n <= 0 || vocab <= 0 || cap <= 0) return MOA_ERR_SHAPE;
   if (logits_dtype != MOA_F32 && logits_dtype != MOA_BF16) return MOA_ERR_DTYPE;
-  if ((long long)batch * n > 0x7fffffffll) return MOA_ERR_SHAPE;
+  if ((long long)batch * n > 65535) return MOA_ERR_SHAPE;          // one cluster per row along gridDim.y
   cudaStream_t s = (cudaStream_t)stream;
-  if (logits_dtype == MOA_F32)
-    launch_pdl(argmax_rows_kernel<float>, dim3(batch * n), dim3(512), 0, s, (const float*)target_logits, vocab, choice);
-  else
-    launch_pdl(argmax_rows_kernel<bf16>, dim3(batch * n), dim3(512), 0, s, (const bf16*)target_logits, vocab, choice);
+  // few rows: a cluster of CTAs per row, so that the rows fill the GPU; many rows: one CTA per row
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const int rows = batch * n;
+  const bool spread = rows < 4 * sms;
+  if (logits_dtype == MOA_F32) {
+    if (spread) launch_pdl(argmax_rows_kernel<float, AM_CLUSTER>, dim3(AM_CLUSTER, rows), dim3(256), 0, s, (const float*)target_logits, vocab, choice);
+    else launch_pdl(argmax_rows_kernel<float, 1>, dim3(1, rows), dim3(256), 0, s, (const float*)target_logits, vocab, choice);
+  } else {
+    if (spread) launch_pdl(argmax_rows_kernel<bf16, AM_CLUSTER>, dim3(AM_CLUSTER, rows), dim3(256), 0, s, (const bf16*)target_logits, vocab, choice);
+    else launch_pdl(argmax_rows_kernel<bf16, 1>, dim3(1, rows), dim3(256), 0, s, (const bf16*)target_logits, vocab, choice);
+  }
   MOA_CHECK_LAUNCH();
-  launch_pdl(verify_walk_kernel, dim3((batch + 63) / 64), dim3(64), 0, s, tok, parent, (const int*)choice, batch, n, cap, acc_slot,
+  launch_pdl(verify_walk_kernel, dim3((batch + 3) / 4), dim3(128), 0, s, tok, parent, (const int*)choice, batch, n, cap, acc_slot,
              acc_tok, acc_len, next_tok);
   MOA_CHECK_LAUNCH();
   return MOA_OK;

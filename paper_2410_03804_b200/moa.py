@@ -160,20 +160,25 @@ def moa_tree_attn_mask(parent: torch.Tensor, packed: bool = False, stream=None) 
     return out
 
 
-def moa_verify_greedy(tok: torch.Tensor, parent: torch.Tensor, target_logits: torch.Tensor, cap: int, stream=None):
+def moa_verify_greedy(tok: torch.Tensor, parent: torch.Tensor, target_logits: torch.Tensor, cap: int, out=None,
+                      stream=None):
     """tok, parent: cuda int32 [batch, n] (the kept tree); target_logits: cuda float32 / bfloat16 [batch, n, V].
-    Returns (choice [batch, n], acc_slot [batch, cap], acc_tok [batch, cap], acc_len [batch], next_tok [batch])."""
+    Returns (choice [batch, n], acc_slot [batch, cap], acc_tok [batch, cap], acc_len [batch], next_tok [batch]);
+    out: the same five int32 tensors preallocated by the caller."""
     assert tok.is_cuda and tok.dtype == torch.int32 and tok.is_contiguous() and tok.dim() == 2
     assert parent.is_cuda and parent.dtype == torch.int32 and parent.is_contiguous() and parent.shape == tok.shape
     assert target_logits.is_cuda and target_logits.is_contiguous() and target_logits.shape[:2] == tok.shape
     assert target_logits.dtype in (torch.float32, torch.bfloat16)
     b, n = tok.shape
     dev = tok.device
-    choice = torch.empty((b, n), dtype=torch.int32, device=dev)
-    acc_slot = torch.empty((b, cap), dtype=torch.int32, device=dev)
-    acc_tok = torch.empty((b, cap), dtype=torch.int32, device=dev)
-    acc_len = torch.empty((b,), dtype=torch.int32, device=dev)
-    next_tok = torch.empty((b,), dtype=torch.int32, device=dev)
+    if out is not None:
+        choice, acc_slot, acc_tok, acc_len, next_tok = out
+    else:
+        choice = torch.empty((b, n), dtype=torch.int32, device=dev)
+        acc_slot = torch.empty((b, cap), dtype=torch.int32, device=dev)
+        acc_tok = torch.empty((b, cap), dtype=torch.int32, device=dev)
+        acc_len = torch.empty((b,), dtype=torch.int32, device=dev)
+        next_tok = torch.empty((b,), dtype=torch.int32, device=dev)
     _check(load_library().moa_verify_greedy(_ptr(tok), _ptr(parent), b, n, _ptr(target_logits),
                                             0 if target_logits.dtype == torch.float32 else 1, target_logits.shape[2],
                                             int(cap), _ptr(choice), _ptr(acc_slot), _ptr(acc_tok), _ptr(acc_len),
