@@ -508,3 +508,51 @@ def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft, tliK=Non
         toks.append(int(out["ids"][0]))
         lps.append(float(out["logp"][0]))
     return toks[1:], lps
+
+
+# --------------------------------------------------------------------------
+# client-server message codec (Section 4.2 "Client-Server"; message-size table in the appendix)
+# --------------------------------------------------------------------------
+def pack_tree(tok, parent):
+    """Client message: every draft-tree node as 3 bytes of token id (little endian) + 1 byte for its position
+    in the tree, 4 bytes per node, so a tree of M nodes is a 4M-byte message (the table's "4M").
+    Reading: the position byte is the parent's slot number (a tree is its parent list; slots are < 255); 255
+    marks "no parent" (the root, or an unused slot, whose token bytes are ff ff ff).
+    tok, parent [n] -> uint8 [n, 4]."""
+    n = len(tok)
+    out = np.zeros((n, 4), np.uint8)
+    for i in range(n):
+        t, q = int(tok[i]), int(parent[i])
+        t = 0xFFFFFF if t < 0 else t & 0xFFFFFF
+        out[i] = [t & 0xFF, (t >> 8) & 0xFF, (t >> 16) & 0xFF, 255 if q < 0 else q & 0xFF]
+    return out
+
+
+def unpack_tree(msg):
+    """Inverse of pack_tree: uint8 [n, 4] -> tok, parent (int64 [n]); ff ff ff -> token -1, 255 -> parent -1."""
+    msg = np.asarray(msg, np.uint8)
+    tok = msg[:, 0].astype(np.int64) | (msg[:, 1].astype(np.int64) << 8) | (msg[:, 2].astype(np.int64) << 16)
+    tok[tok == 0xFFFFFF] = -1
+    parent = msg[:, 3].astype(np.int64)
+    parent[parent == 255] = -1
+    return tok, parent
+
+
+def quantize_rows(x):
+    """8-bit quantisation of activation rows (Section 4.2: the E and E_kv tensors are quantised to 8 bits).
+    Reading (the paper gives no scheme): symmetric, one fp32 scale per row, scale = max|x| / 127,
+    code = round-half-even(x / scale) in [-127, 127]; an all-zero row has scale 0 and codes 0. The decision
+    is taken in fp32 (the precision both sides use). x [rows, width] -> (int8 codes, float32 scales)."""
+    x = np.asarray(x, np.float32)
+    amax = np.max(np.abs(x), axis=-1).astype(np.float32)
+    scale = (amax / np.float32(127.0)).astype(np.float32)
+    safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
+    q = np.rint((x / safe[:, None]).astype(np.float32))
+    q = np.clip(q, -127, 127)
+    q = np.where(scale[:, None] > 0, q, 0)
+    return q.astype(np.int8), scale
+
+
+def dequantize_rows(codes, scales):
+    """x ~ code * scale, one fp32 product per element."""
+    return (np.asarray(codes, np.float32) * np.asarray(scales, np.float32)[:, None]).astype(np.float32)

@@ -593,3 +593,40 @@ def test_verify_greedy_special_cases():
     assert O.verify_greedy(tok, parent, z3)[:2] == ([0], 1)
     tok5, parent5 = [2, 4, 4], [-1, -1, 0]              # slot 1 unused; slot 2 is the real child
     assert O.verify_greedy(tok5, parent5, z[:3])[0] == [0, 2]
+
+
+# ------------------------------------------------------------------ client-server message codec
+def test_pack_tree_layout_size_and_round_trip():
+    """4 bytes per node (the message-size table's 4M for a tree of M nodes): 3 little-endian token bytes and
+    the parent slot; pack and unpack are inverse on every valid tree."""
+    msg = O.pack_tree([0x123456, 7, -1], [-1, 0, -1])
+    assert msg.dtype == np.uint8 and msg.shape == (3, 4) and msg.nbytes == 4 * 3
+    assert msg.tolist() == [[0x56, 0x34, 0x12, 255], [7, 0, 0, 0], [255, 255, 255, 255]]
+    rng = np.random.default_rng(2)
+    for _ in range(20):
+        tok, parent = _random_tree(rng, 61, 128256, width=10)
+        t2, p2 = O.unpack_tree(O.pack_tree(tok, parent))
+        assert t2.tolist() == tok and p2.tolist() == parent
+
+
+def test_quantize_rows_bounds_and_fixed_points():
+    """Closed forms: |x - dequant| <= scale / 2; the row's largest magnitude maps to +-127 exactly; codes stay
+    in [-127, 127]; an all-zero row gives zeros; quantising a dequantised row returns the same codes; a row that
+    is already k * s for integers |k| <= 127 (max 127) is reproduced exactly."""
+    rng = np.random.default_rng(4)
+    x = (rng.standard_normal((50, 333)) * rng.uniform(0.01, 30, (50, 1))).astype(np.float32)
+    x[7] = 0
+    q, s = O.quantize_rows(x)
+    d = O.dequantize_rows(q, s)
+    assert q.dtype == np.int8 and s.dtype == np.float32 and int(np.abs(q.astype(int)).max()) == 127
+    assert np.all(np.abs(x - d) <= s[:, None] * 0.5 * (1 + 1e-6))
+    am = np.argmax(np.abs(x), axis=1)
+    rows = np.arange(50)
+    assert np.all(np.abs(q[rows, am])[s > 0] == 127)
+    assert np.all(q[7] == 0) and s[7] == 0 and np.all(d[7] == 0)
+    q2, s2 = O.quantize_rows(d)
+    assert np.array_equal(q2, q)
+    k = rng.integers(-127, 128, (4, 64)); k[:, 0] = 127
+    y = (k * np.float32(0.25)).astype(np.float32)
+    qy, sy = O.quantize_rows(y)
+    assert np.array_equal(qy, k) and np.all(sy == np.float32(0.25)) and np.array_equal(O.dequantize_rows(qy, sy), y)
