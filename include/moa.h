@@ -237,6 +237,25 @@ moa_status moa_verify_greedy(const int32_t *tok, const int32_t *parent, int32_t 
                              int32_t logits_dtype, int32_t vocab, int32_t cap, int32_t *choice, int32_t *acc_slot,
                              int32_t *acc_tok, int32_t *acc_len, int32_t *next_tok, void *stream);
 
+/* Client-server message codec (Section 4.2 "Client-Server" and the message-size table of the appendix).
+ * moa_pack_tree: every node of the kept tree as 4 bytes -- the token id in 3 bytes, little endian, and 1 byte for
+ * its position in the tree, here the parent's slot number -- so a tree of M nodes is a 4M-byte message. A negative
+ * token id is written as ff ff ff, a negative parent (the root, an unused slot) as 255; token ids must be below
+ * 2^24 - 1 and slots below 255 (larger values are truncated to their low bits).
+ *   tok, parent  device int32 [count]      msg  device bytes [count, 4], 4-byte aligned
+ * moa_unpack_tree is the inverse. */
+moa_status moa_pack_tree(const int32_t *tok, const int32_t *parent, int64_t count, void *msg, void *stream);
+moa_status moa_unpack_tree(const void *msg, int64_t count, int32_t *tok, int32_t *parent, void *stream);
+/* 8-bit quantisation of activation rows (the E / E_kv tensors the server sends, Section 4.2). The paper names no
+ * scheme; this one is symmetric with one fp32 scale per row: scale = max|x| / 127, code = round-half-even(x / scale)
+ * in [-127, 127], decided in fp32; an all-zero row has scale 0 and codes 0. moa_dequantize_rows writes
+ * code * scale in `dtype`.
+ *   x / out  device [rows, width] of dtype (moa_dtype)    codes  device int8 [rows, width]    scales  device float [rows] */
+moa_status moa_quantize_rows(const void *x, int32_t dtype, int64_t rows, int32_t width, int8_t *codes, float *scales,
+                             void *stream);
+moa_status moa_dequantize_rows(const int8_t *codes, const float *scales, int64_t rows, int32_t width, void *out,
+                               int32_t dtype, void *stream);
+
 /* Reads back the device status word kept in st->tree (0 = no device-side problem seen). Synchronises the stream. */
 moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
 

@@ -9,6 +9,7 @@
 
 #include "moa_attn.cuh"
 #include "moa_basic.cuh"
+#include "moa_codec.cuh"
 #include "moa_phases.cuh"
 #include "moa_tree.cuh"
 #include "moa_verify.cuh"
@@ -1637,6 +1638,64 @@ moa_status moa_verify_greedy(const int32_t* tok, const int32_t* parent, int32_t 
   MOA_CHECK_LAUNCH();
   launch_pdl(verify_walk_kernel, dim3((batch + 3) / 4), dim3(128), 0, s, tok, parent, (const int*)choice, batch, n, cap, acc_slot,
              acc_tok, acc_len, next_tok);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+moa_status moa_pack_tree(const int32_t* tok, const int32_t* parent, int64_t count, void* msg, void* stream) {
+  if (!tok || !parent || !msg) return MOA_ERR_NULL;
+  if (count < 0 || count > (1ll << 31)) return MOA_ERR_SHAPE;
+  if ((uintptr_t)msg & 3u) return MOA_ERR_ALIGN;
+  if (count == 0) return MOA_OK;
+  launch_pdl(pack_tree_kernel, dim3(blocks_for((size_t)count, 256)), dim3(256), 0, (cudaStream_t)stream, tok, parent, (size_t)count,
+             (uint32_t*)msg);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+moa_status moa_unpack_tree(const void* msg, int64_t count, int32_t* tok, int32_t* parent, void* stream) {
+  if (!tok || !parent || !msg) return MOA_ERR_NULL;
+  if (count < 0 || count > (1ll << 31)) return MOA_ERR_SHAPE;
+  if ((uintptr_t)msg & 3u) return MOA_ERR_ALIGN;
+  if (count == 0) return MOA_OK;
+  launch_pdl(unpack_tree_kernel, dim3(blocks_for((size_t)count, 256)), dim3(256), 0, (cudaStream_t)stream, (const uint32_t*)msg,
+             (size_t)count, tok, parent);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+moa_status moa_quantize_rows(const void* x, int32_t dtype, int64_t rows, int32_t width, int8_t* codes, float* scales,
+                             void* stream) {
+  if (!x || !codes || !scales) return MOA_ERR_NULL;
+  if (dtype != MOA_F32 && dtype != MOA_BF16) return MOA_ERR_DTYPE;
+  if (rows < 0 || width <= 0 || rows > (1ll << 31)) return MOA_ERR_SHAPE;
+  if (rows == 0) return MOA_OK;
+  const int per = dtype == MOA_F32 ? 4 : 8;
+  const int vec = (width % per == 0 && aligned16(x) && ((uintptr_t)codes & 7u) == 0) ? 1 : 0;
+  const unsigned grid = blocks_for((size_t)rows, 8);
+  if (dtype == MOA_F32)
+    launch_pdl(quantize_rows_kernel<float>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, (const float*)x, (long long)rows, width, vec,
+               codes, scales);
+  else
+    launch_pdl(quantize_rows_kernel<bf16>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, (const bf16*)x, (long long)rows, width, vec,
+               codes, scales);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+moa_status moa_dequantize_rows(const int8_t* codes, const float* scales, int64_t rows, int32_t width, void* out, int32_t dtype,
+                               void* stream) {
+  if (!out || !codes || !scales) return MOA_ERR_NULL;
+  if (dtype != MOA_F32 && dtype != MOA_BF16) return MOA_ERR_DTYPE;
+  if (rows < 0 || width <= 0 || rows > (1ll << 31)) return MOA_ERR_SHAPE;
+  if (rows == 0) return MOA_OK;
+  const unsigned grid = blocks_for((size_t)rows * width, 256);
+  if (dtype == MOA_F32)
+    launch_pdl(dequantize_rows_kernel<float>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width,
+               (float*)out);
+  else
+    launch_pdl(dequantize_rows_kernel<bf16>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width,
+               (bf16*)out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }

@@ -21,7 +21,7 @@ MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
-           "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
+           "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_pack_tree", "moa_unpack_tree", "moa_quantize_rows", "moa_dequantize_rows", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
 
 
@@ -112,6 +112,10 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_tree_expand.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.moa_tree_attn_mask.argtypes = [vp, i32, i32, vp, i32, vp]
     lib.moa_verify_greedy.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.moa_pack_tree.argtypes = [vp, vp, C.c_int64, vp, vp]
+    lib.moa_unpack_tree.argtypes = [vp, C.c_int64, vp, vp, vp]
+    lib.moa_quantize_rows.argtypes = [vp, i32, C.c_int64, i32, vp, vp, vp]
+    lib.moa_dequantize_rows.argtypes = [vp, vp, C.c_int64, i32, vp, i32, vp]
     lib.moa_state_status.argtypes = [vp, C.POINTER(MoaState), vp]
     lib.moa_profile_begin.argtypes = [vp]
     lib.moa_profile_end.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
@@ -184,6 +188,43 @@ def moa_verify_greedy(tok: torch.Tensor, parent: torch.Tensor, target_logits: to
                                             int(cap), _ptr(choice), _ptr(acc_slot), _ptr(acc_tok), _ptr(acc_len),
                                             _ptr(next_tok), _stream(stream)), "moa_verify_greedy")
     return choice, acc_slot, acc_tok, acc_len, next_tok
+
+
+def moa_pack_tree(tok: torch.Tensor, parent: torch.Tensor, stream=None) -> torch.Tensor:
+    """cuda int32 [..., n] token ids and parent slots -> cuda uint8 [..., n, 4] (the client's 4-bytes-per-node message)."""
+    assert tok.is_cuda and tok.dtype == torch.int32 and tok.is_contiguous() and parent.shape == tok.shape
+    assert parent.is_cuda and parent.dtype == torch.int32 and parent.is_contiguous()
+    msg = torch.empty(tuple(tok.shape) + (4,), dtype=torch.uint8, device=tok.device)
+    _check(load_library().moa_pack_tree(_ptr(tok), _ptr(parent), tok.numel(), _ptr(msg), _stream(stream)), "moa_pack_tree")
+    return msg
+
+
+def moa_unpack_tree(msg: torch.Tensor, stream=None):
+    assert msg.is_cuda and msg.dtype == torch.uint8 and msg.is_contiguous() and msg.shape[-1] == 4
+    tok = torch.empty(tuple(msg.shape[:-1]), dtype=torch.int32, device=msg.device)
+    parent = torch.empty_like(tok)
+    _check(load_library().moa_unpack_tree(_ptr(msg), tok.numel(), _ptr(tok), _ptr(parent), _stream(stream)), "moa_unpack_tree")
+    return tok, parent
+
+
+def moa_quantize_rows(x: torch.Tensor, out=None, stream=None):
+    """x cuda float32 / bfloat16 [rows, width] -> (int8 codes [rows, width], float32 scales [rows])."""
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 2 and x.dtype in (torch.float32, torch.bfloat16)
+    codes, scales = out if out is not None else (torch.empty(x.shape, dtype=torch.int8, device=x.device),
+                                                 torch.empty((x.shape[0],), dtype=torch.float32, device=x.device))
+    _check(load_library().moa_quantize_rows(_ptr(x), 0 if x.dtype == torch.float32 else 1, x.shape[0], x.shape[1],
+                                            _ptr(codes), _ptr(scales), _stream(stream)), "moa_quantize_rows")
+    return codes, scales
+
+
+def moa_dequantize_rows(codes: torch.Tensor, scales: torch.Tensor, dtype=torch.float32, out=None, stream=None):
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.is_contiguous() and codes.dim() == 2
+    assert scales.is_cuda and scales.dtype == torch.float32 and scales.numel() == codes.shape[0]
+    if out is None:
+        out = torch.empty(codes.shape, dtype=dtype, device=codes.device)
+    _check(load_library().moa_dequantize_rows(_ptr(codes), _ptr(scales), codes.shape[0], codes.shape[1], _ptr(out),
+                                              0 if out.dtype == torch.float32 else 1, _stream(stream)), "moa_dequantize_rows")
+    return out
 
 
 class MoA:
