@@ -249,6 +249,17 @@ def run_lsa_prefill(args, p, dev, rank, world):
     ph = g.moa_profile_phases()
     g.moa_profile_end()
     ms_e2e = timed(step_e2e, args.steps) / args.steps
+    # the server-side message codec on the same activations: 8-bit quantisation of the whole prompt's rows
+    flat = h_dev.reshape(-1, p.d_stack)
+    qout = (torch.empty(flat.shape, dtype=torch.int8, device=dev), torch.empty((flat.shape[0],), dtype=torch.float32, device=dev))
+    moa.moa_quantize_rows(flat, out=qout)
+    ms_q = timed(lambda: moa.moa_quantize_rows(flat, out=qout), args.steps) / args.steps
+    deq = torch.empty_like(flat)
+    moa.moa_dequantize_rows(qout[0], qout[1], out=deq)
+    ms_dq = timed(lambda: moa.moa_dequantize_rows(qout[0], qout[1], out=deq), args.steps) / args.steps
+    q_bytes = flat.numel() * 3 + flat.shape[0] * 4          # bf16 in, int8 out, one scale per row
+    hbm = measured_peaks()[0]
+    del deq
     clocks = sampler.stop()
     assert g.moa_state_status() == 0
     if args.phases:
@@ -276,6 +287,12 @@ def run_lsa_prefill(args, p, dev, rank, world):
                          "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "peak_kind": f"of {kind}",
                          "traffic": None, "algorithmic_flops_per_step": flops,
                          "gemm_phase_share_of_last_pass": gemm_us / max(sum(u for _, u, _w in ph), 1e-9)},
+            "codec": {"what": f"moa_quantize_rows / moa_dequantize_rows over the prompt's {flat.shape[0]} x {flat.shape[1]} "
+                              "bf16 activation rows (the server's first message), timed on their own",
+                      "quantize_ms": ms_q, "quantize_gbs": q_bytes / ms_q / 1e6, "quantize_frac_of_measured_hbm": q_bytes / ms_q / 1e6 / hbm,
+                      "dequantize_ms": ms_dq, "dequantize_gbs": q_bytes / ms_dq / 1e6,
+                      "dequantize_frac_of_measured_hbm": q_bytes / ms_dq / 1e6 / hbm,
+                      "algorithmic_bytes": q_bytes},
             "replicas": "replicas only: no data-path collective" if world > 1 else None}
     if rank == 0:
         print(json.dumps(line))

@@ -247,8 +247,8 @@ moa_status moa_verify_greedy(const int32_t *tok, const int32_t *parent, int32_t 
 moa_status moa_pack_tree(const int32_t *tok, const int32_t *parent, int64_t count, void *msg, void *stream);
 moa_status moa_unpack_tree(const void *msg, int64_t count, int32_t *tok, int32_t *parent, void *stream);
 /* 8-bit quantisation of activation rows (the E / E_kv tensors the server sends, Section 4.2). The paper names no
- * scheme; this one is symmetric with one fp32 scale per row: scale = max|x| / 127, code = round-half-even(x / scale)
- * in [-127, 127], decided in fp32; an all-zero row has scale 0 and codes 0. moa_dequantize_rows writes
+ * scheme; this one is symmetric with one fp32 scale per row: scale = max|x| / 127, code = round-half-even(x * r)
+ * in [-127, 127] with r = 127 / max|x| (one fp32 reciprocal per row, one fp32 product per element), decided in fp32; an all-zero row has scale 0 and codes 0. moa_dequantize_rows writes
  * code * scale in `dtype`.
  *   x / out  device [rows, width] of dtype (moa_dtype)    codes  device int8 [rows, width]    scales  device float [rows] */
 moa_status moa_quantize_rows(const void *x, int32_t dtype, int64_t rows, int32_t width, int8_t *codes, float *scales,

@@ -541,15 +541,16 @@ def unpack_tree(msg):
 def quantize_rows(x):
     """8-bit quantisation of activation rows (Section 4.2: the E and E_kv tensors are quantised to 8 bits).
     Reading (the paper gives no scheme): symmetric, one fp32 scale per row, scale = max|x| / 127,
-    code = round-half-even(x / scale) in [-127, 127]; an all-zero row has scale 0 and codes 0. The decision
-    is taken in fp32 (the precision both sides use). x [rows, width] -> (int8 codes, float32 scales)."""
+    code = round-half-even(x * (127 / max|x|)) in [-127, 127] -- one fp32 reciprocal per row, one fp32 product
+    per element; an all-zero row has scale 0 and codes 0. The decision is taken in fp32 (the precision both
+    sides use). x [rows, width] -> (int8 codes, float32 scales)."""
     x = np.asarray(x, np.float32)
     amax = np.max(np.abs(x), axis=-1).astype(np.float32)
     scale = (amax / np.float32(127.0)).astype(np.float32)
-    safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
-    q = np.rint((x / safe[:, None]).astype(np.float32))
+    nz = amax > 0
+    inv = np.where(nz, np.float32(127.0) / np.where(nz, amax, np.float32(1.0)), np.float32(0.0)).astype(np.float32)
+    q = np.rint((x * inv[:, None]).astype(np.float32))
     q = np.clip(q, -127, 127)
-    q = np.where(scale[:, None] > 0, q, 0)
     return q.astype(np.int8), scale
 
 

@@ -1689,12 +1689,15 @@ moa_status moa_dequantize_rows(const int8_t* codes, const float* scales, int64_t
   if (dtype != MOA_F32 && dtype != MOA_BF16) return MOA_ERR_DTYPE;
   if (rows < 0 || width <= 0 || rows > (1ll << 31)) return MOA_ERR_SHAPE;
   if (rows == 0) return MOA_OK;
-  const unsigned grid = blocks_for((size_t)rows * width, 256);
+  const int vec = (width % 16 == 0 && aligned16(codes) && aligned16(out)) ? 1 : 0;
+  const size_t total = (size_t)rows * width;
+  if ((vec ? total / 16 : total) > 256ull * 0x7fffffffull) return MOA_ERR_SHAPE;       // grid size
+  const unsigned grid = blocks_for(vec ? total / 16 : total, 256);
   if (dtype == MOA_F32)
-    launch_pdl(dequantize_rows_kernel<float>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width,
+    launch_pdl(dequantize_rows_kernel<float>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width, vec,
                (float*)out);
   else
-    launch_pdl(dequantize_rows_kernel<bf16>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width,
+    launch_pdl(dequantize_rows_kernel<bf16>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, codes, scales, (long long)rows, width, vec,
                (bf16*)out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;

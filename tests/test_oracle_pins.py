@@ -610,7 +610,7 @@ def test_pack_tree_layout_size_and_round_trip():
 
 
 def test_quantize_rows_bounds_and_fixed_points():
-    """Closed forms: |x - dequant| <= scale / 2; the row's largest magnitude maps to +-127 exactly; codes stay
+    """Closed forms: |x - dequant| <= scale / 2 (up to the fp32 rounding of the row's reciprocal); the row's largest magnitude maps to +-127 exactly; codes stay
     in [-127, 127]; an all-zero row gives zeros; quantising a dequantised row returns the same codes; a row that
     is already k * s for integers |k| <= 127 (max 127) is reproduced exactly."""
     rng = np.random.default_rng(4)
@@ -619,7 +619,7 @@ def test_quantize_rows_bounds_and_fixed_points():
     q, s = O.quantize_rows(x)
     d = O.dequantize_rows(q, s)
     assert q.dtype == np.int8 and s.dtype == np.float32 and int(np.abs(q.astype(int)).max()) == 127
-    assert np.all(np.abs(x - d) <= s[:, None] * 0.5 * (1 + 1e-6))
+    assert np.all(np.abs(x - d) <= s[:, None] * (0.5 + 1e-4))       # half a step, plus the rounding of the reciprocal
     am = np.argmax(np.abs(x), axis=1)
     rows = np.arange(50)
     assert np.all(np.abs(q[rows, am])[s > 0] == 127)
