@@ -499,6 +499,26 @@ def sequential_decode(dr: Drafter, prefix_toks, path_toks, caK, caV, B, tliK=Non
     return outs
 
 
+def drafter_prefill(dr: Drafter, toks, saK, saV, caK, caV, ca_limit=None):
+    """The drafter over a whole token sequence in one pass (Section 3.1.2: the causal SA mask and the CA layer
+    with its K-step-bounded mask, the pass the drafter is trained with): token i sits at position
+    len(saK) + i, sees the prefix and tokens 0..i in self-attention, and the first ca_limit[i] cached LLM
+    positions in cross-attention (None: all of them, the generation-time setting). TLI is not applied.
+    Returns (o_hat [n, E], K, V) with K, V the self-attention cache extended by the n tokens."""
+    c = dr.c
+    K = np.asarray(saK, F64).reshape(-1, c["sa_hkv"], c["head_dim"])
+    V = np.asarray(saV, F64).reshape(-1, c["sa_hkv"], c["head_dim"])
+    outs = []
+    for i, t in enumerate(toks):
+        lim = len(caK) if ca_limit is None else int(ca_limit[i])
+        e, q, k, v = dr.sa_qkv(int(t), K.shape[0])
+        K = np.concatenate([K, k[None]], 0)
+        V = np.concatenate([V, v[None]], 0)
+        x = dr.sa_block(e, q, K, V)
+        outs.append(dr.ca_block(x, caK[:lim], caV[:lim]))
+    return (np.stack(outs) if outs else np.zeros((0, c["d_model"]), F64)), K, V
+
+
 def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft, tliK=None, tliV=None):
     """Chain drafting (Algorithm 1, inner loop) with greedy choice: K_draft
     tokens, each the most probable continuation. Returns (tokens, logps)."""

@@ -630,3 +630,42 @@ def test_quantize_rows_bounds_and_fixed_points():
     y = (k * np.float32(0.25)).astype(np.float32)
     qy, sy = O.quantize_rows(y)
     assert np.array_equal(qy, k) and np.all(sy == np.float32(0.25)) and np.array_equal(O.dequantize_rows(qy, sy), y)
+
+
+# ------------------------------------------------------------------ whole-sequence drafter pass
+def test_drafter_prefill_equals_token_by_token_decoding_and_the_ca_mask_of_the_figure():
+    """With every cached LLM position visible the one-pass drafter equals plain causal decoding token by token;
+    with the K-step-bounded limits of the mask figure (K = 4 then K = 3 after a 3-token prompt) row j of the
+    output depends on LLM activation i exactly where the figure's cross-attention grid (as its caption states it)
+    is filled, and on token i exactly where the self-attention grid is."""
+    c = tiny_cfg()
+    dr = O.Drafter(c, tiny_weights(c))
+    rng = np.random.default_rng(9)
+    kv = rng.standard_normal((10, c["d_stack"]))
+    toks = [3, 7, 1, 20, 5, 11, 2, 9, 14, 6]
+    Kc, Vc = dr.ca_kv(kv)
+    empty = np.zeros((0, c["sa_hkv"], c["head_dim"]))
+    full, K, V = O.drafter_prefill(dr, toks, empty, empty, Kc, Vc)
+    seq = O.sequential_decode(dr, [], toks, Kc, Vc, 1)
+    assert np.allclose(full, np.stack([o["o_hat"] for o in seq]), atol=1e-12)
+    assert np.allclose(K[-1], seq[-1]["k"], atol=1e-12) and K.shape[0] == 10
+    # a prefix handed in as a cache gives the same as decoding it first
+    pre, Kp, Vp = O.drafter_prefill(dr, toks[:4], empty, empty, Kc, Vc)
+    rest, _, _ = O.drafter_prefill(dr, toks[4:], Kp, Vp, Kc, Vc)
+    assert np.allclose(np.concatenate([pre, rest]), full, atol=1e-12)
+    # the figure's limits: prompt rows causal, then K = 4 rows on 3 activations, then K = 3 rows on 7
+    limits = [1, 2, 3, 3, 3, 3, 3, 7, 7, 7]
+    base, _, _ = O.drafter_prefill(dr, toks, empty, empty, Kc, Vc, limits)
+    dep = np.zeros((10, 10), np.uint8)
+    for i in range(10):
+        kv2 = kv.copy(); kv2[i] += 1.0
+        K2, V2 = dr.ca_kv(kv2)
+        out2, _, _ = O.drafter_prefill(dr, toks, empty, empty, K2, V2, limits)
+        dep[:, i] = np.any(np.abs(out2 - base) > 1e-9, axis=-1)
+    assert np.array_equal(dep, read_grid("mask_ca_10x10.txt"))
+    dep_t = np.zeros((10, 10), np.uint8)
+    for i in range(10):
+        t2 = list(toks); t2[i] = (t2[i] + 1) % c["vocab"]
+        out2, _, _ = O.drafter_prefill(dr, t2, empty, empty, Kc, Vc, limits)
+        dep_t[:, i] = np.any(np.abs(out2 - base) > 1e-9, axis=-1)
+    assert np.array_equal(dep_t, read_grid("mask_sa_10x10.txt"))
