@@ -168,6 +168,20 @@ moa_status moa_lsa_forward(moa_ctx *ctx, moa_state *st, const void *h_stack, con
 moa_status moa_sa_append(moa_ctx *ctx, moa_state *st, const int32_t *tok, const int32_t *n_host, int32_t batch,
                          void *ws, size_t ws_bytes, void *stream);
 
+/* The drafter over whole token sequences in one pass (Section 3.1.2: self-attention with its causal mask over
+ * prompt + response, cross-attention into the cached LSA keys / values; the parallel pass the paper trains the
+ * drafter with, and a way to score many positions at once). Token i of sequence b sits at position sa_len[b] + i:
+ * it sees the prefix and tokens 0..i in self-attention; in cross-attention it sees the first ca_limit[row] cached
+ * positions (the K-step-bounded mask of the mask figure: the LLM activations available when that token is drafted),
+ * or all ca_len[b] of them when ca_limit is NULL (the generation-time setting).
+ *   tok        device int32 [sum n], sequences back to back;  n_host  HOST int32 [batch]
+ *   ca_limit   device int32 [sum n] or NULL; values in 0 .. ca_len[b], non-decreasing within a sequence
+ *   hidden_out T [sum n, E]: the drafter's output activation of every position (the LM head's input)
+ * Appends the tokens' self-attention keys / values to sa_k / sa_v and advances sa_len, as moa_sa_append does.
+ * Target Layer Inference and the LM head are not applied here. MOA_ERR_CAPACITY if the prefix would overflow. */
+moa_status moa_drafter_prefill(moa_ctx *ctx, moa_state *st, const int32_t *tok, const int32_t *n_host, int32_t batch,
+                               const int32_t *ca_limit, void *hidden_out, void *ws, size_t ws_bytes, void *stream);
+
 /* The same operation as moa_sa_append for callers that cannot provide a workspace because they cannot
  * allocate device memory at that point: code running between other components that have already handed
  * all device memory to their own pools, or a serving loop in which a cudaMalloc (a device-wide

@@ -20,7 +20,7 @@ using namespace moa;
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512, WMAP_MAX = 64 };
+enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -113,7 +113,8 @@ static Workspace plan_workspace(const moa_config& c, const moa_tli_config& t, si
   if (p.att_units < 10ll * p.draft_rows * hqmax) p.att_units = 10ll * p.draft_rows * hqmax;   // up to ten parts per (row, head)
   p.att_o = take(elt == 2 ? (size_t)p.att_units * c.head_dim * sizeof(float) : 256);   // split-KV partial outputs
   p.att_ml = take(elt == 2 ? (size_t)p.att_units * 2 * sizeof(float) : 256);           // their (max, sum)
-  p.q32 = take(elt == 2 ? (size_t)p.draft_rows * hqmax * c.head_dim * sizeof(float) : 256);   // draft-step queries, fp32
+  // draft-step queries in fp32; the whole-sequence drafter pass works in chunks of up to PREFILL_ROWS rows
+  p.q32 = take(elt == 2 ? (size_t)imax(p.draft_rows, imin(p.rows_cap, PREFILL_ROWS)) * hqmax * c.head_dim * sizeof(float) : 256);
   p.trace = take((2 * PM_MAX_OPS + 2) * sizeof(unsigned long long));   // phase timestamps of the last fused launch
   p.total = o;
   return p;
@@ -340,11 +341,13 @@ template <typename T>
 static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Workspace& p, int dh, const T* q,
                             const float* q32, int q_splits, size_t q_plane, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
                             int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
-                            int slots_ld, int nB, int n_slots, int rows_per_seq, T* out) {
+                            int slots_ld, int nB, int n_slots, int rows_per_seq, T* out,
+                            RowLimit lim = RowLimit{nullptr, 0, 0}) {
   if (R <= 0) return MOA_OK;
   if (sizeof(T) == 2) {
     AttnParams P;
     memset(&P, 0, sizeof(P));
+    P.lim = lim;
     const int nseq = R / rows_per_seq;
     P.q = (const bf16*)q; P.q32 = q32; P.q_splits = q_splits; P.q_plane = q_plane; P.q_ld = q_ld;
     P.hq = hq; P.hkv = hkv; P.group = hq / hkv;
@@ -379,10 +382,10 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   dim3 grid(R, hq);
   if (dh == 128)
     launch_pdl(attn_rows_kernel<T, 128>, dim3(grid), dim3(128), 0, s, q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
-                                                  slotsB, slots_ld, nB, rows_per_seq, out);
+                                                  slotsB, slots_ld, nB, rows_per_seq, lim, out);
   else
     launch_pdl(attn_rows_kernel<T, 64>, dim3(grid), dim3(128), 0, s, q, q_ld, hq, hkv, kA, vA, capA, posA_ld, lenA, nA_fixed, kB, vB, capB,
-                                                 slotsB, slots_ld, nB, rows_per_seq, out);
+                                                 slotsB, slots_ld, nB, rows_per_seq, lim, out);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -581,6 +584,96 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
   }
   if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
   launch_pdl(lse_topk_rows_kernel, dim3(R), dim3(256), 0, s, logits, V, B, topk_id, topk_logp);
+  MOA_CHECK_LAUNCH();
+  return MOA_OK;
+}
+
+// The drafter over whole token sequences in one pass (Section 3.1.2: causal SA mask, CA with an optional
+// K-step-bounded mask): sequence by sequence, in chunks of up to PREFILL_ROWS rows. A chunk's keys / values go
+// into the self-attention prefix cache first, so its attention reads them, and those of the earlier chunks, there.
+template <typename T>
+static moa_status drafter_prefill_t(moa_ctx* ctx, moa_state* st, const int* tok, const SeqSplit& split, const int* ca_limit,
+                                    void* hidden_out, char* ws, const Workspace& p, cudaStream_t s) {
+  const moa_config& c = ctx->c;
+  const moa_weights& w = ctx->w;
+  void* status_word = (char*)st->tree + ctx->tl.status;
+  const int E = c.d_model, dh = c.head_dim, V = c.vocab;
+  const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh, cq = c.ca_hq * dh, ckv = c.ca_hkv * dh;
+  float* xres = (float*)(ws + p.xres);
+  T* xn = (T*)(ws + p.xn);
+  T* narrow = (T*)(ws + p.narrow);
+  T* obuf = (T*)(ws + p.obuf);
+  float* q32 = sizeof(T) == 2 ? (float*)(ws + p.q32) : nullptr;
+  const int chunk_rows = imin(p.rows_cap, PREFILL_ROWS);
+  LinOut lo;
+  for (int b = 0; b < split.n_seq; ++b) {
+    const int n = split.off[b + 1] - split.off[b];
+    const int base = st->sa_len_host[b], ca_n = st->ca_len_host[b];
+    SeqSplit one;                         // rows of this call map to sequence b at offsets 0 .. n-1
+    one.n_seq = b + 1;
+    for (int i = 0; i <= 64; ++i) one.off[i] = i <= b ? 0 : n;
+    const T* sa_k = (const T*)st->sa_k + (size_t)b * c.max_ctx * nkv;
+    const T* sa_v = (const T*)st->sa_v + (size_t)b * c.max_ctx * nkv;
+    const T* ca_k = (const T*)st->ca_k + (size_t)b * c.max_ctx * ckv;
+    const T* ca_v = (const T*)st->ca_v + (size_t)b * c.max_ctx * ckv;
+    for (int r0 = 0; r0 < n; r0 += chunk_rows) {
+      const int R = imin(chunk_rows, n - r0);
+      const int g0 = split.off[b] + r0;                 // first row of the chunk in the caller's arrays
+      // ---- self-attention block ----
+      launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, tok + g0, V, (const T*)w.sa_norm1, E, c.rms_eps,
+                 xres, xn, lo_rows_of(sizeof(T), R));
+      MOA_CHECK_LAUNCH();
+      {
+        const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
+        const int N3[3] = {nq, nkv, nkv};
+        MOA_TRY(linear<T>(ctx, s, xn, R, E, 3, W3, N3, ws, p, &lo, status_word));
+      }
+      RopeRows rr;
+      memset(&rr, 0, sizeof(rr));
+      rr.mode = 1;
+      rr.max_ctx = c.max_ctx;
+      rr.split = one;
+      rr.row0 = r0;
+      launch_pdl(rope_store_kernel<T>, dim3(dim3(R, c.sa_hq + 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq,
+                 nq + nkv, c.sa_hq, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, (T*)st->sa_k, (T*)st->sa_v);
+      MOA_CHECK_LAUNCH();
+      // row i of the chunk sits at position base + r0 + i and sees positions 0 .. base + r0 + i
+      MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, c.sa_hq, c.sa_hkv, sa_k, sa_v, c.max_ctx, nkv, nullptr,
+                           base + r0 + R, base + r0 + R, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0, R, obuf,
+                           RowLimit{nullptr, base + r0 + 1, 1}));
+      {
+        const void* W1[1] = {w.sa_wo};
+        const int N1[1] = {E};
+        MOA_TRY(linear<T>(ctx, s, obuf, R, nq, 1, W1, N1, ws, p, &lo, status_word));
+      }
+      MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.sa_norm2, nullptr));
+      MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.sa_mlp, w.sa_wgate, w.sa_wup, w.sa_wdown, &lo, status_word));
+      // ---- cross-attention block ----
+      MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_normq, nullptr));
+      {
+        const void* W1[1] = {w.ca_wq};
+        const int N1[1] = {cq};
+        MOA_TRY(linear<T>(ctx, s, xn, R, E, 1, W1, N1, ws, p, &lo, status_word));
+        if (!q32) {
+          const size_t tot = (size_t)R * cq;
+          launch_pdl(sum_cast_kernel<T>, dim3(blocks_for(tot / 8, 256)), dim3(256), 0, s, lo.part, lo.splits, lo.plane, tot, narrow);
+          MOA_CHECK_LAUNCH();
+        }
+      }
+      MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32 ? lo.part : nullptr, lo.splits, lo.plane, cq, R, c.ca_hq, c.ca_hkv, ca_k, ca_v,
+                           c.max_ctx, ckv, nullptr, ca_n, ca_n, (const T*)nullptr, (const T*)nullptr, 0, nullptr, 0, 0, 0, R, obuf,
+                           RowLimit{ca_limit ? ca_limit + g0 : nullptr, 0, 0}));
+      {
+        const void* W1[1] = {w.ca_wo};
+        const int N1[1] = {E};
+        MOA_TRY(linear<T>(ctx, s, obuf, R, cq, 1, W1, N1, ws, p, &lo, status_word));
+      }
+      MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, w.ca_norm2, nullptr));
+      MOA_TRY(mlp_block<T>(s, ctx, p, ws, R, E, c.ca_mlp, w.ca_wgate, w.ca_wup, w.ca_wdown, &lo, status_word));
+      MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, nullptr, (T*)hidden_out + (size_t)g0 * E));
+    }
+  }
+  add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -1471,6 +1564,27 @@ moa_status moa_sa_append(moa_ctx* ctx, moa_state* st, const int32_t* tok, const 
   const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
   moa_status r = ctx->c.dtype == MOA_F32 ? sa_append_t<float>(ctx, st, tok, split, (char*)ws, p, (cudaStream_t)stream)
                                          : sa_append_t<bf16>(ctx, st, tok, split, (char*)ws, p, (cudaStream_t)stream);
+  if (r == MOA_OK)
+    for (int b = 0; b < batch; ++b) st->sa_len_host[b] += n_host[b];
+  return r;
+}
+
+moa_status moa_drafter_prefill(moa_ctx* ctx, moa_state* st, const int32_t* tok, const int32_t* n_host, int32_t batch,
+                               const int32_t* ca_limit, void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+  MOA_TRY(check_state(ctx, st, batch));
+  if (!n_host || !ws || !hidden_out) return MOA_ERR_NULL;
+  SeqSplit split;
+  MOA_TRY(make_split(n_host, batch, &split));
+  if (split.off[batch] > 0 && !tok) return MOA_ERR_NULL;
+  if (!aligned16(ws) || !aligned16(hidden_out)) return MOA_ERR_ALIGN;
+  for (int b = 0; b < batch; ++b)
+    if ((long long)st->sa_len_host[b] + n_host[b] > ctx->c.max_ctx) return MOA_ERR_CAPACITY;
+  const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
+  if (chunk < 1) return MOA_ERR_WORKSPACE;
+  const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
+  moa_status r = ctx->c.dtype == MOA_F32
+                     ? drafter_prefill_t<float>(ctx, st, tok, split, ca_limit, hidden_out, (char*)ws, p, (cudaStream_t)stream)
+                     : drafter_prefill_t<bf16>(ctx, st, tok, split, ca_limit, hidden_out, (char*)ws, p, (cudaStream_t)stream);
   if (r == MOA_OK)
     for (int b = 0; b < batch; ++b) st->sa_len_host[b] += n_host[b];
   return r;

@@ -28,6 +28,7 @@ struct AttnParams {
   int rows_per_seq;                      // query rows of one sequence (tree rows, or LSA layers)
   const bf16* kA; const bf16* vA; int capA; int posA_ld;   // segment A: (seq*capA + j)*posA_ld + g*DH
   const int* lenA; int nA_fixed;         // valid positions: lenA[seq] or the fixed count
+  RowLimit lim;                          // optional per-row bound on segment A (whole-sequence pass)
   const bf16* kB; const bf16* vB; int capB;                // segment B: ((seq*capB + slot)*hkv + g)*DH
   const int* slotsB; int slots_ld; int nB; int n_slots;    // row's ancestor slots [nB]; slots in use
   int n_split;                           // splits of segment A
@@ -99,6 +100,10 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     const int b0 = (int)(((long long)part * blocks) / P.n_split), b1 = (int)(((long long)(part + 1) * blocks) / P.n_split);
     k_begin = b0 * AT_KB;
     k_end = min(b1 * AT_KB, len);
+    if (P.lim.active()) {                  // limits do not decrease with the row: the tile's last row has the largest
+      const int q_last = min(Qn, (qt + 1) * QT) - 1;
+      k_end = min(k_end, P.lim.of(seq * P.rows_per_seq + q_last / P.group));
+    }
   } else {
     k_begin = 0;
     k_end = P.n_slots;
@@ -177,10 +182,12 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
 #pragma unroll
   for (int i = 0; i < DH / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
   int seqrow[2];                 // sequence-local row of each query (for the tree mask)
+  int limrow[2];                 // its bound on segment A
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const int qi = qt * QT + warp * 16 + gq + 8 * h;
     seqrow[h] = qi < Qn ? qi / P.group : 0;
+    limrow[h] = P.lim.active() ? P.lim.of(seq * P.rows_per_seq + seqrow[h]) : 0x7fffffff;
   }
 
   for (int blk = 0; blk < n_blocks; ++blk) {
@@ -226,6 +233,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
         const int h = e >> 1;
         bool ok = key < k_end;
         if (tree_part && ok) ok = (allow[seqrow[h]][key >> 6] >> (key & 63)) & 1ull;
+        if (!tree_part && ok) ok = key < limrow[h];
         const float v = ok ? s[nt][e] * P.scale_log2 : -INFINITY;
         s[nt][e] = v;
         mx[h] = fmaxf(mx[h], v);

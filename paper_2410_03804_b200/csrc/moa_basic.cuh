@@ -457,7 +457,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
                                                         const int* __restrict__ lenA, int nA_fixed,
                                                         const T* __restrict__ kB, const T* __restrict__ vB, int capB,
                                                         const int* __restrict__ slotsB, int slots_ld, int nB,
-                                                        int rows_per_seq, T* __restrict__ out) {
+                                                        int rows_per_seq, RowLimit lim, T* __restrict__ out) {
   pdl_trigger();
   pdl_wait();
   constexpr int VEC = DH / 32;
@@ -466,7 +466,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
   const int g = h / (hq / hkv);
   const int seq = r / rows_per_seq;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nA = lenA ? lenA[seq] : nA_fixed;
+  const int nA = min(lenA ? lenA[seq] : nA_fixed, lim.of(r));
   const float scale = rsqrtf((float)DH);
   float qv[VEC];
 #pragma unroll

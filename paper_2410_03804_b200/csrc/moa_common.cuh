@@ -66,6 +66,15 @@ __device__ __forceinline__ float block_max(float v, float* red) {
   return red[32];
 }
 
+// Optional per-row bound on the cache positions a query row may attend (causal / K-step-bounded masks of the
+// whole-sequence drafter pass): row r sees positions 0 .. of(r) - 1. Non-decreasing in r within a launch.
+struct RowLimit {
+  const int* ptr;      // explicit limits, one per row, or nullptr
+  int base, inc;       // else base + r * inc when inc != 0; no bound when inc == 0
+  __host__ __device__ bool active() const { return ptr != nullptr || inc != 0; }
+  __device__ __forceinline__ int of(int r) const { return ptr ? ptr[r] : (inc ? base + r * inc : 0x7fffffff); }
+};
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);

@@ -20,7 +20,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
 MOA_OK = 0
 
 EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
-           "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_tree_begin", "moa_draft_step",
+           "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_drafter_prefill", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_pack_tree", "moa_unpack_tree", "moa_quantize_rows", "moa_dequantize_rows", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count"]
 
@@ -106,6 +106,7 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_state_set_len.argtypes = [vp, C.POINTER(MoaState), i32, vp, i32, vp]
     lib.moa_lsa_forward.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, vp, sz, vp]
     lib.moa_sa_append.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, sz, vp]
+    lib.moa_drafter_prefill.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp, vp, vp, sz, vp]
     lib.moa_sa_append_static.argtypes = [vp, C.POINTER(MoaState), vp, vp, i32, vp]
     lib.moa_tree_begin.argtypes = [vp, C.POINTER(MoaState), vp, i32, vp]
     lib.moa_draft_step.argtypes = [vp, C.POINTER(MoaState), i32, vp, vp, vp, vp, sz, vp]
@@ -344,6 +345,19 @@ class MoA:
         assert tok.numel() == sum(n)
         _check(self.lib.moa_sa_append(self.h, C.byref(self.st), _ptr(tok), _host_i32(n), len(n), _ptr(self.ws),
                                       self.ws_bytes, _stream(stream)), "moa_sa_append")
+
+    def moa_drafter_prefill(self, tok: torch.Tensor, n, ca_limit=None, out=None, stream=None):
+        """The drafter over whole sequences in one pass: tok cuda int32 [sum n]; ca_limit cuda int32 [sum n] or
+        None. Returns hidden [sum n, E] and appends the tokens to the self-attention prefix."""
+        assert tok.is_cuda and tok.dtype == torch.int32 and tok.is_contiguous()
+        n = [int(v) for v in n]
+        assert tok.numel() == sum(n)
+        if ca_limit is not None:
+            assert ca_limit.is_cuda and ca_limit.dtype == torch.int32 and ca_limit.numel() == sum(n)
+        hid = out if out is not None else torch.empty((sum(n), self.cfg.d_model), dtype=self.dtype, device=self.device)
+        _check(self.lib.moa_drafter_prefill(self.h, C.byref(self.st), _ptr(tok), _host_i32(n), len(n), _ptr(ca_limit),
+                                            _ptr(hid), _ptr(self.ws), self.ws_bytes, _stream(stream)), "moa_drafter_prefill")
+        return hid
 
     def moa_sa_append_static(self, tok: torch.Tensor, n, stream=None):
         """moa_sa_append without a workspace: the library's fixed scratch array is used, nothing is allocated.
