@@ -491,6 +491,24 @@ def main():
     ms_verify = timed(vgraph.replay, 1) / args.steps
     vbytes = vz.numel() * vz.element_size()
     del vz
+    # the whole-sequence drafter pass (moa_drafter_prefill) over min(context, 2048) tokens of one sequence,
+    # every cached LLM position visible: timed on its own, not part of the step
+    n_pre = min(p.ctx, 2048)
+    pre_tok = synth.make_tokens(synth.scaled(p, batch=1), n_pre, tensor_index=44).reshape(-1).contiguous().to(dev)
+    pre_out = torch.empty((n_pre, p.d_model), dtype=p.torch_dtype, device=dev)
+
+    def prefill():
+        g.moa_state_set_len("sa", [0] * nb)
+        g.moa_drafter_prefill(pre_tok, [n_pre] + [0] * (nb - 1), out=pre_out)
+
+    prefill()
+    ms_prefill = timed(prefill, 3) / 3
+    g.moa_state_set_len("sa", lens)
+    assert g.moa_state_status() == 0
+    dh = p.head_dim
+    pre_flops = n_pre * 2.0 * ((p.sa_hq + 2 * p.sa_hkv) * dh * p.d_model + p.sa_hq * dh * p.d_model + 3 * p.d_model * p.sa_mlp
+                               + 2 * p.ca_hq * dh * p.d_model + 3 * p.d_model * p.ca_mlp) \
+        + 4.0 * dh * (p.sa_hq * n_pre * (n_pre + 1) / 2 + p.ca_hq * n_pre * p.ctx)
     clocks = sampler.stop()
     launches = launches_per_cycle * args.steps
     assert g.moa_state_status() == 0
@@ -533,6 +551,10 @@ def main():
                    "us": ms_verify * 1e3, "bytes": vbytes, "achieved_gbs": vbytes / ms_verify / 1e6,
                    "frac_of_measured": vbytes / ms_verify / 1e6 / peak,
                    "l2": "logits larger than L2" if vbytes > 126e6 else "logits fit in L2: not an HBM figure"},
+        "prefill": {"what": f"moa_drafter_prefill over {n_pre} tokens of one sequence (causal SA, CA over {p.ctx} cached positions), "
+                            "chunks of 256 rows, timed on its own",
+                    "ms": ms_prefill, "tokens_per_sec": n_pre / ms_prefill * 1e3, "algorithmic_flops": pre_flops,
+                    "tflops": pre_flops / ms_prefill / 1e9},
         "replicas": "replicas only: no data-path collective" if world > 1 else None,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
