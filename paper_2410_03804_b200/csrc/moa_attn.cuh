@@ -61,6 +61,12 @@ __device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// 2^x by the special-function unit (x <= 0 here; 2^-inf = 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 // Byte offset of (row, 16-byte chunk) in a tile of DH-wide bf16 rows, chunks XOR-swizzled by the row.
 template <int DH>
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
@@ -147,17 +153,21 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   }
   cp_async_commit();
 
+  // A thread always copies the same 16-byte column of the rows r0, r0 + rstep, ...: one pointer increment per row.
+  const int ld_c = threadIdx.x & (CH - 1), ld_r0 = threadIdx.x / CH, ld_rstep = blockDim.x / CH;
+  const size_t row_stride = tree_part ? (size_t)P.hkv * DH : (size_t)P.posA_ld;       // elements between two positions
+  const size_t seg_base = tree_part ? ((size_t)seq * P.capB * P.hkv + g) * DH : (size_t)seq * P.capA * P.posA_ld + g * DH;
+  const bf16* const k_src = (tree_part ? P.kB : P.kA) + seg_base + ld_c * 8;
+  const bf16* const v_src = (tree_part ? P.vB : P.vA) + seg_base + ld_c * 8;
   auto load_block = [&](int stage, int k0) {
     const uint32_t sK = sKV + stage * 2 * TILE_BYTES, sV = sK + TILE_BYTES;
-    for (int i = threadIdx.x; i < AT_KB * CH; i += blockDim.x) {
-      const int kr = i / CH, c = i - kr * CH;
-      const int j = k0 + kr;
-      const bool valid = j < k_end;
-      size_t off;
-      if (!tree_part) off = ((size_t)seq * P.capA + (valid ? j : 0)) * P.posA_ld + g * DH + c * 8;
-      else off = (((size_t)seq * P.capB + (valid ? j : 0)) * P.hkv + g) * DH + c * 8;
-      cp_async16(sK + tile_off<DH>(kr, c), (tree_part ? P.kB : P.kA) + off, valid);
-      cp_async16(sV + tile_off<DH>(kr, c), (tree_part ? P.vB : P.vA) + off, valid);
+    size_t off = (size_t)(k0 + ld_r0) * row_stride;
+    for (int kr = ld_r0; kr < AT_KB; kr += ld_rstep, off += (size_t)ld_rstep * row_stride) {
+      const bool valid = k0 + kr < k_end;
+      const size_t o = valid ? off : 0;                    // an address inside the segment; nothing is read when !valid
+      const uint32_t d = tile_off<DH>(kr, ld_c);
+      cp_async16(sK + d, k_src + o, valid);
+      cp_async16(sV + d, v_src + o, valid);
     }
   };
 
@@ -203,6 +213,9 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     float s[AT_KB / 8][4];
 #pragma unroll
     for (int nt = 0; nt < AT_KB / 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    // Tensor-core instructions that add into the same accumulator wait for one another, so they are issued
+    // accumulator by accumulator in rounds: the eight key tiles' fragments are loaded first, then every round
+    // touches each of the eight accumulators once.
 #pragma unroll
     for (int ks2 = 0; ks2 < KS / 2; ++ks2) {
       uint32_t ql0[4], ql1[4];         // QSPLIT: the low query terms of these two k-steps
@@ -211,32 +224,44 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
         ldsm_x4(sQlo + tile_off<DH>(row, (2 * ks2) * 2 + (lane >> 4)), ql0[0], ql0[1], ql0[2], ql0[3]);
         ldsm_x4(sQlo + tile_off<DH>(row, (2 * ks2 + 1) * 2 + (lane >> 4)), ql1[0], ql1[1], ql1[2], ql1[3]);
       }
+      uint32_t kb[AT_KB / 8][4];       // two k-steps: chunks 4*ks2 .. 4*ks2+3 of key row nt*8 + lane%8
 #pragma unroll
-      for (int nt = 0; nt < AT_KB / 8; ++nt) {
-        uint32_t b0, b1, b2, b3;       // two k-steps: chunks 4*ks2 .. 4*ks2+3 of key row nt*8 + lane%8
-        ldsm_x4(sK + tile_off<DH>(nt * 8 + (lane & 7), ks2 * 4 + (lane >> 3)), b0, b1, b2, b3);
-        mma_bf16_16816(s[nt], qf[2 * ks2], b0, b1);
-        mma_bf16_16816(s[nt], qf[2 * ks2 + 1], b2, b3);
-        if (QSPLIT) {
-          mma_bf16_16816(s[nt], ql0, b0, b1);
-          mma_bf16_16816(s[nt], ql1, b2, b3);
-        }
+      for (int nt = 0; nt < AT_KB / 8; ++nt)
+        ldsm_x4(sK + tile_off<DH>(nt * 8 + (lane & 7), ks2 * 4 + (lane >> 3)), kb[nt][0], kb[nt][1], kb[nt][2], kb[nt][3]);
+#pragma unroll
+      for (int nt = 0; nt < AT_KB / 8; ++nt) mma_bf16_16816(s[nt], qf[2 * ks2], kb[nt][0], kb[nt][1]);
+#pragma unroll
+      for (int nt = 0; nt < AT_KB / 8; ++nt) mma_bf16_16816(s[nt], qf[2 * ks2 + 1], kb[nt][2], kb[nt][3]);
+      if (QSPLIT) {
+#pragma unroll
+        for (int nt = 0; nt < AT_KB / 8; ++nt) mma_bf16_16816(s[nt], ql0, kb[nt][0], kb[nt][1]);
+#pragma unroll
+        for (int nt = 0; nt < AT_KB / 8; ++nt) mma_bf16_16816(s[nt], ql1, kb[nt][2], kb[nt][3]);
       }
     }
-    // scale, mask, block row max
+    // mask, block row max (of the raw scores: the scale is positive and goes into the exponent's multiply-add).
+    // Most blocks of a cache segment need no mask at all (warp-uniform test).
     float mx[2] = {-INFINITY, -INFINITY};
+    if (!tree_part && !P.lim.active() && k0 + AT_KB <= k_end) {
 #pragma unroll
-    for (int nt = 0; nt < AT_KB / 8; ++nt) {
+      for (int nt = 0; nt < AT_KB / 8; ++nt) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = k0 + nt * 8 + tq * 2 + (e & 1);
-        const int h = e >> 1;
-        bool ok = key < k_end;
-        if (tree_part && ok) ok = (allow[seqrow[h]][key >> 6] >> (key & 63)) & 1ull;
-        if (!tree_part && ok) ok = key < limrow[h];
-        const float v = ok ? s[nt][e] * P.scale_log2 : -INFINITY;
-        s[nt][e] = v;
-        mx[h] = fmaxf(mx[h], v);
+        for (int e = 0; e < 4; ++e) mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < AT_KB / 8; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int key = k0 + nt * 8 + tq * 2 + (e & 1);
+          const int h = e >> 1;
+          bool ok = key < k_end;
+          if (tree_part && ok) ok = (allow[seqrow[h]][key >> 6] >> (key & 63)) & 1ull;
+          if (!tree_part && ok) ok = key < limrow[h];
+          const float v = ok ? s[nt][e] : -INFINITY;
+          s[nt][e] = v;
+          mx[h] = fmaxf(mx[h], v);
+        }
       }
     }
     float corr[2], msub[2];
@@ -244,8 +269,8 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     for (int h = 0; h < 2; ++h) {
       mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
       mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
-      const float mn = fmaxf(m_run[h], mx[h]);
-      corr[h] = (m_run[h] == -INFINITY) ? 0.f : exp2f(m_run[h] - mn);
+      const float mn = fmaxf(m_run[h], mx[h] * P.scale_log2);       // log2 domain
+      corr[h] = (m_run[h] == -INFINITY) ? 0.f : ex2_approx(m_run[h] - mn);
       msub[h] = (mn == -INFINITY) ? 0.f : mn;      // a fully masked row keeps p = exp2(-inf) = 0
       m_run[h] = mn;
     }
@@ -253,37 +278,47 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     uint32_t pf[AT_KB / 16][4], pl[AT_KB / 16][4];      // probabilities as hi (+ lo with PSPLIT) bf16 terms
 #pragma unroll
     for (int nt = 0; nt < AT_KB / 8; ++nt) {
-      const float p0 = exp2f(s[nt][0] - msub[0]), p1 = exp2f(s[nt][1] - msub[0]);
-      const float p2 = exp2f(s[nt][2] - msub[1]), p3 = exp2f(s[nt][3] - msub[1]);
+      const float p0 = ex2_approx(fmaf(s[nt][0], P.scale_log2, -msub[0])), p1 = ex2_approx(fmaf(s[nt][1], P.scale_log2, -msub[0]));
+      const float p2 = ex2_approx(fmaf(s[nt][2], P.scale_log2, -msub[1])), p3 = ex2_approx(fmaf(s[nt][3], P.scale_log2, -msub[1]));
       rs[0] += p0 + p1;
       rs[1] += p2 + p3;
-      const bf16 h0 = __float2bfloat16_rn(p0), h1 = __float2bfloat16_rn(p1), h2 = __float2bfloat16_rn(p2),
-                 h3 = __float2bfloat16_rn(p3);
-      pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-      pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(__bfloat162float(h2), __bfloat162float(h3));
-      pl[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0 - __bfloat162float(h0), p1 - __bfloat162float(h1));
-      pl[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2 - __bfloat162float(h2), p3 - __bfloat162float(h3));
+      const uint32_t h01 = pack_bf16(p0, p1), h23 = pack_bf16(p2, p3);     // a bf16 is the upper half of a float
+      pf[nt >> 1][(nt & 1) * 2 + 0] = h01;
+      pf[nt >> 1][(nt & 1) * 2 + 1] = h23;
+      if (PSPLIT) {
+        pl[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xffff0000u));
+        pl[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xffff0000u));
+      }
     }
 #pragma unroll
     for (int h = 0; h < 2; ++h) l_run[h] = l_run[h] * corr[h] + rs[h];
+    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {      // the running maxima settle after a few blocks
 #pragma unroll
-    for (int i = 0; i < DH / 8; ++i) {
-      o[i][0] *= corr[0]; o[i][1] *= corr[0];
-      o[i][2] *= corr[1]; o[i][3] *= corr[1];
+      for (int i = 0; i < DH / 8; ++i) {
+        o[i][0] *= corr[0]; o[i][1] *= corr[0];
+        o[i][2] *= corr[1]; o[i][3] *= corr[1];
+      }
     }
-    // O += P V: k-steps of 16 keys, n-tiles of 8 output columns (two per ldmatrix)
+    // O += P V: k-steps of 16 keys, n-tiles of 8 output columns (two per ldmatrix); same issue order in rounds
+    // over independent accumulators, four ldmatrix results (eight output tiles) at a time
 #pragma unroll
     for (int kk = 0; kk < AT_KB / 16; ++kk) {
+      const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-      for (int n2 = 0; n2 < DH / 16; ++n2) {
-        uint32_t b0, b1, b2, b3;
-        const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        ldsm_x4_t(sV + tile_off<DH>(key, n2 * 2 + (lane >> 4)), b0, b1, b2, b3);
-        mma_bf16_16816(o[2 * n2], pf[kk], b0, b1);
-        mma_bf16_16816(o[2 * n2 + 1], pf[kk], b2, b3);
+      for (int n4 = 0; n4 < DH / 64; ++n4) {
+        uint32_t vb[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          ldsm_x4_t(sV + tile_off<DH>(key, (n4 * 4 + j) * 2 + (lane >> 4)), vb[j][0], vb[j][1], vb[j][2], vb[j][3]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mma_bf16_16816(o[2 * (n4 * 4 + j)], pf[kk], vb[j][0], vb[j][1]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mma_bf16_16816(o[2 * (n4 * 4 + j) + 1], pf[kk], vb[j][2], vb[j][3]);
         if (PSPLIT) {
-          mma_bf16_16816(o[2 * n2], pl[kk], b0, b1);
-          mma_bf16_16816(o[2 * n2 + 1], pl[kk], b2, b3);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_bf16_16816(o[2 * (n4 * 4 + j)], pl[kk], vb[j][0], vb[j][1]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_bf16_16816(o[2 * (n4 * 4 + j) + 1], pl[kk], vb[j][2], vb[j][3]);
         }
       }
     }
