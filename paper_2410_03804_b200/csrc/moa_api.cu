@@ -361,7 +361,8 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.q_tiles = (Qn + nwarps * 16 - 1) / (nwarps * 16);
     const int has_tree = (kB != nullptr && nB > 0) ? 1 : 0;
     const int blocks = imax(1, (max_len + AT_KB - 1) / AT_KB);
-    int n_split = imax(1, imin(blocks, (2 * ctx->sm_count) / imax(1, nseq * hkv * P.q_tiles)));
+    // cache parts plus the tree part fill one wave of two CTAs per SM: a few CTAs more would run alone afterwards
+    int n_split = imax(1, imin(blocks, (2 * ctx->sm_count) / imax(1, nseq * hkv * P.q_tiles) - has_tree));
     const long long per_part = (long long)R * hq;
     while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
     if (per_part * (n_split + has_tree) > p.att_units && n_split + has_tree > 1) return MOA_ERR_WORKSPACE;
