@@ -328,7 +328,7 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
   launch_pdl(attn_split_kernel<DH, QSPLIT, PSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
-    launch_pdl(attn_combine_kernel<DH>, dim3((nseq * P.rows_per_seq * P.hq + 7) / 8), dim3(256), 0, s, P.part_o, P.part_ml, P.n_parts,
+    launch_pdl(attn_combine_kernel<DH>, dim3(nseq * P.rows_per_seq * P.hq), dim3(CB_WARPS * 32), 0, s, P.part_o, P.part_ml, P.n_parts,
                nseq * P.rows_per_seq * P.hq, P.out, P.out_lo, P.hq);
     MOA_CHECK_LAUNCH();
   }

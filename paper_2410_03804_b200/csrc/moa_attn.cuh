@@ -364,18 +364,21 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   }
 }
 
-// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One warp per (row, head): the parts'
-// (max, sum) pairs are loaded one per lane, their weights travel by shuffles, and the partial outputs are read
-// four parts at a time, so the merge costs a few memory round trips whatever the number of parts.
+// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One CTA of CB_WARPS warps per (row, head):
+// every warp loads the parts' (max, sum) pairs (one per lane) for the common maximum and the weights, then adds
+// up its share of the partial outputs (parts w, w + CB_WARPS, ..., two in flight); the warps' sums meet in shared
+// memory. The merge is a chain of dependent memory round trips, so it is spread as wide as the parts allow.
+constexpr int CB_WARPS = 4;
+
 template <int DH>
-__global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o,
-                                                           const float* __restrict__ part_ml, int n_parts, int n_rh,
-                                                           bf16* __restrict__ out, int out_lo, int hq) {
+__global__ void __launch_bounds__(CB_WARPS * 32) attn_combine_kernel(const float* __restrict__ part_o,
+                                                                    const float* __restrict__ part_ml, int n_parts, int n_rh,
+                                                                    bf16* __restrict__ out, int out_lo, int hq) {
   pdl_trigger();
   pdl_wait();
-  const int lane = threadIdx.x & 31;
-  const int rh = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (rh >= n_rh) return;
+  __shared__ float acc_sh[CB_WARPS][DH];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int rh = blockIdx.x;
   float M = -INFINITY;
   for (int p0 = 0; p0 < n_parts; p0 += 32) {
     const float m = p0 + lane < n_parts ? part_ml[((size_t)rh * n_parts + p0 + lane) * 2] : -INFINITY;
@@ -393,26 +396,33 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restri
     }
     L += warp_sum(wl);
     const int np = min(32, n_parts - p0);
-    for (int pp = 0; pp < np; pp += 4) {
-      float x[4][DH / 32];
+    for (int pp = w; pp < np; pp += 2 * CB_WARPS) {          // this warp's parts of the group of 32, two at a time
+      float x[2][DH / 32];
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
+      for (int u = 0; u < 2; ++u)
 #pragma unroll
         for (int e = 0; e < DH / 32; ++e)
-          x[u][e] = pp + u < np ? part_o[((size_t)rh * n_parts + p0 + pp + u) * DH + lane + 32 * e] : 0.f;
+          x[u][e] = pp + u * CB_WARPS < np ? part_o[((size_t)rh * n_parts + p0 + pp + u * CB_WARPS) * DH + lane + 32 * e] : 0.f;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float wu = __shfl_sync(0xffffffffu, ww, (pp + u) & 31);
-        if (pp + u < np)
+      for (int u = 0; u < 2; ++u) {
+        const float wu = __shfl_sync(0xffffffffu, ww, (pp + u * CB_WARPS) & 31);
+        if (pp + u * CB_WARPS < np)
 #pragma unroll
           for (int e = 0; e < DH / 32; ++e) acc[e] += wu * x[u][e];
       }
     }
   }
+#pragma unroll
+  for (int e = 0; e < DH / 32; ++e) acc_sh[w][lane + 32 * e] = acc[e];
+  __syncthreads();
+  if (w != 0) return;
   const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll
   for (int e = 0; e < DH / 32; ++e) {
-    const float a = acc[e] * inv;
+    float a = 0.f;
+#pragma unroll
+    for (int k = 0; k < CB_WARPS; ++k) a += acc_sh[k][lane + 32 * e];      // fixed order
+    a *= inv;
     const bf16 h = __float2bfloat16_rn(a);
     out[(size_t)rh * DH + lane + 32 * e] = h;
     if (out_lo > 0) out[((size_t)out_lo * hq + rh) * DH + lane + 32 * e] = __float2bfloat16_rn(a - __bfloat162float(h));
