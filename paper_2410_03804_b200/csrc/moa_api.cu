@@ -328,8 +328,10 @@ static moa_status launch_attn_split(cudaStream_t s, const AttnParams& P, int nse
   launch_pdl(attn_split_kernel<DH, QSPLIT, PSPLIT>, dim3(grid), dim3(nwarps * 32), smem, s, P);
   MOA_CHECK_LAUNCH();
   if (P.n_parts > 1) {
-    launch_pdl(attn_combine_kernel<DH>, dim3(nseq * P.rows_per_seq * P.hq), dim3(CB_WARPS * 32), 0, s, P.part_o, P.part_ml, P.n_parts,
-               nseq * P.rows_per_seq * P.hq, P.out, P.out_lo, P.hq);
+    const int n_rh = nseq * P.rows_per_seq * P.hq;
+    const int share = P.n_parts >= CB_SHARE_FROM ? 1 : 0;
+    launch_pdl(attn_combine_kernel<DH>, dim3(share ? n_rh : (n_rh + CB_WARPS - 1) / CB_WARPS), dim3(CB_WARPS * 32), 0, s, P.part_o,
+               P.part_ml, P.n_parts, n_rh, share, P.out, P.out_lo, P.hq);
     MOA_CHECK_LAUNCH();
   }
   return MOA_OK;
@@ -373,8 +375,8 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.out = (bf16*)out;
     P.out_lo = lo_rows_of(sizeof(T), R);
     P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
-    // fp32 queries are split into two bf16 terms; the probabilities too when the output itself carries two terms
-    if (q32 && P.out_lo > 0)
+    // fp32 queries and the probabilities are split into two bf16 terms each
+    if (q32)
       return dh == 128 ? launch_attn_split<128, true, true>(s, P, nseq, nwarps) : launch_attn_split<64, true, true>(s, P, nseq, nwarps);
     if (q32)
       return dh == 128 ? launch_attn_split<128, true, false>(s, P, nseq, nwarps) : launch_attn_split<64, true, false>(s, P, nseq, nwarps);

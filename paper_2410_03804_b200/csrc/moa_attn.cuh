@@ -364,65 +364,78 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   }
 }
 
-// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p.  One CTA of CB_WARPS warps per (row, head):
-// every warp loads the parts' (max, sum) pairs (one per lane) for the common maximum and the weights, then adds
-// up its share of the partial outputs (parts w, w + CB_WARPS, ..., two in flight); the warps' sums meet in shared
-// memory. The merge is a chain of dependent memory round trips, so it is spread as wide as the parts allow.
+// out[row, head, :] = sum_p 2^(m_p - M) O_p / sum_p 2^(m_p - M) l_p. The merge is a chain of dependent memory
+// round trips, so it is spread as wide as the parts allow. share = 1 (many parts): one CTA of CB_WARPS warps per
+// (row, head); every warp loads the parts' (max, sum) pairs (one per lane) for the common maximum and the weights,
+// then adds up its share of the partial outputs (parts w, w + CB_WARPS, ..., two in flight) and the warps' sums
+// meet in shared memory. share = 0 (few parts): one warp per (row, head), CB_WARPS of them per CTA.
 constexpr int CB_WARPS = 4;
+constexpr int CB_SHARE_FROM = 9;       // parts from which a (row, head) gets a whole CTA
 
 template <int DH>
 __global__ void __launch_bounds__(CB_WARPS * 32) attn_combine_kernel(const float* __restrict__ part_o,
                                                                     const float* __restrict__ part_ml, int n_parts, int n_rh,
-                                                                    bf16* __restrict__ out, int out_lo, int hq) {
+                                                                    int share, bf16* __restrict__ out, int out_lo, int hq) {
   pdl_trigger();
   pdl_wait();
   __shared__ float acc_sh[CB_WARPS][DH];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int rh = blockIdx.x;
+  const int rh = share ? blockIdx.x : blockIdx.x * CB_WARPS + w;
+  const int first = share ? w : 0, step = share ? CB_WARPS : 1;      // this warp's parts: first, first + step, ...
+  const bool live = rh < n_rh;
   float M = -INFINITY;
-  for (int p0 = 0; p0 < n_parts; p0 += 32) {
-    const float m = p0 + lane < n_parts ? part_ml[((size_t)rh * n_parts + p0 + lane) * 2] : -INFINITY;
-    M = fmaxf(M, warp_max(m));
-  }
   float L = 0.f, acc[DH / 32];
 #pragma unroll
   for (int e = 0; e < DH / 32; ++e) acc[e] = 0.f;
-  for (int p0 = 0; p0 < n_parts; p0 += 32) {
-    float wl = 0.f, ww = 0.f;
-    if (p0 + lane < n_parts) {
-      const float2 ml = *reinterpret_cast<const float2*>(part_ml + ((size_t)rh * n_parts + p0 + lane) * 2);
-      ww = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
-      wl = ww * ml.y;
+  if (live) {
+    for (int p0 = 0; p0 < n_parts; p0 += 32) {
+      const float m = p0 + lane < n_parts ? part_ml[((size_t)rh * n_parts + p0 + lane) * 2] : -INFINITY;
+      M = fmaxf(M, warp_max(m));
     }
-    L += warp_sum(wl);
-    const int np = min(32, n_parts - p0);
-    for (int pp = w; pp < np; pp += 2 * CB_WARPS) {          // this warp's parts of the group of 32, two at a time
-      float x[2][DH / 32];
+    for (int p0 = 0; p0 < n_parts; p0 += 32) {
+      float wl = 0.f, ww = 0.f;
+      if (p0 + lane < n_parts) {
+        const float2 ml = *reinterpret_cast<const float2*>(part_ml + ((size_t)rh * n_parts + p0 + lane) * 2);
+        ww = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+        wl = ww * ml.y;
+      }
+      L += warp_sum(wl);
+      const int np = min(32, n_parts - p0);
+      for (int pp = first; pp < np; pp += 2 * step) {          // two parts in flight
+        float x[2][DH / 32];
 #pragma unroll
-      for (int u = 0; u < 2; ++u)
+        for (int u = 0; u < 2; ++u)
 #pragma unroll
-        for (int e = 0; e < DH / 32; ++e)
-          x[u][e] = pp + u * CB_WARPS < np ? part_o[((size_t)rh * n_parts + p0 + pp + u * CB_WARPS) * DH + lane + 32 * e] : 0.f;
+          for (int e = 0; e < DH / 32; ++e)
+            x[u][e] = pp + u * step < np ? part_o[((size_t)rh * n_parts + p0 + pp + u * step) * DH + lane + 32 * e] : 0.f;
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const float wu = __shfl_sync(0xffffffffu, ww, (pp + u * CB_WARPS) & 31);
-        if (pp + u * CB_WARPS < np)
+        for (int u = 0; u < 2; ++u) {
+          const float wu = __shfl_sync(0xffffffffu, ww, (pp + u * step) & 31);
+          if (pp + u * step < np)
 #pragma unroll
-          for (int e = 0; e < DH / 32; ++e) acc[e] += wu * x[u][e];
+            for (int e = 0; e < DH / 32; ++e) acc[e] += wu * x[u][e];
+        }
       }
     }
   }
+  if (share) {
 #pragma unroll
-  for (int e = 0; e < DH / 32; ++e) acc_sh[w][lane + 32 * e] = acc[e];
-  __syncthreads();
-  if (w != 0) return;
+    for (int e = 0; e < DH / 32; ++e) acc_sh[w][lane + 32 * e] = acc[e];
+    __syncthreads();
+    if (w != 0) return;
+#pragma unroll
+    for (int e = 0; e < DH / 32; ++e) {
+      float a = 0.f;
+#pragma unroll
+      for (int k = 0; k < CB_WARPS; ++k) a += acc_sh[k][lane + 32 * e];      // fixed order
+      acc[e] = a;
+    }
+  }
+  if (!live) return;
   const float inv = L > 0.f ? 1.f / L : 0.f;
 #pragma unroll
   for (int e = 0; e < DH / 32; ++e) {
-    float a = 0.f;
-#pragma unroll
-    for (int k = 0; k < CB_WARPS; ++k) a += acc_sh[k][lane + 32 * e];      // fixed order
-    a *= inv;
+    const float a = acc[e] * inv;
     const bf16 h = __float2bfloat16_rn(a);
     out[(size_t)rh * DH + lane + 32 * e] = h;
     if (out_lo > 0) out[((size_t)out_lo * hq + rh) * DH + lane + 32 * e] = __float2bfloat16_rn(a - __bfloat162float(h));
