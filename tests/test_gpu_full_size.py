@@ -85,6 +85,41 @@ def test_c2_llama8b_target_layer_inference_one_layer():
     g.close()
 
 
+def test_c2_whole_sequence_pass_sampled_positions(llama8b):
+    """Config 2's drafter over a 300-token sequence in one pass (two chunks at this workspace size) behind a
+    100-token prefix, with K-step-bounded cross-attention limits; the oracle computes sampled positions one by
+    one (first, last, both sides of the chunk boundary, two in between) and every appended key / value row."""
+    import numpy as np
+    from oracle import moa_oracle as O
+    p, w, g, oracles = llama8b
+    exact, _ = oracles
+    tol = H.tol_of(p)
+    caK, caV = synth.make_cache(p, "ca")
+    g.fill_cache("ca", caK.cuda(), caV.cuda())
+    g.moa_state_set_len("sa", [0])
+    n_pre, n = 100, 300
+    toks = synth.make_tokens(p, n_pre + n, tensor_index=45)[0]
+    g.moa_sa_append(toks[:n_pre].contiguous().cuda(), [n_pre])
+    lim = np.minimum(p.ctx, 400 + 7 * (np.arange(n) // 5)).astype(np.int32)      # segments of 5 tokens, growing view
+    hid = g.moa_drafter_prefill(toks[n_pre:].contiguous().cuda(), [n], ca_limit=torch.from_numpy(lim).cuda())
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0 and g.sa_len[:1].tolist() == [n_pre + n]
+    assert bool(torch.isfinite(hid.float()).all())
+    K, V = exact.sa_prefix(toks.tolist())
+    H.assert_rows_close(H.np32(g.sa_k[0, :n_pre + n].cpu()).reshape(n_pre + n, -1), K.reshape(n_pre + n, -1), tol, "SA K rows")
+    H.assert_rows_close(H.np32(g.sa_v[0, :n_pre + n].cpu()).reshape(n_pre + n, -1), V.reshape(n_pre + n, -1), tol, "SA V rows")
+    cK, cV = H.np32(caK[0]), H.np32(caV[0])
+    worst = 0.0
+    for i in (0, 57, 159, 160, 233, n - 1):
+        pos = n_pre + i
+        e, q, k, v = exact.sa_qkv(int(toks[pos]), pos)
+        x = exact.sa_block(e, q, K[:pos + 1], V[:pos + 1])
+        want = exact.ca_block(x, cK[:lim[i]], cV[:lim[i]])
+        worst = max(worst, H.assert_rows_close(H.np32(hid[i].cpu())[None], want[None], tol, f"prefill hidden position {i}"))
+    print(f"[prefill c2 full size] worst hidden {worst:.2e}")
+    g.moa_state_set_len("sa", [0])
+
+
 def test_c4_long_context_32k(llama8b):
     """Config 4: config 2's drafter over 32768-entry caches (both attentions), every row checked."""
     p2, w, g, oracles = llama8b
