@@ -236,11 +236,16 @@ static moa_status launch_ws_any(cudaStream_t s, const WsParams& P, int npad, int
     case 32: return launch_ws<32>(s, P, grid);
     case 64: return launch_ws<64>(s, P, grid);
     case 128: return launch_ws<128>(s, P, grid);
+    case 160: return launch_ws<160>(s, P, grid);
+    case 192: return launch_ws<192>(s, P, grid);
+    case 224: return launch_ws<224>(s, P, grid);
     default: return launch_ws<256>(s, P, grid);
   }
 }
 
-static inline int npad_for(int R) { return R <= 16 ? 16 : R <= 32 ? 32 : R <= 64 ? 64 : R <= 128 ? 128 : 256; }
+// MMA N (and activation-tile rows) for R rows: a power of two up to 128, then the next multiple of 32 -- a
+// smaller activation tile leaves room for more stages of the weight ring (R = 160: six stages instead of four).
+static inline int npad_for(int R) { return R <= 16 ? 16 : R <= 32 ? 32 : R <= 64 ? 64 : R <= 128 ? 128 : imin(256, (R + 31) / 32 * 32); }
 
 // Up to 128 rows, bf16 activations travel between kernels as two terms (hi + lo): the low-order rows start at this
 // row offset of every X buffer (0: single term). Producers and the GEMM that consumes them derive it from the same R.

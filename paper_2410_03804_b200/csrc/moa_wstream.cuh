@@ -27,7 +27,7 @@ constexpr int WS_BM = 128;         // weight rows per tile (MMA M)
 constexpr int WS_BK = 64;          // k elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int WS_THREADS = 320;     // TMA warp, MMA warp, eight epilogue warps (two per TMEM lane quadrant)
 constexpr int WS_W_BYTES = WS_BM * WS_BK * 2;
-constexpr int WS_SMEM_BUDGET = 200 * 1024;
+constexpr int WS_SMEM_BUDGET = 224 * 1024;    // ring of stages; 1.25 KB more for alignment and barriers stays under 227 KB
 constexpr long long WS_WAIT_CYCLES = 4000000000ll;   // ~2 s at boost clock
 
 struct WsParams {
@@ -164,7 +164,8 @@ template <int NPAD>
 __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __grid_constant__ WsParams P) {
   constexpr int STAGES = ws_stages(NPAD);
   constexpr int STAGE_BYTES = ws_stage_bytes(NPAD);
-  constexpr uint32_t TMEM_COLS = (2 * NPAD) < 32 ? 32 : (2 * NPAD);
+  // two accumulators of NPAD columns; the allocation is a power of two of at least 32 columns
+  constexpr uint32_t TMEM_COLS = (2 * NPAD) <= 32 ? 32 : (2 * NPAD) <= 64 ? 64 : (2 * NPAD) <= 128 ? 128 : (2 * NPAD) <= 256 ? 256 : 512;
   constexpr uint32_t IDESC = umma_idesc_bf16(WS_BM, NPAD);
 
   extern __shared__ uint8_t smem_raw[];
