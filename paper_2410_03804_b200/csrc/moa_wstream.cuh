@@ -354,37 +354,59 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] += w2[i];
           }
-#pragma unroll 1
-          for (int i = 0; i < 16; ++i) {
-            const int r = c0 + i;
-            if (r >= P.R) break;
-            float val = valid ? v[i] : -INFINITY;
-            int id = nrow;
-            const float wmax = warp_max(val);
-            const float e = (valid && wmax > -INFINITY) ? __expf(val - wmax) : 0.f;
-            const float wsum = warp_sum(e);
-            // bitonic sort of the 32 (value, id) pairs: best (largest value, then smallest id) ends in lane 0
+          // two activation rows at a time: their shuffle chains are independent and interleave
 #pragma unroll
-            for (int k = 2; k <= 32; k <<= 1) {
+          for (int i = 0; i < 16; i += 2) {
+            if (c0 + i < P.R) {
+              float val[2], wmax[2], wsum[2];
+              int id[2];
 #pragma unroll
-              for (int jj = k >> 1; jj > 0; jj >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, val, jj);
-                const int oi = __shfl_xor_sync(0xffffffffu, id, jj);
-                const bool lower = (lane & jj) == 0;
-                const bool up = (lane & k) == 0;
-                const bool want_better = lower == up;
-                const bool other_better = ranks_before(ov, oi, val, id);
-                if (want_better == other_better) { val = ov; id = oi; }
+              for (int u = 0; u < 2; ++u) {
+                val[u] = valid ? v[i + u] : -INFINITY;
+                id[u] = nrow;
+                wmax[u] = val[u];
               }
-            }
-            const size_t at = (size_t)r * n_sub + sub;       // row-major over slices: the merge reads them coalesced
-            if (lane < B) {
-              P.c_val[at * B + lane] = val;
-              P.c_id[at * B + lane] = id;
-            }
-            if (lane == 0) {
-              P.p_max[at] = wmax;
-              P.p_sum[at] = wsum;
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u) wmax[u] = fmaxf(wmax[u], __shfl_xor_sync(0xffffffffu, wmax[u], o));
+              }
+#pragma unroll
+              for (int u = 0; u < 2; ++u) wsum[u] = (valid && wmax[u] > -INFINITY) ? __expf(val[u] - wmax[u]) : 0.f;
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u) wsum[u] += __shfl_xor_sync(0xffffffffu, wsum[u], o);
+              }
+              // bitonic sort of the 32 (value, id) pairs: best (largest value, then smallest id) ends in lane 0
+#pragma unroll
+              for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+                for (int jj = k >> 1; jj > 0; jj >>= 1) {
+                  const bool want_better = ((lane & jj) == 0) == ((lane & k) == 0);
+#pragma unroll
+                  for (int u = 0; u < 2; ++u) {
+                    const float ov = __shfl_xor_sync(0xffffffffu, val[u], jj);
+                    const int oi = __shfl_xor_sync(0xffffffffu, id[u], jj);
+                    if (want_better == ranks_before(ov, oi, val[u], id[u])) { val[u] = ov; id[u] = oi; }
+                  }
+                }
+              }
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                const int r = c0 + i + u;
+                if (r < P.R) {
+                  const size_t at = (size_t)r * n_sub + sub;       // row-major over slices: the merge reads them coalesced
+                  if (lane < B) {
+                    P.c_val[at * B + lane] = val[u];
+                    P.c_id[at * B + lane] = id[u];
+                  }
+                  if (lane == 0) {
+                    P.p_max[at] = wmax[u];
+                    P.p_sum[at] = wsum[u];
+                  }
+                }
+              }
             }
           }
         }
