@@ -27,6 +27,7 @@ constexpr int WS_BM = 128;         // weight rows per tile (MMA M)
 constexpr int WS_BK = 64;          // k elements per stage: 128 bytes of bf16 = one swizzle row
 constexpr int WS_THREADS = 320;     // TMA warp, MMA warp, eight epilogue warps (two per TMEM lane quadrant)
 constexpr int WS_W_BYTES = WS_BM * WS_BK * 2;
+constexpr int EPI_U = 4;          // activation rows the LM-head epilogue sorts side by side
 constexpr int WS_SMEM_BUDGET = 224 * 1024;    // ring of stages; 1.25 KB more for alignment and barriers stays under 227 KB
 constexpr long long WS_WAIT_CYCLES = 4000000000ll;   // ~2 s at boost clock
 
@@ -354,14 +355,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] += w2[i];
           }
-          // two activation rows at a time: their shuffle chains are independent and interleave
+          // EPI_U activation rows at a time: their shuffle chains are independent and interleave
 #pragma unroll
-          for (int i = 0; i < 16; i += 2) {
+          for (int i = 0; i < 16; i += EPI_U) {
             if (c0 + i < P.R) {
-              float val[2], wmax[2], wsum[2];
-              int id[2];
+              float val[EPI_U], wmax[EPI_U], wsum[EPI_U];
+              int id[EPI_U];
 #pragma unroll
-              for (int u = 0; u < 2; ++u) {
+              for (int u = 0; u < EPI_U; ++u) {
                 val[u] = valid ? v[i + u] : -INFINITY;
                 id[u] = nrow;
                 wmax[u] = val[u];
@@ -369,14 +370,14 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
 #pragma unroll
               for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-                for (int u = 0; u < 2; ++u) wmax[u] = fmaxf(wmax[u], __shfl_xor_sync(0xffffffffu, wmax[u], o));
+                for (int u = 0; u < EPI_U; ++u) wmax[u] = fmaxf(wmax[u], __shfl_xor_sync(0xffffffffu, wmax[u], o));
               }
 #pragma unroll
-              for (int u = 0; u < 2; ++u) wsum[u] = (valid && wmax[u] > -INFINITY) ? __expf(val[u] - wmax[u]) : 0.f;
+              for (int u = 0; u < EPI_U; ++u) wsum[u] = (valid && wmax[u] > -INFINITY) ? __expf(val[u] - wmax[u]) : 0.f;
 #pragma unroll
               for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-                for (int u = 0; u < 2; ++u) wsum[u] += __shfl_xor_sync(0xffffffffu, wsum[u], o);
+                for (int u = 0; u < EPI_U; ++u) wsum[u] += __shfl_xor_sync(0xffffffffu, wsum[u], o);
               }
               // bitonic sort of the 32 (value, id) pairs: best (largest value, then smallest id) ends in lane 0
 #pragma unroll
@@ -385,7 +386,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
                 for (int jj = k >> 1; jj > 0; jj >>= 1) {
                   const bool want_better = ((lane & jj) == 0) == ((lane & k) == 0);
 #pragma unroll
-                  for (int u = 0; u < 2; ++u) {
+                  for (int u = 0; u < EPI_U; ++u) {
                     const float ov = __shfl_xor_sync(0xffffffffu, val[u], jj);
                     const int oi = __shfl_xor_sync(0xffffffffu, id[u], jj);
                     if (want_better == ranks_before(ov, oi, val[u], id[u])) { val[u] = ov; id[u] = oi; }
@@ -393,7 +394,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
                 }
               }
 #pragma unroll
-              for (int u = 0; u < 2; ++u) {
+              for (int u = 0; u < EPI_U; ++u) {
                 const int r = c0 + i + u;
                 if (r < P.R) {
                   const size_t at = (size_t)r * n_sub + sub;       // row-major over slices: the merge reads them coalesced
