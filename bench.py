@@ -47,9 +47,9 @@ def algorithmic_bytes(p) -> dict:
     return dict(step=(sa_w + ca_w + lm + caches + tli) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (wstream_gemm_kernel<16>, mode 1) from the ncu
+# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (wstream_gemm_kernel<32>, mode 1) from the ncu
 # capture summarised in profiles/lm_head_wstream_c2.md; set back to None when that kernel changes.
-LM_HEAD_TRAFFIC = {"c2": 1051065600 + 12941056}
+LM_HEAD_TRAFFIC = {"c2": 1051208704 + 3780352}
 
 
 class ClockSampler:
