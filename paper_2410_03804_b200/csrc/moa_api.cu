@@ -92,7 +92,7 @@ static Workspace plan_workspace(const moa_config& c, const moa_tli_config& t, si
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 255) / 256 * 256; return at; };
   p.xres = take((size_t)p.rows_cap * dmax * sizeof(float));      // residual stream, fp32
-  const size_t xpad = 128;                                       // an X buffer's low-order half starts up to 128 rows in
+  const size_t xpad = 256;                                       // an X buffer's low-order rows start up to 256 rows in
   p.xn = take(((size_t)p.rows_cap + xpad) * dmax * elt);         // normalised GEMM operand, T
   p.part = take((size_t)p.part_rows * p.wide * sizeof(float));   // GEMM outputs: K-split partial planes, fp32
   p.narrow = take(((size_t)p.rows_cap + xpad) * narrow * elt);   // q|k|v or silu(gate)*up, T
@@ -213,24 +213,32 @@ struct LinOut {          // where a linear layer left its result: `splits` fp32 
   int ld;
 };
 
-template <int NPAD>
+template <int NPAD, bool XS2 = false>
 static moa_status launch_ws(cudaStream_t s, const WsParams& P, int grid) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(wstream_gemm_kernel<NPAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ws_smem_bytes(NPAD));
+    cudaError_t e = cudaFuncSetAttribute(wstream_gemm_kernel<NPAD, XS2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ws_smem_bytes(NPAD, XS2));
     if (e != cudaSuccess) {
       snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
       return MOA_ERR_CUDA;
     }
     attr_set = true;
   }
-  launch_pdl(wstream_gemm_kernel<NPAD>, dim3(grid), dim3(WS_THREADS), ws_smem_bytes(NPAD), s, P);
+  launch_pdl(wstream_gemm_kernel<NPAD, XS2>, dim3(grid), dim3(WS_THREADS), ws_smem_bytes(NPAD, XS2), s, P);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
 
-static moa_status launch_ws_any(cudaStream_t s, const WsParams& P, int npad, int grid) {
+static moa_status launch_ws_any(cudaStream_t s, const WsParams& P, int npad, int grid, bool xs2 = false) {
+  if (xs2) {                       // two-term activations of more than 128 rows
+    switch (npad) {
+      case 160: return launch_ws<160, true>(s, P, grid);
+      case 192: return launch_ws<192, true>(s, P, grid);
+      case 224: return launch_ws<224, true>(s, P, grid);
+      default: return launch_ws<256, true>(s, P, grid);
+    }
+  }
   switch (npad) {
     case 16: return launch_ws<16>(s, P, grid);
     case 32: return launch_ws<32>(s, P, grid);
@@ -249,7 +257,13 @@ static inline int npad_for(int R) { return R <= 16 ? 16 : R <= 32 ? 32 : R <= 64
 
 // Up to 128 rows, bf16 activations travel between kernels as two terms (hi + lo): the low-order rows start at this
 // row offset of every X buffer (0: single term). Producers and the GEMM that consumes them derive it from the same R.
-static inline int lo_rows_of(size_t elt, int R) { return (elt == 2 && R > 0 && R <= 128) ? npad_for(R) : 0; }
+// (129 to 256 rows: the low-order rows start at row 256 and the GEMM multiplies the two terms one after the other
+// into the same accumulator; more rows: a single term.)
+constexpr int LO_ROW_WIDE = 256;
+static inline int lo_rows_of(size_t elt, int R) {
+  if (elt != 2 || R <= 0 || R > 256) return 0;
+  return R <= 128 ? npad_for(R) : LO_ROW_WIDE;
+}
 
 static bool fast_shape(const moa_ctx* ctx, int K, int nseg, const void* const* W) {
   if (!ctx->fast || K % WS_BK != 0) return false;
@@ -292,17 +306,19 @@ static moa_status linear(moa_ctx* ctx, cudaStream_t s, const T* X, int R, int K,
     P.status = (int*)status_word;
     const int nblk = (R + 255) / 256;
     const int lo = lo_rows_of(sizeof(T), R);
-    P.xsplit = lo > 0 ? 1 : 0;
+    const bool wide = lo == LO_ROW_WIDE && R > 128;      // two activation tiles per stage instead of one tile of both terms
+    P.xsplit = (lo > 0 && !wide) ? 1 : 0;
+    P.lo_row = lo;
     P.splits = pick_splits(tiles * nblk, P.kb_total, R, p.part_rows, ctx->sm_count);
     out->splits = P.splits;
     for (int r0 = 0; r0 < R; r0 += 256) {
       const int rows = imin(256, R - r0);
-      const int npad = lo > 0 ? 2 * lo : npad_for(rows);
+      const int npad = (lo > 0 && !wide) ? 2 * lo : npad_for(rows);
       if (!encode_map(ctx, &P.tmX, (const bf16*)X + (size_t)r0 * K, lo > 0 ? lo + rows : rows, K, npad)) return MOA_ERR_CUDA;
       P.R = rows;
       P.out = part + (size_t)r0 * ntot;
       const int units = tiles * P.splits;
-      MOA_TRY(launch_ws_any(s, P, npad, imin(units, ctx->sm_count)));
+      MOA_TRY(launch_ws_any(s, P, npad, imin(units, ctx->sm_count), wide));
     }
     return MOA_OK;
   }
@@ -566,11 +582,13 @@ static moa_status lm_head_t(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.c_id = (int*)(ws + p.cid);
     P.status = (int*)status_word;
     const int lo = lo_rows_of(sizeof(T), R);
-    P.xsplit = lo > 0 ? 1 : 0;
-    const int npad = lo > 0 ? 2 * lo : npad_for(R);
+    const bool wide = lo == LO_ROW_WIDE && R > 128;
+    P.xsplit = (lo > 0 && !wide) ? 1 : 0;
+    P.lo_row = lo;
+    const int npad = (lo > 0 && !wide) ? 2 * lo : npad_for(R);
     if (!encode_map(ctx, &P.tmX, xn, lo > 0 ? lo + R : R, E, npad)) return MOA_ERR_CUDA;
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s);
-    MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count)));
+    MOA_TRY(launch_ws_any(s, P, npad, imin(P.tiles_total, ctx->sm_count), wide));
     if (timed) cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n++ + 1], s);
     MergeScratch sc;
     sc.ms = (float*)(ws + p.mrg_ms);

@@ -44,6 +44,7 @@ struct WsParams {
   int splits;              // K splits per tile
   int mode;                // 0: fp32 partials, 1: LM-head partial top-B
   int xsplit;              // activations carried as two bf16 terms: rows [0, R) hi, rows [NPAD/2, NPAD/2 + R) lo
+  int lo_row;              // XS2 kernels: first row of the low-order terms in the activation buffer
   int ldo;                 // mode 0: columns of one partial plane
   float* out;              // mode 0: plane `split` starts at out + split * plane; row r, column c at [r * ldo + c]
   size_t plane;            // mode 0: elements between two partial planes
@@ -55,11 +56,16 @@ struct WsParams {
   int* status;             // device status word (may be nullptr)
 };
 
-__host__ __device__ constexpr int ws_stage_bytes(int npad) { return WS_W_BYTES + npad * WS_BK * 2; }
-__host__ __device__ constexpr int ws_stages(int npad) {
-  return (WS_SMEM_BUDGET / ws_stage_bytes(npad)) > 12 ? 12 : (WS_SMEM_BUDGET / ws_stage_bytes(npad));
+// xs2: the stage holds two activation tiles (high-order and low-order terms), multiplied one after the other into
+// the same accumulator -- the two-term form for more than 128 rows, where the terms no longer fit side by side
+// in the N of one instruction.
+__host__ __device__ constexpr int ws_stage_bytes(int npad, bool xs2 = false) { return WS_W_BYTES + (xs2 ? 2 : 1) * npad * WS_BK * 2; }
+__host__ __device__ constexpr int ws_stages(int npad, bool xs2 = false) {
+  return (WS_SMEM_BUDGET / ws_stage_bytes(npad, xs2)) > 12 ? 12 : (WS_SMEM_BUDGET / ws_stage_bytes(npad, xs2));
 }
-__host__ __device__ constexpr int ws_smem_bytes(int npad) { return ws_stages(npad) * ws_stage_bytes(npad) + 1024 + 256; }
+__host__ __device__ constexpr int ws_smem_bytes(int npad, bool xs2 = false) {
+  return ws_stages(npad, xs2) * ws_stage_bytes(npad, xs2) + 1024 + 256;
+}
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -161,10 +167,11 @@ __device__ __forceinline__ bool ranks_before(float va, int ia, float vb, int ib)
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int NPAD>
+template <int NPAD, bool XS2>
 __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __grid_constant__ WsParams P) {
-  constexpr int STAGES = ws_stages(NPAD);
-  constexpr int STAGE_BYTES = ws_stage_bytes(NPAD);
+  constexpr int STAGES = ws_stages(NPAD, XS2);
+  constexpr int STAGE_BYTES = ws_stage_bytes(NPAD, XS2);
+  constexpr int X_BYTES = NPAD * WS_BK * 2;       // one activation tile
   // two accumulators of NPAD columns; the allocation is a power of two of at least 32 columns
   constexpr uint32_t TMEM_COLS = (2 * NPAD) <= 32 ? 32 : (2 * NPAD) <= 64 ? 64 : (2 * NPAD) <= 128 ? 128 : (2 * NPAD) <= 256 ? 256 : 512;
   constexpr uint32_t IDESC = umma_idesc_bf16(WS_BM, NPAD);
@@ -241,8 +248,10 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
         for (int u = blockIdx.x; u < units && i2 < pre; u += gridDim.x) {
           int seg, n0, kb0, kb1, split, tile;
           decode(u, seg, n0, kb0, kb1, split, tile);
-          for (int kb = kb0; kb < kb1 && i2 < pre; ++kb, ++i2)
+          for (int kb = kb0; kb < kb1 && i2 < pre; ++kb, ++i2) {
             tma_load_2d(base + i2 * STAGE_BYTES + WS_W_BYTES, &P.tmX, kb * WS_BK, 0, full_bar(i2));
+            if (XS2) tma_load_2d(base + i2 * STAGE_BYTES + WS_W_BYTES + X_BYTES, &P.tmX, kb * WS_BK, P.lo_row, full_bar(i2));
+          }
         }
       }
       uint32_t it = 0;
@@ -260,6 +269,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
           const uint32_t dst = base + s * STAGE_BYTES;
           tma_load_2d(dst, tw, kb * WS_BK, n0, full_bar(s));
           tma_load_2d(dst + WS_W_BYTES, &P.tmX, kb * WS_BK, 0, full_bar(s));
+          if (XS2) tma_load_2d(dst + WS_W_BYTES + X_BYTES, &P.tmX, kb * WS_BK, P.lo_row, full_bar(s));
         }
       }
       if (!ok) {
@@ -299,6 +309,11 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
           for (int kk = 0; kk < WS_BK / 16; ++kk) {
             // advancing 16 k-elements = 32 bytes inside the swizzled row: +2 in the descriptor's 16-byte units
             tc_mma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, IDESC, (kb > kb0 || kk > 0) ? 1u : 0u);
+          }
+          if (XS2) {                       // W x = W hi + W lo, the second product into the same accumulator
+            const uint64_t ldesc = umma_desc_sw128(wa + WS_W_BYTES + X_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < WS_BK / 16; ++kk) tc_mma_bf16(d_tmem, adesc + 2u * kk, ldesc + 2u * kk, IDESC, 1u);
           }
           tc_commit(empty_bar(s));       // frees the stage once these MMAs have read it
         }
