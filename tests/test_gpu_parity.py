@@ -3,10 +3,10 @@
 Tolerances (stated by the benchmark spec): hidden states and log-probabilities within
 max-abs 1e-4 (fp32 path) / 2e-2 (bf16 path) of the row's max |value|; token ids and tree structure
 bit-exact except where the oracle's competing log-probabilities differ by less than the tie window
-(1e-3 on the fp32 path; helpers.tie_window derives the bf16 ones). bf16 forwards of up to 128 rows carry their
-activations as two bf16 terms, so their top-B decisions are compared with the unrounded fp64 oracle directly;
-larger bf16 forwards (plain 16-bit activations) with the oracle in its bf16-storage mode, their values with the
-unrounded oracle walking the same tree.
+(1e-3 on the fp32 path; helpers.tie_window derives the bf16 ones). bf16 forwards of up to 256 rows (every draft
+step) carry their activations as two bf16 terms, so their top-B decisions are compared with the unrounded fp64
+oracle directly; larger bf16 passes (plain 16-bit activations) would be compared with the oracle in its
+bf16-storage mode, their values with the unrounded oracle.
 """
 import numpy as np
 import pytest

@@ -63,7 +63,7 @@ def test_prefill_c1_fp32_with_and_without_limits():
 @pytest.mark.parametrize("dtype,use_limits", [("bf16", True), ("bf16", False), ("f32", True)])
 def test_prefill_reduced_llama_shape_ragged_batch(dtype, use_limits):
     """Reduced Llama-3 shape, three sequences of different lengths over different prefixes; the longest one spans
-    two chunks of 256 rows (one of them in the two-term regime of up to 128 rows)."""
+    two chunks of 256 rows (one with the two activation terms side by side in one tile, one with two tiles)."""
     p = synth.scaled(synth.PRESETS["c2"], d_model=512, n_stack=5, d_stack=384, vocab=5003, lsa_hq=8, lsa_hkv=2,
                      lsa_mlp=768, sa_hq=8, sa_hkv=2, sa_mlp=64, ca_hq=8, ca_hkv=4, ca_mlp=896, ctx=90, batch=3,
                      tree_topk=5, tree_depth=3, tree_keep=12, dtype=dtype, lsa_tokens=4)
