@@ -135,8 +135,8 @@ moa_status moa_tli_configure(moa_ctx *ctx, const moa_tli_config *cfg, const moa_
 
 /* Options. MOA_OPT_FUSED_STEP (bf16 only): run moa_draft_step, and moa_lsa_forward passes of any size, as ONE
  * persistent cooperative kernel (phases separated by grid-wide barriers, weights prefetched across phases,
- * activations carried as two bf16 terms) instead of a chain of launches. Same results within tolerance, closer
- * to the fp64 values; off by default because the chain is faster at small row counts. */
+ * activations carried as two bf16 terms up to 128 rows) instead of a chain of launches. Same results within
+ * tolerance; off by default because the chain is faster at small row counts. */
 #define MOA_OPT_FUSED_STEP 1
 moa_status moa_set_option(moa_ctx *ctx, int32_t option, int32_t value);
 
