@@ -129,16 +129,17 @@ def test_c4_long_context_32k(llama8b):
 
 
 def test_c5_llama70b_batch16_sampled_sequences():
-    """Config 5: d 8192, 80 layers, 64/8 heads, batch 16 x context 4096. The oracle walks sequences 0 and 15
-    (first and last of the batch) row by row and two LSA tokens of each; the other 14 sequences are checked
+    """Config 5: d 8192, 80 layers, 64/8 heads, batch 16 x context 4096. The oracle walks sequences 0, 2 and 15
+    (first and last of the batch, and one whose hidden states were outside the bound while 160-row steps still
+    carried one-term activations) row by row and two LSA tokens of each; the other 13 sequences are checked
     through the tree properties."""
     p = synth.PRESETS["c5"]
     w = synth.make_weights(p)
     g = H.make_gpu(p, w, max_ctx=p.ctx + 64, lsa_chunk_tokens=p.batch * p.lsa_tokens)
     oracles = H.make_oracles(p, w)
     del w
-    stats = _given_caches_cycle(p, g, oracles, seqs=[0, 15])
-    assert stats["rows"] == 2 * (1 + 5 * 10)
+    stats = _given_caches_cycle(p, g, oracles, seqs=[0, 2, 15])
+    assert stats["rows"] == 3 * (1 + 5 * 10)
     g.close()
 
 
