@@ -208,8 +208,8 @@ def test_target_layer_inference_reduced_llama_shape(dtype, batch, n_tli):
 
 
 def test_maximum_rows_per_step_256():
-    """The largest forward the library takes: 16 sequences x breadth 16 = 256 rows (single-term bf16 activations,
-    N = 256 tiles, 64 queries per kv head in the attention, 16-wide top lists), depth 2, reduced widths."""
+    """The largest forward the library takes: 16 sequences x breadth 16 = 256 rows (two-term activations as two
+    256-row tiles per stage, 64 queries per kv head in the attention, 16-wide top lists), depth 2, reduced widths."""
     p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=2051, lsa_hq=2, lsa_hkv=2,
                      lsa_mlp=128, sa_hq=4, sa_hkv=1, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=448, ctx=70, batch=16,
                      tree_topk=16, tree_depth=2, tree_keep=40, lsa_tokens=2)
@@ -220,6 +220,22 @@ def test_maximum_rows_per_step_256():
     stats = run_cycle(p, g, H.make_oracles(p, w), None, None, synth.make_root(p), ca_cache=(caK, caV), sa_cache=(saK, saV),
                       seqs=[0, 7, 15])
     assert stats["rows"] == 3 * (1 + 16)
+
+
+@pytest.mark.parametrize("batch,topk", [(13, 10), (24, 8), (15, 15)])
+def test_row_counts_between_128_and_256(batch, topk):
+    """Forwards of 130, 192 and 225 rows: activation tiles of 160, 192 and 256 rows, two tiles (high- and low-order
+    terms) per stage; the step-0 forward of each (13, 24, 15 rows) takes the one-tile form."""
+    p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=2051, lsa_hq=2, lsa_hkv=2,
+                     lsa_mlp=128, sa_hq=4, sa_hkv=1, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=448, ctx=70, batch=batch,
+                     tree_topk=topk, tree_depth=3, tree_keep=30, lsa_tokens=2)
+    w = synth.make_weights(p)
+    g = H.make_gpu(p, w, max_ctx=80, lsa_chunk_tokens=32)
+    caK, caV = synth.make_cache(p, "ca")
+    saK, saV = synth.make_cache(p, "sa")
+    stats = run_cycle(p, g, H.make_oracles(p, w), None, None, synth.make_root(p), ca_cache=(caK, caV), sa_cache=(saK, saV),
+                      seqs=[0, batch - 1])
+    assert stats["rows"] == 2 * (1 + 2 * topk)
 
 
 def test_synthetic_caches_and_ragged_lengths():
