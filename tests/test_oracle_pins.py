@@ -669,3 +669,165 @@ def test_drafter_prefill_equals_token_by_token_decoding_and_the_ca_mask_of_the_f
         out2, _, _ = O.drafter_prefill(dr, t2, empty, empty, Kc, Vc, limits)
         dep_t[:, i] = np.any(np.abs(out2 - base) > 1e-9, axis=-1)
     assert np.array_equal(dep_t, read_grid("mask_sa_10x10.txt"))
+
+
+# ------------------------------------------------------------------ whole-block recomputations (MLP legs on)
+def _T(a):
+    return torch.tensor(np.asarray(a), dtype=torch.float64)
+
+
+def _t_norm(a, g, eps):
+    return a * torch.rsqrt((a * a).mean(-1, keepdim=True) + eps) * _T(g)
+
+
+def _t_mlp(u, w, block):
+    return (torch.nn.functional.silu(u @ _T(w[block + "_wgate"]).T) * (u @ _T(w[block + "_wup"]).T)) @ _T(w[block + "_wdown"]).T
+
+
+def _t_rot(a, pos, theta):
+    """[n, H, dh] rotated at positions pos [n]: the pair (i, i + dh/2) as one complex number times e^{i pos theta_i}."""
+    dh = a.shape[-1]
+    z = torch.complex(a[..., :dh // 2], a[..., dh // 2:])
+    ang = pos[:, None, None] * theta ** (-torch.arange(0, dh, 2, dtype=torch.float64) / dh)
+    z = z * torch.polar(torch.ones_like(ang), ang)
+    return torch.cat([z.real, z.imag], -1)
+
+
+def _lsa_block_library(c, w, X):
+    """Section 3.1.1 as a decoder layer over the layer axis, written with torch routines only."""
+    S, dh, hq, hkv, eps = X.shape[0], c["head_dim"], c["lsa_hq"], c["lsa_hkv"], c["rms_eps"]
+    x = _T(X)
+    u = _t_norm(x, w["lsa_norm1"], eps)
+    q = (u @ _T(w["lsa_wq"]).T).view(S, hq, dh).transpose(0, 1)
+    k = (u @ _T(w["lsa_wk"]).T).view(S, hkv, dh).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    v = (u @ _T(w["lsa_wv"]).T).view(S, hkv, dh).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v).transpose(0, 1).reshape(S, hq * dh)
+    y = x + o @ _T(w["lsa_wo"]).T
+    return (y + _t_mlp(_t_norm(y, w["lsa_norm2"], eps), w, "lsa")).numpy()
+
+
+def _sa_block_library(c, w, toks, p0):
+    """Section 3.1.2 "Self-Attention" over a token sequence at positions p0, p0+1, ...: one causal pass."""
+    n, dh, hq, hkv, eps = len(toks), c["head_dim"], c["sa_hq"], c["sa_hkv"], c["rms_eps"]
+    e = _T(w["embed"])[torch.tensor(toks)]
+    u = _t_norm(e, w["sa_norm1"], eps)
+    pos = torch.arange(p0, p0 + n, dtype=torch.float64)
+    q = _t_rot((u @ _T(w["sa_wq"]).T).view(n, hq, dh), pos, c["rope_theta"]).transpose(0, 1)
+    k = _t_rot((u @ _T(w["sa_wk"]).T).view(n, hkv, dh), pos, c["rope_theta"]).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    v = (u @ _T(w["sa_wv"]).T).view(n, hkv, dh).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True).transpose(0, 1).reshape(n, hq * dh)
+    a = e + o @ _T(w["sa_wo"]).T
+    return (a + _t_mlp(_t_norm(a, w["sa_norm2"], eps), w, "sa")).numpy()
+
+
+def _ca_block_library(c, w, xs, kv):
+    """Section 3.1.2 "Cross-Attention": queries from the rows xs, keys / values from the LSA outputs kv, no mask."""
+    n, m, dh, hq, hkv, eps = xs.shape[0], kv.shape[0], c["head_dim"], c["ca_hq"], c["ca_hkv"], c["rms_eps"]
+    x = _T(xs)
+    ukv = _t_norm(_T(kv), w["ca_normkv"], eps)
+    q = (_t_norm(x, w["ca_normq"], eps) @ _T(w["ca_wq"]).T).view(n, hq, dh).transpose(0, 1)
+    k = (ukv @ _T(w["ca_wk"]).T).view(m, hkv, dh).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    v = (ukv @ _T(w["ca_wv"]).T).view(m, hkv, dh).transpose(0, 1).repeat_interleave(hq // hkv, 0)
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v).transpose(0, 1).reshape(n, hq * dh)
+    cc = x + o @ _T(w["ca_wo"]).T
+    return (cc + _t_mlp(_t_norm(cc, w["ca_norm2"], eps), w, "ca")).numpy()
+
+
+def _oracle_sa_rows(dr, toks, p0):
+    """The oracle's SA block fed token by token with a growing key / value set."""
+    c = dr.c
+    K = np.zeros((0, c["sa_hkv"], c["head_dim"])); V = np.zeros((0, c["sa_hkv"], c["head_dim"]))
+    out = []
+    for i, t in enumerate(toks):
+        e, q, k, v = dr.sa_qkv(t, p0 + i)
+        K = np.concatenate([K, k[None]]); V = np.concatenate([V, v[None]])
+        out.append(dr.sa_block(e, q, K, V))
+    return np.stack(out)
+
+
+def _block_pin_inputs():
+    c = tiny_cfg(n_stack=5)
+    rng = np.random.default_rng(77)
+    w = tiny_weights(c, scale=0.5, rng=rng)            # every matrix non-zero, every gain different from 1
+    X = rng.standard_normal((c["n_stack"], c["d_stack"])) * 1.5
+    toks, p0 = [3, 17, 5, 5, 22, 0, 9], 4
+    xs = rng.standard_normal((3, c["d_model"]))
+    kv = rng.standard_normal((4, c["d_stack"]))
+    return c, w, X, toks, p0, xs, kv
+
+
+def test_lsa_block_with_mlp_equals_library_recomputation():
+    """The whole LSA block of one token, attention and MLP legs both on, against torch (Section 3.1.1; the
+    6144-wide MLP of the hyper-parameter table): pins the second pre-norm (on Y, with its own gain), the SwiGLU
+    leg and both residuals."""
+    c, w, X, *_ = _block_pin_inputs()
+    assert np.allclose(O.Drafter(c, w).lsa_rows(X), _lsa_block_library(c, w, X), atol=1e-10)
+
+
+def test_sa_block_with_mlp_equals_causal_library_attention_over_a_sequence():
+    """sa_qkv + sa_block over a short sequence against one causal torch pass with the rotation as a complex
+    product (Section 3.1.2 "Self-Attention"): pins the pre-norm gain, the rotation of q and k but not v, the
+    residual from the embedding, the second pre-norm and the MLP leg."""
+    c, w, _, toks, p0, *_ = _block_pin_inputs()
+    assert np.allclose(_oracle_sa_rows(O.Drafter(c, w), toks, p0), _sa_block_library(c, w, toks, p0), atol=1e-10)
+
+
+def test_ca_block_with_mlp_and_several_keys_equals_library_recomputation():
+    """ca_kv + ca_block with four cached entries against torch (Section 3.1.2 "Cross-Attention"): with more than
+    one key the query leg (its own norm gain and W_q) matters; the MLP leg is on."""
+    c, w, _, _, _, xs, kv = _block_pin_inputs()
+    dr = O.Drafter(c, w)
+    Kc, Vc = dr.ca_kv(kv)
+    got = np.stack([dr.ca_block(x, Kc, Vc) for x in xs])
+    assert np.allclose(got, _ca_block_library(c, w, xs, kv), atol=1e-10)
+
+
+def test_block_pins_catch_planted_mistakes():
+    """Each plausible slip, planted in a copy of the oracle on the CPU, must break one of the three pins above."""
+    c, w, X, toks, p0, xs, kv = _block_pin_inputs()
+
+    class MlpNormsX(O.Drafter):                      # MLP leg normalises X instead of Y
+        def lsa_rows(self, X):
+            self._x = np.asarray(X, np.float64)
+            return super().lsa_rows(X)
+
+        def mlp(self, u, block):
+            if block == "lsa":
+                u = O.rmsnorm(self._x, self.w("lsa_norm2"), self.c["rms_eps"])
+            return super().mlp(u, block)
+
+    class MlpUsesNorm1(O.Drafter):                   # MLP pre-norm takes the attention pre-norm's gain
+        def w(self, name):
+            return super().w("lsa_norm1" if name == "lsa_norm2" else name)
+
+    class RotatesV(O.Drafter):                       # v rotated like k
+        def sa_qkv(self, tok, pos):
+            e, q, k, v = super().sa_qkv(tok, pos)
+            return e, q, k, O.rope(v, pos, self.c["rope_theta"])
+
+    class SaWrongGain(O.Drafter):
+        def w(self, name):
+            return super().w("sa_norm2" if name == "sa_norm1" else name)
+
+    class SaDropsResidual(O.Drafter):                # a = W_o o without the embedding
+        def sa_block(self, e, q, K, V):
+            return super().sa_block(np.zeros_like(e), q, K, V)
+
+    class CaQueryGain(O.Drafter):                    # query pre-norm uses the MLP pre-norm's gain
+        def w(self, name):
+            return super().w("ca_norm2" if name == "ca_normq" else name)
+
+    class CaQueryTransposedHeads(O.Drafter):         # W_q rows permuted: heads read in the wrong order
+        def w(self, name):
+            m = super().w(name)
+            return m[::-1] if name == "ca_wq" else m
+
+    lsa_ref, sa_ref, ca_ref = _lsa_block_library(c, w, X), _sa_block_library(c, w, toks, p0), _ca_block_library(c, w, xs, kv)
+    for cls in (MlpNormsX, MlpUsesNorm1):
+        assert not np.allclose(cls(c, w).lsa_rows(X), lsa_ref, atol=1e-6), cls.__name__
+    for cls in (RotatesV, SaWrongGain, SaDropsResidual):
+        assert not np.allclose(_oracle_sa_rows(cls(c, w), toks, p0), sa_ref, atol=1e-6), cls.__name__
+    for cls in (CaQueryGain, CaQueryTransposedHeads):
+        dr = cls(c, w)
+        Kc, Vc = dr.ca_kv(kv)
+        assert not np.allclose(np.stack([dr.ca_block(x, Kc, Vc) for x in xs]), ca_ref, atol=1e-6), cls.__name__
