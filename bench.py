@@ -316,7 +316,13 @@ def main():
                     help="Target Layer Inference: run the last N Llama-shaped decoder layers in every forward (default 0, "
                          "the headline configuration)")
     ap.add_argument("--phases", action="store_true", help="with --fused-step or --workload c3: print per-phase times to stderr")
+    ap.add_argument("--timeline", action="store_true",
+                    help="stage-by-stage timeline of one drafting cycle (library variant built with -DMOA_TRACE: every kernel "
+                         "stamps the GPU timer when its predecessor completes); prints a table instead of the bench line")
+    ap.add_argument("--set-option", action="append", default=[], metavar="ID=VALUE", help="moa_set_option(ID, VALUE) before the run")
     args = ap.parse_args()
+    if args.timeline:
+        os.environ["MOA_TRACE_BUILD"] = "1"
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     from paper_2410_03804_b200 import synth
@@ -353,6 +359,9 @@ def main():
     cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
     max_ctx = p.ctx + 64
     g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens, fused_step=args.fused_step)
+    for kv in args.set_option:
+        oid, val = kv.split("=")
+        assert g.lib.moa_set_option(g.h, int(oid), int(val)) == 0, kv
     caK, caV = synth.make_cache(p, "ca")
     saK, saV = synth.make_cache(p, "sa")
     g.fill_cache("ca", caK.to(dev), caV.to(dev))
@@ -431,6 +440,33 @@ def main():
         cycle_e2e()
     torch.cuda.synchronize()
     assert g.moa_state_status() == 0
+
+    if args.timeline:
+        # one warm cycle traced kernel by kernel, stream launches; a stage's cost = next stamp - its own stamp
+        for _ in range(3):
+            cycle(h_dev, tok_dev, root_dev)
+        torch.cuda.synchronize()
+        g.moa_trace_begin()
+        cycle(h_dev, tok_dev, root_dev)
+        cycle(h_dev, tok_dev, root_dev)          # its first stamp closes the last stage of the traced cycle
+        tr = g.moa_trace_end()
+        n_cycle = len(tr) // 2
+        rows = [(k, grid, (tr[i + 1][2] - t) * 1e-3) for i, (k, grid, t) in enumerate(tr[:n_cycle])]
+        kinds = [r[0] for r in rows]          # a drafter forward opens with: row norm, q/k/v product, rotary, attention
+        first = [i for i in range(len(rows) - 3) if kinds[i:i + 4] == ["row_norm", "gemm", "rope", "attention"]]
+        print(f"# stage timeline of one {p.name} drafting cycle ({n_cycle} kernels, {sum(r[2] for r in rows):.1f} us)")
+        print("| # | kernel | grid.x | us |\n|---|---|---|---|")
+        for i, (k, grid, us) in enumerate(rows):
+            mark = " (forward %d starts)" % first.index(i) if i in first else ""
+            print(f"| {i} | {k}{mark} | {grid} | {us:.1f} |")
+        if len(first) >= 3:
+            a, b = first[2], first[3] if len(first) > 3 else n_cycle
+            print(f"# forward 2 (steady state, {b - a} kernels): {sum(r[2] for r in rows[a:b]):.1f} us")
+            by = {}
+            for k, _, us in rows[a:b]:
+                by[k] = by.get(k, 0.0) + us
+            print("# by kind: " + ", ".join(f"{k} {v:.1f}" for k, v in sorted(by.items(), key=lambda kv: -kv[1])))
+        return
 
     # The cycle's launches are recorded once into CUDA graphs (one with device-resident inputs, one with the
     # host<->device copies of the end-to-end path) and replayed: the library only enqueues work on the caller's

@@ -292,6 +292,16 @@ moa_status moa_profile_phases(moa_ctx *ctx, const void *ws, size_t ws_bytes, int
                               double *wait_us_out, int32_t *kind_out, int32_t *n_out, void *stream);
 /* Kernels launched so far by this host thread through the library. */
 int64_t moa_launch_count(void);
+/* Stage trace (no counterpart in the paper; only in a library built with -DMOA_TRACE, otherwise both calls return
+ * MOA_ERR_STATE and the kernels carry no trace code). Between the two calls every kernel of the library stores one
+ * entry when its first thread is released by the completion of the kernel before it in the stream:
+ * dev_buf[2 i] = the GPU's nanosecond timer, dev_buf[2 i + 1] = kernel id << 32 | gridDim.x (ids: 1 embedding,
+ * 2 GEMM, 3 attention, 4 attention merge, 5 LM-head merge, 6 tree expansion, 7 row norm, 8 residual + norm,
+ * 9 SwiGLU, 10 sum + cast, 11 rotary, 12 cache append, 13 layer mean, 0 other). The difference of two consecutive
+ * entries is what the earlier kernel cost inside the chain. dev_buf: device uint64 [2 * cap], caller-owned.
+ * moa_trace_end synchronises the device and returns the number of entries made (entries beyond cap are dropped). */
+moa_status moa_trace_begin(void *dev_buf, int32_t cap);
+moa_status moa_trace_end(int32_t *n_out);
 
 #ifdef __cplusplus
 }

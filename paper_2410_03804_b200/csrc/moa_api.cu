@@ -512,10 +512,10 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     const int N2[2] = {ckv, ckv};
     MOA_TRY(linear<T>(ctx, s, kvn, nt, D, 2, W2, N2, ws, p, &lo, status_word));
     launch_pdl(cache_append_kernel<T>, dim3(nt), dim3(256), 0, s, lo.part, lo.splits, lo.plane, 2 * ckv, 0, ckv, ckv, st->ca_len, c.max_ctx,
-                                              split, t0, (T*)st->ca_k, (T*)st->ca_v);
+                                              split, t0, (T*)st->ca_k, (T*)st->ca_v, (int*)status_word);
     MOA_CHECK_LAUNCH();
   }
-  add_len_kernel<<<1, 64, 0, s>>>(st->ca_len, split);
+  add_len_kernel<<<1, 64, 0, s>>>(st->ca_len, split, c.max_ctx);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -545,10 +545,10 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
     rr.split = split;
     rr.row0 = t0;
     launch_pdl(rope_store_kernel<T>, dim3(dim3(R, 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
-                                           c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (float*)nullptr, (T*)st->sa_k, (T*)st->sa_v);
+                                           c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (float*)nullptr, (T*)st->sa_k, (T*)st->sa_v, (int*)status_word);
     MOA_CHECK_LAUNCH();
   }
-  add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split);
+  add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split, c.max_ctx);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -661,7 +661,7 @@ static moa_status drafter_prefill_t(moa_ctx* ctx, moa_state* st, const int* tok,
       rr.split = one;
       rr.row0 = r0;
       launch_pdl(rope_store_kernel<T>, dim3(dim3(R, c.sa_hq + 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq,
-                 nq + nkv, c.sa_hq, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, (T*)st->sa_k, (T*)st->sa_v);
+                 nq + nkv, c.sa_hq, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, (T*)st->sa_k, (T*)st->sa_v, (int*)status_word);
       MOA_CHECK_LAUNCH();
       // row i of the chunk sits at position base + r0 + i and sees positions 0 .. base + r0 + i
       MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, c.sa_hq, c.sa_hkv, sa_k, sa_v, c.max_ctx, nkv, nullptr,
@@ -699,7 +699,7 @@ static moa_status drafter_prefill_t(moa_ctx* ctx, moa_state* st, const int* tok,
       MOA_TRY(residual_norm<T>(s, ctx, ws, p, R, E, &lo, nullptr, (T*)hidden_out + (size_t)g0 * E));
     }
   }
-  add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split);
+  add_len_kernel<<<1, 64, 0, s>>>(st->sa_len, split, c.max_ctx);
   MOA_CHECK_LAUNCH();
   return MOA_OK;
 }
@@ -741,7 +741,7 @@ static moa_status tree_attn_layer(moa_ctx* ctx, moa_state* st, cudaStream_t s, c
   rr.B = B;
   rr.slots = L.NS;
   launch_pdl(rope_store_kernel<T>, dim3(dim3(R, a.hq + 2 * a.hkv)), dim3(64), 0, s, lo->part, lo->splits, lo->plane, nq + 2 * nkv, 0, nq,
-             nq + nkv, a.hq, a.hkv, dh, a.theta, st->sa_len, rr, narrow, q32, (T*)a.tk, (T*)a.tv);
+             nq + nkv, a.hq, a.hkv, dh, a.theta, st->sa_len, rr, narrow, q32, (T*)a.tk, (T*)a.tv, (int*)status_word);
   MOA_CHECK_LAUNCH();
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, a.hq, a.hkv, (const T*)a.ck, (const T*)a.cv, c.max_ctx, nkv,
                        st->sa_len, 0, max_len, (const T*)a.tk, (const T*)a.tv, L.NS, row_anc, D, step + 1,
@@ -1454,6 +1454,46 @@ moa_status moa_profile_end(moa_ctx* ctx, double* ms_total, int32_t* launches) {
 
 int64_t moa_launch_count(void) { return g_launches; }
 
+moa_status moa_trace_begin(void* dev_buf, int32_t cap) {
+#ifdef MOA_TRACE
+  if (!dev_buf) return MOA_ERR_NULL;
+  if (cap <= 0) return MOA_ERR_SHAPE;
+  const int zero = 0;
+  unsigned long long* b = (unsigned long long*)dev_buf;
+  cudaError_t e = cudaMemcpyToSymbol(g_moa_trace_n, &zero, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_moa_trace_cap, &cap, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_moa_trace_buf, &b, sizeof(b));
+  if (e != cudaSuccess) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_trace_begin: %s", cudaGetErrorString(e));
+    return MOA_ERR_CUDA;
+  }
+  return MOA_OK;
+#else
+  (void)dev_buf; (void)cap;
+  return MOA_ERR_STATE;
+#endif
+}
+
+moa_status moa_trace_end(int32_t* n_out) {
+#ifdef MOA_TRACE
+  if (!n_out) return MOA_ERR_NULL;
+  unsigned long long* none = nullptr;
+  int n = 0;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpyFromSymbol(&n, g_moa_trace_n, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_moa_trace_buf, &none, sizeof(none));
+  if (e != cudaSuccess) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "moa_trace_end: %s", cudaGetErrorString(e));
+    return MOA_ERR_CUDA;
+  }
+  *n_out = n;
+  return MOA_OK;
+#else
+  (void)n_out;
+  return MOA_ERR_STATE;
+#endif
+}
+
 moa_status moa_set_option(moa_ctx* ctx, int32_t option, int32_t value) {
   if (!ctx) return MOA_ERR_NULL;
   if (option == MOA_OPT_FUSED_STEP) { ctx->fused_step = value != 0; return MOA_OK; }
@@ -1562,7 +1602,7 @@ moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, con
                       kv_out ? (bf16*)kv_out + (size_t)t0 * D : nullptr, (char*)ws, p, (cudaStream_t)stream);
     }
     if (r == MOA_OK) {
-      add_len_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(st->ca_len, split);
+      add_len_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(st->ca_len, split, ctx->c.max_ctx);
       MOA_CHECK_LAUNCH();
     }
   } else {

@@ -80,7 +80,7 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 template <int DH, bool QSPLIT, bool PSPLIT>
 __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_ATTN);
   constexpr int CH = DH / 8;                 // 16-byte chunks per row
   constexpr int KS = DH / 16;                // k-steps of the Q.K^T product
   constexpr int TILE_BYTES = AT_KB * DH * 2;
@@ -124,35 +124,6 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
     }
   }
 
-  // ---- Q tile -> shared (zero rows for queries beyond Qn) ----
-  for (int i = threadIdx.x; i < QT * CH; i += blockDim.x) {
-    const int ql = i / CH, c = i - ql * CH;
-    const int qi = qt * QT + ql;
-    const bool valid = qi < Qn;
-    const int row = seq * P.rows_per_seq + (valid ? qi / P.group : 0);
-    const int head = g * P.group + (valid ? qi % P.group : 0);
-    if (QSPLIT) {
-      uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
-      if (valid) {
-        float x[8];
-        load8_planes(P.q32 + (size_t)row * P.q_ld + head * DH + c * 8, P.q_splits, P.q_plane, x);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const bf16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
-          hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-          lo[e] = pack_bf16(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
-        }
-      }
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQ + tile_off<DH>(ql, c)), "r"(hi[0]), "r"(hi[1]),
-                   "r"(hi[2]), "r"(hi[3]) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQlo + tile_off<DH>(ql, c)), "r"(lo[0]), "r"(lo[1]),
-                   "r"(lo[2]), "r"(lo[3]) : "memory");
-    } else {
-      cp_async16(sQ + tile_off<DH>(ql, c), P.q + (size_t)row * P.q_ld + head * DH + c * 8, valid);
-    }
-  }
-  cp_async_commit();
-
   // A thread always copies the same 16-byte column of the rows r0, r0 + rstep, ...: one pointer increment per row.
   const int ld_c = threadIdx.x & (CH - 1), ld_r0 = threadIdx.x / CH, ld_rstep = blockDim.x / CH;
   const size_t row_stride = tree_part ? (size_t)P.hkv * DH : (size_t)P.posA_ld;       // elements between two positions
@@ -172,9 +143,61 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   };
 
   const int n_blocks = (k_end - k_begin + AT_KB - 1) / AT_KB;
-  if (n_blocks > 0) load_block(0, k_begin);
+  if (n_blocks > 0) load_block(0, k_begin);      // on its way while the queries are staged
   cp_async_commit();
-  cp_async_wait<1>();            // Q has landed
+
+  // ---- Q tile -> shared (zero rows for queries beyond Qn) ----
+  if (QSPLIT) {
+    // fp32 queries: four 8-element pieces per thread at a time, all their loads in flight before the first is used
+    // (one memory round trip per four pieces instead of one per piece)
+    for (int i0 = threadIdx.x; i0 < QT * CH; i0 += 4 * blockDim.x) {
+      float x[4][8];
+      bool valid[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * blockDim.x;
+        const int ql = i / CH, c = i - ql * CH;
+        const int qi = qt * QT + ql;
+        valid[u] = i < QT * CH && qi < Qn;
+        if (valid[u]) {
+          const int row = seq * P.rows_per_seq + qi / P.group;
+          const int head = g * P.group + qi % P.group;
+          load8_planes(P.q32 + (size_t)row * P.q_ld + head * DH + c * 8, P.q_splits, P.q_plane, x[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * blockDim.x;
+        if (i >= QT * CH) continue;
+        const int ql = i / CH, c = i - ql * CH;
+        uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+        if (valid[u]) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const bf16 h0 = __float2bfloat16_rn(x[u][2 * e]), h1 = __float2bfloat16_rn(x[u][2 * e + 1]);
+            hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+            lo[e] = pack_bf16(x[u][2 * e] - __bfloat162float(h0), x[u][2 * e + 1] - __bfloat162float(h1));
+          }
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQ + tile_off<DH>(ql, c)), "r"(hi[0]), "r"(hi[1]),
+                     "r"(hi[2]), "r"(hi[3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sQlo + tile_off<DH>(ql, c)), "r"(lo[0]), "r"(lo[1]),
+                     "r"(lo[2]), "r"(lo[3]) : "memory");
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < QT * CH; i += blockDim.x) {
+      const int ql = i / CH, c = i - ql * CH;
+      const int qi = qt * QT + ql;
+      const bool valid = qi < Qn;
+      const int row = seq * P.rows_per_seq + (valid ? qi / P.group : 0);
+      const int head = g * P.group + (valid ? qi % P.group : 0);
+      cp_async16(sQ + tile_off<DH>(ql, c), P.q + (size_t)row * P.q_ld + head * DH + c * 8, valid);
+    }
+  }
+  cp_async_commit();
+
+  cp_async_wait<0>();            // Q and the first key / value block have landed
   __syncthreads();
 
   // ---- Q fragments of this warp's 16 queries ----
@@ -377,7 +400,7 @@ __global__ void __launch_bounds__(CB_WARPS * 32) attn_combine_kernel(const float
                                                                     const float* __restrict__ part_ml, int n_parts, int n_rh,
                                                                     int share, bf16* __restrict__ out, int out_lo, int hq) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_ATTN_MERGE);
   __shared__ float acc_sh[CB_WARPS][DH];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int rh = share ? blockIdx.x : blockIdx.x * CB_WARPS + w;

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict
                                                            int vocab, const T* __restrict__ gain, int K, float eps,
                                                            float* __restrict__ res_out, T* __restrict__ y, int lo_rows) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_NORM);
   __shared__ float red[33];
   const int r = blockIdx.x;
   const TIN* xr;
@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(256) gemm_fma_kernel(const T* __restrict__ A, 
                                                        int R, int N, int K, const float* res, int ldr,
                                                        float* C, int ldc) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_GEMM);
   __shared__ float As[16][64 + 4];
   __shared__ float Ws[16][64 + 4];
   const int tid = threadIdx.x;
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(256) residual_norm_kernel(float* __restrict__ 
                                                             float eps, T* __restrict__ xn, T* __restrict__ hidden_out,
                                                             int lo_rows) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_RESNORM);
   __shared__ float red[33];
   const int r = blockIdx.x;
   const int nch = K >> 3;
@@ -227,7 +227,7 @@ __global__ void __cluster_dims__(RN_CLUSTER, 1, 1) __launch_bounds__(256)
                                  int K, const T* __restrict__ gain, float eps, T* __restrict__ xn,
                                  T* __restrict__ hidden_out, int lo_rows) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_RESNORM);
   __shared__ float red[33];
   __shared__ float cta_ss;
   const int r = blockIdx.y;
@@ -295,7 +295,7 @@ template <typename T>
 __global__ void silu_mul_split_kernel(const float* __restrict__ part, int splits, size_t plane, int F,
                                       T* __restrict__ h, size_t total, int lo_rows) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_SILU);
   const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (i >= total) return;
   const size_t r = i / F;
@@ -313,7 +313,7 @@ template <typename T>
 __global__ void sum_cast_kernel(const float* __restrict__ part, int splits, size_t plane, size_t total,
                                 T* __restrict__ y) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_SUMCAST);
   const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (i >= total) return;
   float v[8];
@@ -344,13 +344,14 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
                                   int v_off,
                                   int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
                                   RopeRows rr, T* __restrict__ qdst, float* __restrict__ qdst32, T* __restrict__ kdst,
-                                  T* __restrict__ vdst) {
+                                  T* __restrict__ vdst, int* __restrict__ status) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_ROPE);
   __shared__ float cs[64], sn[64];
   const int r = blockIdx.x;
   int seq, pos_add;
   size_t dst;
+  bool store_kv = true;
   if (rr.mode == 0) {
     seq = rr.step == 0 ? r : r / rr.B;
     pos_add = rr.step;
@@ -361,6 +362,12 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
     seq = rr.split.seq_of(t);
     pos_add = t - rr.split.off[seq];
     dst = (size_t)seq * rr.max_ctx + pos_base[seq] + pos_add;
+    // The host checked the capacity against its own count when the call was enqueued; a replayed graph can have
+    // moved the device count since. A row that would land outside the cache is dropped and reported.
+    if (pos_base[seq] + pos_add >= rr.max_ctx || pos_base[seq] < 0) {
+      store_kv = false;
+      if (threadIdx.x == 0 && blockIdx.y == 0 && status) atomicMax(status, DEV_ERR_BOUNDS);
+    }
   }
   const int pos = pos_base[seq] + pos_add;
   const int half = dh >> 1;
@@ -396,6 +403,7 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
     return;
   }
   h -= nqh;
+  if (!store_kv) return;
   if (h < hkv) {
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
       const float x1 = row(k_off + h * dh + j), x2 = row(k_off + h * dh + half + j);
@@ -413,13 +421,17 @@ template <typename T>
 __global__ void cache_append_kernel(const float* __restrict__ kv, int splits, size_t plane, int ld, int k_off, int v_off,
                                     int width,
                                     const int* __restrict__ len, int max_ctx, SeqSplit split, int row0,
-                                    T* __restrict__ kdst, T* __restrict__ vdst) {
+                                    T* __restrict__ kdst, T* __restrict__ vdst, int* __restrict__ status) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_APPEND);
   const int r = blockIdx.x;
   const int t = row0 + r;
   const int seq = split.seq_of(t);
   const int i = t - split.off[seq];
+  if (len[seq] < 0 || len[seq] + i >= max_ctx) {       // see rope_store_kernel: the device count decides
+    if (threadIdx.x == 0 && status) atomicMax(status, DEV_ERR_BOUNDS);
+    return;
+  }
   const size_t dst = ((size_t)seq * max_ctx + len[seq] + i) * width;
   const int nch = width >> 3;
   for (int c = threadIdx.x; c < 2 * nch; c += blockDim.x) {      // one thread per 8 columns of k, then of v
@@ -431,9 +443,9 @@ __global__ void cache_append_kernel(const float* __restrict__ kv, int splits, si
   }
 }
 
-__global__ void add_len_kernel(int* len, SeqSplit split) {
+__global__ void add_len_kernel(int* len, SeqSplit split, int max_ctx) {
   const int b = threadIdx.x;
-  if (b < split.n_seq) len[b] += split.off[b + 1] - split.off[b];
+  if (b < split.n_seq) len[b] = min(max_ctx, len[b] + split.off[b + 1] - split.off[b]);
 }
 struct LenVals { int n; int v[64]; };
 __global__ void set_len_kernel(int* len, LenVals lv) {
@@ -459,7 +471,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(const T* __restrict__ q,
                                                         const int* __restrict__ slotsB, int slots_ld, int nB,
                                                         int rows_per_seq, RowLimit lim, T* __restrict__ out) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_ATTN);
   constexpr int VEC = DH / 32;
   __shared__ float s_m[4], s_l[4], s_acc[4][DH];
   const int r = blockIdx.x, h = blockIdx.y;
@@ -526,7 +538,7 @@ template <typename T>
 __global__ void mean_layers_kernel(const float* __restrict__ Z, int S, int D, float* __restrict__ kvf,
                                    T* __restrict__ kv_out) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_MEAN);
   const int t = blockIdx.x;                                   // grid (tokens, ceil(D / blockDim.x))
   const int c = blockIdx.y * blockDim.x + threadIdx.x;
   if (c >= D) return;
@@ -548,7 +560,7 @@ __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {   /
 __global__ void __launch_bounds__(256) lse_topk_rows_kernel(const float* __restrict__ z, int V, int B,
                                                             int* __restrict__ ids, float* __restrict__ logp) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_LM_MERGE);
   __shared__ float red[33];
   __shared__ float s_v[8];
   __shared__ int s_i[8];

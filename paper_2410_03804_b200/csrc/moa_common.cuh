@@ -21,7 +21,31 @@ template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __flo
 // completed and its writes are visible. Every kernel of a chain calls pdl_wait() before it reads or overwrites
 // anything another kernel of the chain touches (so completion stays transitive); both are no-ops otherwise.
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Kernel ids of the optional stage trace (library built with -DMOA_TRACE; see moa_trace_begin).
+enum : int { KID_OTHER = 0, KID_EMBED, KID_GEMM, KID_ATTN, KID_ATTN_MERGE, KID_LM_MERGE, KID_EXPAND, KID_NORM, KID_RESNORM,
+             KID_SILU, KID_SUMCAST, KID_ROPE, KID_APPEND, KID_MEAN, KID_COUNT };
+#ifdef MOA_TRACE
+__device__ unsigned long long* g_moa_trace_buf = nullptr;   // [cap][2]: %globaltimer, kernel id << 32 | gridDim.x
+__device__ int g_moa_trace_cap = 0;
+__device__ int g_moa_trace_n = 0;
+#endif
+__device__ __forceinline__ void pdl_wait(int kid = KID_OTHER) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef MOA_TRACE
+  // one stamp per kernel, at the moment its first thread is released by its predecessor's completion
+  if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && g_moa_trace_buf) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    const int i = atomicAdd(&g_moa_trace_n, 1);
+    if (i < g_moa_trace_cap) {
+      g_moa_trace_buf[2 * i] = t;
+      g_moa_trace_buf[2 * i + 1] = ((unsigned long long)kid << 32) | (unsigned long long)gridDim.x;
+    }
+  }
+#else
+  (void)kid;
+#endif
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

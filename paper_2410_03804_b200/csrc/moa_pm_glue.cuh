@@ -281,7 +281,7 @@ __device__ __noinline__ void pm_mean_norm(PmSmem& S_, const PmOp& op, int wt) {
 
 // Cross-attention cache append: planes [tokens, k | v] -> bf16 cache rows at (seq, len[seq] + i).
 //  p[0] len, p[1] kdst, p[2] vdst; i[0] width, i[1] max_ctx, i[2] first token of this pass; rows = tokens
-__device__ __noinline__ void pm_cache_append(PmSmem& S, const PmOp& op, int wt) {
+__device__ __noinline__ void pm_cache_append(PmSmem& S, const PmOp& op, int wt, int* status) {
   const PmGemm& G = S.g[op.gemm];
   const float* out = G.out;
   const int splits = G.splits;
@@ -294,7 +294,12 @@ __device__ __noinline__ void pm_cache_append(PmSmem& S, const PmOp& op, int wt) 
     const int t = row0 + r;
     const int seq = S.split.seq_of(t);
     const int i = t - S.split.off[seq];
-    const size_t dst = (size_t)seq * max_ctx + __ldcg(len + seq) + i;
+    const int at = __ldcg(len + seq) + i;
+    if (at < i || at >= max_ctx) {                       // the device count decides: a row outside the cache is dropped and reported
+      if (wt == 0 && status) atomicMax(status, DEV_ERR_BOUNDS);
+      continue;
+    }
+    const size_t dst = (size_t)seq * max_ctx + at;
     for (int c = wt; c < 2 * nch; c += PM_WORKERS) {
       const bool isv = c >= nch;
       const int cc = isv ? c - nch : c;

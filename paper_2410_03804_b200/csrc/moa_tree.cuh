@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(512) tree_expand_kernel(TreePtrs t, int B, int
                                                           int* __restrict__ out_depth, float* __restrict__ out_score,
                                                           int* __restrict__ out_n) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_EXPAND);
   extern __shared__ unsigned char smem_raw[];
   float* c_score = (float*)smem_raw;                 // [max(C, P)]
   int* c_aux = (int*)(c_score + (P > 256 ? P : 256)); // [P] kept flags / slots

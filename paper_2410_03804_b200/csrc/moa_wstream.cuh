@@ -123,6 +123,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// The same copy with an L2 eviction-priority hint. Weight tiles are read once per call: marking them evict-first
+// keeps a gigabyte of LM-head weights from flushing what the chain re-reads (activations, partial planes, the
+// attention caches, the kernels' own code) out of L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -233,16 +247,17 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
     if (lane == 0) {
       // Weights depend on nothing: the tiles of the first ring pass go out at once. The activations were
       // written by the kernel before this one, so their tiles wait for it (programmatic dependent launch).
+      const uint64_t w_policy = l2_policy_evict_first();
       uint32_t pre = 0;
       for (int u = blockIdx.x; u < units && pre < (uint32_t)STAGES; u += gridDim.x) {
         int seg, n0, kb0, kb1, split, tile;
         decode(u, seg, n0, kb0, kb1, split, tile);
         for (int kb = kb0; kb < kb1 && pre < (uint32_t)STAGES; ++kb, ++pre) {
           mbar_expect_tx(full_bar(pre), STAGE_BYTES);
-          tma_load_2d(base + pre * STAGE_BYTES, &P.tmW[seg], kb * WS_BK, n0, full_bar(pre));
+          tma_load_2d_hint(base + pre * STAGE_BYTES, &P.tmW[seg], kb * WS_BK, n0, full_bar(pre), w_policy);
         }
       }
-      pdl_wait();
+      pdl_wait(KID_GEMM);
       {
         uint32_t i2 = 0;
         for (int u = blockIdx.x; u < units && i2 < pre; u += gridDim.x) {
@@ -267,7 +282,7 @@ __global__ void __launch_bounds__(WS_THREADS, 1) wstream_gemm_kernel(const __gri
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), STAGE_BYTES);
           const uint32_t dst = base + s * STAGE_BYTES;
-          tma_load_2d(dst, tw, kb * WS_BK, n0, full_bar(s));
+          tma_load_2d_hint(dst, tw, kb * WS_BK, n0, full_bar(s), w_policy);
           tma_load_2d(dst + WS_W_BYTES, &P.tmX, kb * WS_BK, 0, full_bar(s));
           if (XS2) tma_load_2d(dst + WS_W_BYTES + X_BYTES, &P.tmX, kb * WS_BK, P.lo_row, full_bar(s));
         }
@@ -489,7 +504,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) lm_merge_kernel(const float* __
                                                                  MergeScratch sc, int* __restrict__ ids,
                                                                  float* __restrict__ logp) {
   pdl_trigger();
-  pdl_wait();
+  pdl_wait(KID_LM_MERGE);
   __shared__ float red[33];
   __shared__ float w_val[MERGE_WARPS][MERGE_MAXB];
   __shared__ int w_id[MERGE_WARPS][MERGE_MAXB];

@@ -22,7 +22,7 @@ MOA_OK = 0
 EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_drafter_prefill", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_pack_tree", "moa_unpack_tree", "moa_quantize_rows", "moa_dequantize_rows", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
-           "moa_launch_count"]
+           "moa_launch_count", "moa_trace_begin", "moa_trace_end"]
 
 
 class MoaConfig(C.Structure):
@@ -86,9 +86,10 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
+    trace = os.environ.get("MOA_TRACE_BUILD", "") == "1"          # the variant whose kernels stamp the stage trace
+    path = _build.LIB_TRACE if trace else _build.LIB
     if rebuild_if_stale and (os.path.exists("/usr/local/cuda/bin/nvcc") or os.environ.get("NVCC")):
-        path = _build.build()
+        path = _build.build(trace=trace)
     if not os.path.exists(path):
         raise RuntimeError(f"{path} not found: build it with `python -m paper_2410_03804_b200.build`")
     lib = C.CDLL(path)
@@ -123,6 +124,8 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_profile_phases.argtypes = [vp, vp, sz, i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i32),
                                        C.POINTER(i32), vp]
     lib.moa_launch_count.argtypes = []
+    lib.moa_trace_begin.argtypes = [vp, i32]
+    lib.moa_trace_end.argtypes = [C.POINTER(i32)]
     for n in EXPORTS:
         if n not in ("moa_destroy", "moa_status_str", "moa_last_cuda_error", "moa_launch_count"):
             getattr(lib, n).restype = i32
@@ -434,6 +437,21 @@ class MoA:
 
     def moa_launch_count(self) -> int:
         return int(self.lib.moa_launch_count())
+
+    TRACE_KINDS = ["other", "embed", "gemm", "attention", "attn_merge", "lm_merge", "tree_expand", "row_norm", "res_norm",
+                   "swiglu", "sum_cast", "rope", "cache_append", "layer_mean"]
+
+    def moa_trace_begin(self, cap: int = 4096):
+        """Starts the stage trace (library built with MOA_TRACE_BUILD=1 only)."""
+        self._trace = torch.zeros(2 * cap, dtype=torch.int64, device=self.device)
+        _check(self.lib.moa_trace_begin(_ptr(self._trace), cap), "moa_trace_begin")
+
+    def moa_trace_end(self):
+        """[(kernel kind, gridDim.x, nanosecond stamp)] in launch order."""
+        n = C.c_int32()
+        _check(self.lib.moa_trace_end(C.byref(n)), "moa_trace_end")
+        t = self._trace.cpu().tolist()
+        return [(self.TRACE_KINDS[(t[2 * i + 1] >> 32) & 0xff], t[2 * i + 1] & 0xffffffff, t[2 * i]) for i in range(min(n.value, len(t) // 2))]
 
     # ---- convenience for tests / bench: raw views of the tree blob ---------------------------
     def fill_cache(self, which: str, k: torch.Tensor, v: torch.Tensor):

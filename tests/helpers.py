@@ -83,12 +83,13 @@ def tie_window(p: synth.Preset, z) -> float:
     return 1e-3 + 2e-3 * scale if split_regime(p) else 2e-2 * scale
 
 
-def check_topk(gpu_ids, gpu_lp, z, tol, window=1e-3, what=""):
+def check_topk(gpu_ids, gpu_lp, z, tol, window=1e-3, what="", literal=None):
     """One row's top-B against the oracle's full logits z.
 
     Each reported log-probability must match the oracle's for that token within tol * max|z|; the j-th pick
     must be within `window` of the oracle's j-th best log-probability (either of two near-tied tokens is
-    accepted); ids are distinct. Returns True when the id list equals the oracle's exactly."""
+    accepted); ids are distinct. Returns True when the id list equals the oracle's exactly. With `literal` (a
+    list) given, appends whether the row also passes the window the task states literally (1e-3)."""
     z = np.asarray(z, np.float64)
     lse = z.max() + np.log(np.exp(z - z.max()).sum())
     logp = z - lse
@@ -97,7 +98,11 @@ def check_topk(gpu_ids, gpu_lp, z, tol, window=1e-3, what=""):
     ids = [int(i) for i in gpu_ids]
     assert len(set(ids)) == B and min(ids) >= 0 and max(ids) < z.shape[0], (what, ids)
     scale = np.max(np.abs(z))
+    lit = True
     for j in range(B):
         assert abs(float(gpu_lp[j]) - logp[ids[j]]) <= tol * scale, (what, j, float(gpu_lp[j]), logp[ids[j]])
         assert logp[ids[j]] >= logp[order[j]] - window, (what, j, ids[j], logp[ids[j]], logp[order[j]])
+        lit = lit and logp[ids[j]] >= logp[order[j]] - 1e-3
+    if literal is not None:
+        literal.append(bool(lit))
     return ids == [int(i) for i in order[:B]]

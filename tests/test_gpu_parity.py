@@ -57,7 +57,8 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
     forced = {b: [([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in od["trees"][b][1]] for b in seqs}
     ox = od if exact is dec else oracle_cycle(p, exact, h_stack, prompt, root, ca_cache, sa_cache, forced, seqs=seqs,
                                               tli_cache=tli_cache)
-    stats = dict(rows=0, exact=0, worst_hidden=0.0, worst_logp=0.0)
+    stats = dict(rows=0, exact=0, literal=0, worst_hidden=0.0, worst_logp=0.0)
+    literal = []
     if ca_cache is None:
         n_tok = [h_stack.shape[0] // nb] * nb
         n = n_tok[0]
@@ -104,7 +105,8 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
                 lp_err = np.max(np.abs(lp[gr] - lpx[ids[gr]])) / np.max(np.abs(zx))
                 stats["worst_logp"] = max(stats["worst_logp"], float(lp_err))
                 assert lp_err <= tol, f"logp s{s} r{gr}"
-                stats["exact"] += H.check_topk(ids[gr], lp[gr], rd["z"], tol, H.tie_window(p, rd["z"]), f"topk s{s} r{gr}")
+                stats["exact"] += H.check_topk(ids[gr], lp[gr], rd["z"], tol, H.tie_window(p, rd["z"]), f"topk s{s} r{gr}",
+                                               literal)
                 stats["rows"] += 1
                 f_ids[gr] = rd["ids"]
                 f_lp[gr] = rd["logp"].astype(np.float32)
@@ -123,6 +125,7 @@ def run_cycle(p, g, oracles, h_stack, prompt, root, ca_cache=None, sa_cache=None
         assert np.all(parent[b, 1:k] < np.arange(1, k)) and np.all(parent[b, 1:k] >= 0)
         assert np.array_equal(depth[b, 1:k], depth[b, parent[b, 1:k]] + 1)
         assert np.all(score[b, 1:k] <= score[b, parent[b, 1:k]])
+    stats["literal"] = int(sum(literal))       # rows whose every pick is within 1e-3 of the oracle's pick of that rank
     print(f"[parity {p.name} {p.dtype}] {stats}")
     return stats
 
@@ -304,3 +307,45 @@ def test_api_misuse_returns_status_and_launches_nothing():
     with pytest.raises(MoaError, match="ERR_SHAPE"):
         from paper_2410_03804_b200 import moa
         moa.MoA(bad, {k: v.cuda() for k, v in w.items()}, 1, 16)
+
+
+@pytest.mark.parametrize("dtype,lsa_tokens", [("bf16", 6), ("f32", 6), ("bf16", 60)])
+def test_device_side_capacity_guard_when_the_host_count_is_stale(dtype, lsa_tokens):
+    """A recorded graph replays cache appends with the host-side capacity check frozen at capture time. Here the host
+    count is set back by hand (the state a replay is in): the kernels must drop the rows that would land beyond
+    max_ctx, clamp the device count and raise the status word. Sequence 1's cache region lies right behind
+    sequence 0's, so a missing guard would show there, inside the allocation. 60 tokens x 5 layers = 300 rows takes the
+    dense-regime LSA pass (one persistent kernel), 6 tokens the weight-streaming launch chain."""
+    p = synth.scaled(synth.PRESETS["c2"], d_model=512, n_stack=5, d_stack=384, vocab=5003, lsa_hq=8, lsa_hkv=2,
+                     lsa_mlp=768, sa_hq=8, sa_hkv=2, sa_mlp=64, ca_hq=8, ca_hkv=4, ca_mlp=896, ctx=0, batch=1,
+                     tree_topk=5, tree_depth=2, tree_keep=8, dtype=dtype)
+    w = synth.make_weights(p)
+    cap = lsa_tokens + lsa_tokens // 2                     # the second append overflows by half of its rows
+    g = H.make_gpu(p, w, max_ctx=cap, lsa_chunk_tokens=64, max_batch=2)
+    g.moa_tree_begin(synth.make_root(p).cuda())            # clears the status word
+    for t in (g.sa_k, g.sa_v, g.ca_k, g.ca_v):
+        t[1].fill_(7.0)                                    # sentinel in the neighbour's region
+    n = lsa_tokens
+    toks = synth.make_tokens(p, 2 * n, tensor_index=47)[0]
+    h = synth.make_h_stack(p, 2 * n)
+    g.moa_sa_append(toks[:n].contiguous().cuda(), [n])
+    g.moa_lsa_forward(h[:n].cuda(), [n], want_kv=False)
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0 and g.sa_len[:1].tolist() == [n] and g.ca_len[:1].tolist() == [n]
+    k_before, ck_before = g.sa_k[0, :n].clone(), g.ca_k[0, :n].clone()
+    g._sa_len_host[0] = 0                                  # the host's view at capture time
+    g._ca_len_host[0] = 0
+    g.moa_sa_append(toks[n:].contiguous().cuda(), [n])
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 6                       # MOA_ERR_CAPACITY, raised on the device
+    assert g.sa_len[:1].tolist() == [cap]
+    g.moa_tree_begin(synth.make_root(p).cuda())
+    g.moa_lsa_forward(h[n:].cuda(), [n], want_kv=False)
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 6
+    assert g.ca_len[:1].tolist() == [cap]
+    for t in (g.sa_k, g.sa_v, g.ca_k, g.ca_v):
+        assert bool((t[1] == 7.0).all()), "a row was written beyond max_ctx"
+    # the rows that fit were written, the earlier ones are untouched
+    assert torch.equal(g.sa_k[0, :n], k_before) and torch.equal(g.ca_k[0, :n], ck_before)
+    assert float(g.sa_k[0, n:cap].float().abs().max()) > 0 and float(g.ca_k[0, n:cap].float().abs().max()) > 0
