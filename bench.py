@@ -310,16 +310,13 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every cycle on the stream instead of replaying a CUDA graph")
-    ap.add_argument("--fused-step", action="store_true",
-                    help="every forward as one persistent kernel (MOA_OPT_FUSED_STEP); implies --no-graph")
     ap.add_argument("--tli", type=int, default=0,
                     help="Target Layer Inference: run the last N Llama-shaped decoder layers in every forward (default 0, "
                          "the headline configuration)")
-    ap.add_argument("--phases", action="store_true", help="with --fused-step or --workload c3: print per-phase times to stderr")
+    ap.add_argument("--phases", action="store_true", help="with --workload c3: print per-phase times of the last dense LSA pass to stderr")
     ap.add_argument("--timeline", action="store_true",
                     help="stage-by-stage timeline of one drafting cycle (library variant built with -DMOA_TRACE: every kernel "
                          "stamps the GPU timer when its predecessor completes); prints a table instead of the bench line")
-    ap.add_argument("--set-option", action="append", default=[], metavar="ID=VALUE", help="moa_set_option(ID, VALUE) before the run")
     args = ap.parse_args()
     if args.timeline:
         os.environ["MOA_TRACE_BUILD"] = "1"
@@ -351,17 +348,12 @@ def main():
         if world > 1:
             dist.destroy_process_group()
         return
-    if args.fused_step:
-        args.no_graph = True
     # Replicas only: the path does not shard (one sequence batch per GPU, no data-path collective).
     w = {k: v.to(dev) for k, v in synth.make_weights(p).items()}
     w.update({k: v.to(dev) for k, v in synth.make_tli_weights(p).items()})
     cfg = {k: p.as_dict()[k] for k in CFG_KEYS}
     max_ctx = p.ctx + 64
-    g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens, fused_step=args.fused_step)
-    for kv in args.set_option:
-        oid, val = kv.split("=")
-        assert g.lib.moa_set_option(g.h, int(oid), int(val)) == 0, kv
+    g = moa.MoA(cfg, w, p.batch, max_ctx, lsa_chunk_tokens=p.batch * p.lsa_tokens)
     caK, caV = synth.make_cache(p, "ca")
     saK, saV = synth.make_cache(p, "sa")
     g.fill_cache("ca", caK.to(dev), caV.to(dev))
@@ -388,7 +380,7 @@ def main():
 
     split_ev = []      # when filled by the caller: (before forwards, after forwards) event pairs of each cycle
 
-    def cycle(h, tok, root, show=False, mark=False):
+    def cycle(h, tok, root, mark=False):
         g.moa_state_set_len("ca", lens)
         g.moa_state_set_len("sa", lens)
         g.moa_lsa_forward(h, [A] * nb, want_kv=False)
@@ -401,10 +393,6 @@ def main():
         for s in range(D):
             R = nb if s == 0 else nb * B
             ids, lp, _ = g.moa_draft_step(out=(ids_buf[:R], lp_buf[:R], None))
-            if show and s in (0, 1):
-                ph = g.moa_profile_phases()
-                sys.stderr.write(f"[phases, forward {s}] total {sum(u for _, u, _w in ph):.1f} us: " +
-                                 " ".join(f"{k}:{u:.1f}({w_:.1f})" for k, u, w_ in ph) + "\n")
             res = g.moa_tree_expand(ids, lp, out=outs)
         if mark:
             split_ev[-1][1].record()
@@ -506,8 +494,6 @@ def main():
     # the stream (events cannot be read inside a graph), directly after the timed replays
     g.moa_profile_begin()
     ms_stream = timed(lambda: cycle(h_dev, tok_dev, root_dev), args.steps)
-    if args.fused_step and args.phases:
-        cycle(h_dev, tok_dev, root_dev, show=True)
     lm_ms, lm_n = g.moa_profile_end()
     # the D forwards alone (draft step + expansion), stream launches, events around them inside each cycle
     timed(lambda: cycle(h_dev, tok_dev, root_dev, mark=True), args.steps)

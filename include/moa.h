@@ -116,7 +116,7 @@ void moa_destroy(moa_ctx *ctx);
  *   k, v    device T [max_batch, max_ctx, hkv, head_dim] per layer: the LLM's cache of that layer (keys already
  *           rotated), owned and filled by the caller, never written by the library
  * Call it before moa_state_bytes: both sizes grow. n_layers = 0 (layers and caches may be NULL) turns it off
- * again. With TLI on, MOA_OPT_FUSED_STEP does not apply to moa_draft_step (the launch chain is used).
+ * again.
  * MOA_ERR_SHAPE for n_layers > MOA_MAX_TLI, hq % hkv != 0, mlp % 16 != 0. */
 typedef struct {
   int32_t n_layers;  /* N = TLI, 0 .. MOA_MAX_TLI */
@@ -132,13 +132,6 @@ typedef struct {
 } moa_tli_caches;
 moa_status moa_tli_configure(moa_ctx *ctx, const moa_tli_config *cfg, const moa_tli_layer *layers_host,
                              const moa_tli_caches *caches);
-
-/* Options. MOA_OPT_FUSED_STEP (bf16 only): run moa_draft_step, and moa_lsa_forward passes of any size, as ONE
- * persistent cooperative kernel (phases separated by grid-wide barriers, weights prefetched across phases,
- * activations carried as two bf16 terms up to 128 rows) instead of a chain of launches. Same results within
- * tolerance; off by default because the chain is faster at small row counts. */
-#define MOA_OPT_FUSED_STEP 1
-moa_status moa_set_option(moa_ctx *ctx, int32_t option, int32_t value);
 
 /* Sizes in bytes of moa_state.tree and of the workspace every compute call needs.
  * lsa_chunk_tokens (>= 1) is the number of tokens moa_lsa_forward processes per internal
@@ -280,13 +273,12 @@ moa_status moa_state_status(moa_ctx *ctx, moa_state *st, void *stream);
  * Do not use inside a stream capture. */
 moa_status moa_profile_begin(moa_ctx *ctx);
 moa_status moa_profile_end(moa_ctx *ctx, double *ms_total, int32_t *launches);
-/* Phase timing of the LAST fused launch (on the bf16 path a drafter forward or an LSA pass runs as one
- * persistent kernel made of phases separated by grid-wide barriers). Valid when that launch was made between
+/* Phase timing of the LAST dense LSA pass (on the bf16 path an LSA pass of more than 256 (token, layer) rows runs as
+ * one persistent kernel made of phases separated by grid-wide barriers). Valid when that launch was made between
  * moa_profile_begin and moa_profile_end with the same workspace. us_out[i] = microseconds phase i took on CTA 0
  * including its closing barrier, wait_us_out[i] (may be NULL) = the part of it CTA 0 spent in that barrier,
- * kind_out[i] = its kind (0 GEMM, 1 embed+norm, 2 row norm, 3 residual+norm, 4 rotary, 5 attention,
- * 6 attention merge, 7 SwiGLU, 8 sum+cast, 9 layer mean+norm, 10 cache append, 11 LM-head merge,
- * 12 layer self-attention).
+ * kind_out[i] = its kind (0 GEMM, 1 row norm, 2 residual + norm, 3 layer mean + norm, 4 cache append,
+ * 5 layer self-attention).
  * Synchronises the stream. HOST output arrays of `cap` entries. */
 moa_status moa_profile_phases(moa_ctx *ctx, const void *ws, size_t ws_bytes, int32_t cap, double *us_out,
                               double *wait_us_out, int32_t *kind_out, int32_t *n_out, void *stream);

@@ -7,6 +7,8 @@
 #include <mutex>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "moa_attn.cuh"
 #include "moa_basic.cuh"
 #include "moa_codec.cuh"
@@ -16,6 +18,14 @@
 #include "moa_wstream.cuh"
 
 using namespace moa;
+
+// One NVTX range per compute call of the C ABI (a profiler's timeline then shows the calls by name; without a
+// tool attached a range costs a function-pointer test).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+#define MOA_RANGE() NvtxRange nvtx_range__(__func__)
 
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
@@ -48,8 +58,7 @@ struct moa_ctx {
   moa_tli_layer tli_w[MOA_MAX_TLI];
   moa_tli_caches tli_c;
   bool fast;           // weight-streaming tcgen05 GEMMs usable
-  bool coop;           // cooperative launches available: the phase-machine kernels are used
-  bool fused_step;     // moa_draft_step as one persistent kernel (moa_set_option)
+  bool coop;           // cooperative launches available: the dense LSA pass can run as one persistent kernel
   int smem_optin;      // largest dynamic shared memory a CTA may ask for
   int last_n_ops;      // phase kinds of the last fused launch (for moa_profile_phases)
   int last_kinds[PM_MAX_OPS];
@@ -365,12 +374,13 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
                             const float* q32, int q_splits, size_t q_plane, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
                             int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
                             int slots_ld, int nB, int n_slots, int rows_per_seq, T* out,
-                            RowLimit lim = RowLimit{nullptr, 0, 0}) {
+                            RowLimit lim = RowLimit{nullptr, 0, 0}, void* status_word = nullptr) {
   if (R <= 0) return MOA_OK;
   if (sizeof(T) == 2) {
     AttnParams P;
     memset(&P, 0, sizeof(P));
     P.lim = lim;
+    P.status = (int*)status_word;
     const int nseq = R / rows_per_seq;
     P.q = (const bf16*)q; P.q32 = q32; P.q_splits = q_splits; P.q_plane = q_plane; P.q_ld = q_ld;
     P.hq = hq; P.hkv = hkv; P.group = hq / hkv;
@@ -399,8 +409,6 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     // fp32 queries and the probabilities are split into two bf16 terms each
     if (q32)
       return dh == 128 ? launch_attn_split<128, true, true>(s, P, nseq, nwarps) : launch_attn_split<64, true, true>(s, P, nseq, nwarps);
-    if (q32)
-      return dh == 128 ? launch_attn_split<128, true, false>(s, P, nseq, nwarps) : launch_attn_split<64, true, false>(s, P, nseq, nwarps);
     return dh == 128 ? launch_attn_split<128, false, false>(s, P, nseq, nwarps) : launch_attn_split<64, false, false>(s, P, nseq, nwarps);
   }
   dim3 grid(R, hq);
@@ -479,7 +487,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     const T* x = (const T*)h_stack + (size_t)t0 * S * D;
     // pre-norm and q, k, v projections of every (token, layer) row: rows of [q | k | v]
     launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, x, nullptr, 0, (const T*)w.lsa_norm1, D, c.rms_eps, xres, xn,
-               lo_rows_of(sizeof(T), R));
+               lo_rows_of(sizeof(T), R), (int*)status_word);
     MOA_CHECK_LAUNCH();
     const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
     const int N3[3] = {nq, nkv, nkv};
@@ -505,7 +513,7 @@ static moa_status lsa_forward_t(moa_ctx* ctx, moa_state* st, const void* h_stack
     MOA_CHECK_LAUNCH();
     // cross-attention keys / values of the new positions, appended to the cache
     launch_pdl(rmsnorm_rows_kernel<float, T>, dim3(nt), dim3(256), 0, s, kvf, nullptr, 0, (const T*)w.ca_normkv, D, c.rms_eps, nullptr, kvn,
-               lo_rows_of(sizeof(T), nt));
+               lo_rows_of(sizeof(T), nt), (int*)status_word);
     MOA_CHECK_LAUNCH();
     const int ckv = c.ca_hkv * dh;
     const void* W2[2] = {w.ca_wk, w.ca_wv};
@@ -533,7 +541,7 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
   for (int t0 = 0; t0 < total; t0 += p.rows_cap) {
     const int R = (total - t0) < p.rows_cap ? (total - t0) : p.rows_cap;
     launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, tok + t0, c.vocab, (const T*)w.sa_norm1, E,
-                                                c.rms_eps, nullptr, xn, lo_rows_of(sizeof(T), R));
+                                                c.rms_eps, nullptr, xn, lo_rows_of(sizeof(T), R), (int*)status_word);
     MOA_CHECK_LAUNCH();
     const void* W2[2] = {w.sa_wk, w.sa_wv};
     const int N2[2] = {nkv, nkv};
@@ -647,7 +655,7 @@ static moa_status drafter_prefill_t(moa_ctx* ctx, moa_state* st, const int* tok,
       const int g0 = split.off[b] + r0;                 // first row of the chunk in the caller's arrays
       // ---- self-attention block ----
       launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, tok + g0, V, (const T*)w.sa_norm1, E, c.rms_eps,
-                 xres, xn, lo_rows_of(sizeof(T), R));
+                 xres, xn, lo_rows_of(sizeof(T), R), (int*)status_word);
       MOA_CHECK_LAUNCH();
       {
         const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
@@ -745,7 +753,7 @@ static moa_status tree_attn_layer(moa_ctx* ctx, moa_state* st, cudaStream_t s, c
   MOA_CHECK_LAUNCH();
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, a.hq, a.hkv, (const T*)a.ck, (const T*)a.cv, c.max_ctx, nkv,
                        st->sa_len, 0, max_len, (const T*)a.tk, (const T*)a.tv, L.NS, row_anc, D, step + 1,
-                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf));
+                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word));
   {
     const void* W1[1] = {a.wo};
     const int N1[1] = {E};
@@ -785,7 +793,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
 
   // ---- self-attention block ----
   launch_pdl(rmsnorm_rows_kernel<T, T>, dim3(R), dim3(256), 0, s, (const T*)w.embed, row_tok, V, (const T*)w.sa_norm1, E, c.rms_eps, xres, xn,
-             lo_rows_of(sizeof(T), R));
+             lo_rows_of(sizeof(T), R), (int*)status_word);
   MOA_CHECK_LAUNCH();
   {
     TreeAttnLayer a = {w.sa_wq, w.sa_wk, w.sa_wv, w.sa_wo, w.sa_norm2, w.sa_wgate, w.sa_wup, w.sa_wdown,
@@ -810,7 +818,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   // bf16 path: the attention kernel reads the projection's split planes itself (fp32 queries, two bf16 terms)
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32 ? lo.part : nullptr, lo.splits, lo.plane, cq, R, c.ca_hq, c.ca_hkv,
                        (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr,
-                       (const T*)nullptr, 0, nullptr, 0, 0, 0, rows_per_seq, obuf));
+                       (const T*)nullptr, 0, nullptr, 0, 0, 0, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word));
   {
     const void* W1[1] = {w.ca_wo};
     const int N1[1] = {E};
@@ -840,29 +848,20 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
 struct PmBuild {
   PmParams P;
   moa_ctx* ctx;
-  int NB, xsplit, lo_rows, grid;
+  int NB, grid;
   int unit_run;          // units scheduled so far (rotates the CTA that gets unit 0 of the next GEMM)
-  size_t attn_bytes;
-  bool dense;
+  size_t attn_bytes;     // shared memory the layer self-attention phase needs (laid over the ring)
   moa_status err;
 };
 
-static void pm_init(PmBuild& b, moa_ctx* ctx, int R, bool dense, void* tree, const TreeLayout& L, char* ws,
-                    const Workspace& p) {
+static void pm_init(PmBuild& b, moa_ctx* ctx, void* tree, const TreeLayout& L, char* ws, const Workspace& p) {
   memset(&b.P, 0, sizeof(b.P));
   b.ctx = ctx;
-  b.dense = dense;
   b.grid = ctx->sm_count;
   b.unit_run = 0;
   b.attn_bytes = 4096;
   b.err = MOA_OK;
-  if (dense) { b.NB = 256; b.xsplit = 0; }
-  else if (R <= 16) { b.NB = 32; b.xsplit = 1; }
-  else if (R <= 32) { b.NB = 64; b.xsplit = 1; }
-  else if (R <= 64) { b.NB = 128; b.xsplit = 1; }
-  else if (R <= 128) { b.NB = 256; b.xsplit = 1; }
-  else { b.NB = 256; b.xsplit = 0; }
-  b.lo_rows = b.xsplit ? b.NB / 2 : 0;
+  b.NB = 256;
   b.P.sync = (int*)((char*)tree + L.status) + 4;
   b.P.flags = (int*)((char*)tree + L.flags);
   b.P.status = (int*)((char*)tree + L.status);
@@ -884,7 +883,7 @@ static int pm_gemm(PmBuild& b, const void* X, int R, int K, int nseg, const void
   const int gi = b.P.n_gemms++;
   PmGemm& G = b.P.g[gi];
   memset(&G, 0, sizeof(G));
-  G.n_seg = nseg; G.mode = mode; G.R = R; G.xsplit = b.xsplit;
+  G.n_seg = nseg; G.mode = mode; G.R = R;
   int tiles = 0, col = 0;
   for (int i = 0; i < nseg; ++i) {
     const WeightMap* wm = find_wmap(b.ctx, W[i]);
@@ -898,7 +897,7 @@ static int pm_gemm(PmBuild& b, const void* X, int R, int K, int nseg, const void
   G.tiles_total = tiles;
   G.kb_total = K / WS_BK;
   G.rows_per_block = mode == 4 ? 128 : b.NB;
-  G.row_blocks = b.dense && mode >= 2 ? (R + G.rows_per_block - 1) / G.rows_per_block : 1;
+  G.row_blocks = mode >= 2 ? (R + G.rows_per_block - 1) / G.rows_per_block : 1;
   G.splits = mode == 0 ? pick_splits(tiles, G.kb_total, R, part_rows, b.grid) : 1;
   G.units = tiles * G.splits * G.row_blocks;
   G.rot = b.unit_run % b.grid;
@@ -906,7 +905,7 @@ static int pm_gemm(PmBuild& b, const void* X, int R, int K, int nseg, const void
   G.ldo = col;
   G.plane = (size_t)R * col;
   G.out = part;
-  const int rows_total = b.xsplit ? b.lo_rows + R : R;
+  const int rows_total = R;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows_total};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
   cuuint32_t box[2] = {(cuuint32_t)WS_BK, (cuuint32_t)G.rows_per_block};
@@ -950,76 +949,32 @@ static moa_status pm_launch(PmBuild& b, cudaStream_t s) {
   for (int i = 0; i < b.P.n_ops; ++i) b.ctx->last_kinds[i] = b.P.op[i].kind;
   const int stage = WS_W_BYTES + b.NB * WS_BK * 2;
   const size_t fixed = PM_FIXED_SMEM;                     // alignment slack, barriers, descriptor copies
-  const size_t budget = (size_t)b.ctx->smem_optin;
-  const size_t ring_room = budget - fixed - (b.dense ? 0 : b.attn_bytes);
-  int stages = (int)(ring_room / stage);
+  int stages = (int)(((size_t)b.ctx->smem_optin - fixed) / stage);
   if (stages > PM_MAX_STAGES) stages = PM_MAX_STAGES;
-  if (stages < 2 || (b.dense && (size_t)stages * stage < b.attn_bytes)) return MOA_ERR_SHAPE;
+  if (stages < 2 || (size_t)stages * stage < b.attn_bytes) return MOA_ERR_SHAPE;
   b.P.stages = stages;
-  b.P.alias_attn = b.dense ? 1 : 0;
-  b.P.attn_off = b.dense ? 0u : (uint32_t)((size_t)stages * stage + (PM_FIXED_SMEM - 1024));
-  const size_t smem = fixed + (size_t)stages * stage + (b.dense ? 0 : b.attn_bytes);
-  switch (b.NB) {
-    case 32: return pm_launch_nb<32>(s, b.P, b.grid, smem);
-    case 64: return pm_launch_nb<64>(s, b.P, b.grid, smem);
-    case 128: return pm_launch_nb<128>(s, b.P, b.grid, smem);
-    default: return pm_launch_nb<256>(s, b.P, b.grid, smem);
-  }
-}
-
-// attention phase + (when it has several parts) the merge of the parts; result in the X buffer `out`
-static void pm_attention_ops(PmBuild& b, const Workspace& p, char* ws, int R, int n_seq, int rows_per_seq, int hq, int hkv,
-                             int dh, const bf16* q16, const float* q32, int q_ld, int q_gemm, const bf16* kA,
-                             const bf16* vA, int capA, int posA_ld, const int* lenA, int nA_fixed, int max_len,
-                             const bf16* kB, const bf16* vB, int capB, const int* slotsB, int slots_ld, int nB,
-                             int n_slots, bf16* out) {
-  const int group = hq / hkv, Qn = rows_per_seq * group;
-  const int q_tiles = (Qn + PM_WWARPS * 16 - 1) / (PM_WWARPS * 16);
-  const int has_tree = (kB != nullptr && nB > 0) ? 1 : 0;
-  const int blocks = imax(1, (max_len + PM_KB - 1) / PM_KB);
-  int n_split = imax(1, imin(blocks, b.grid / imax(1, n_seq * hkv * q_tiles) - has_tree));
-  const long long per_part = (long long)R * hq;
-  while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
-  if (n_split + has_tree > 1 && per_part * (n_split + has_tree) > p.att_units) { b.err = MOA_ERR_WORKSPACE; return; }
-  const int n_parts = n_split + has_tree;
-  {
-    const int q_rows = Qn < PM_WWARPS * 16 ? ((Qn + 15) & ~15) : PM_WWARPS * 16;
-    const size_t need = (size_t)2 * q_rows * dh * 2 + (size_t)2 * PM_KVST * PM_KB * dh * 2 + 512;
-    if (need > b.attn_bytes) b.attn_bytes = need;
-  }
-  PmOp* op = pm_op(b, PH_ATTN, q_gemm, R, n_seq);
-  op->p[0] = q16; op->p[1] = q32; op->p[2] = kA; op->p[3] = vA; op->p[4] = lenA; op->p[5] = kB; op->p[6] = vB;
-  op->p[7] = slotsB; op->p[8] = ws + p.att_o; op->p[9] = ws + p.att_ml; op->p[10] = out;
-  op->i[0] = q_ld; op->i[1] = hq; op->i[2] = hkv; op->i[3] = rows_per_seq; op->i[4] = capA; op->i[5] = posA_ld;
-  op->i[6] = nA_fixed; op->i[7] = capB; op->i[8] = slots_ld; op->i[9] = nB; op->i[10] = n_slots; op->i[11] = n_split;
-  op->i[12] = q_gemm >= 0 ? b.P.g[q_gemm].splits : 1; op->i[13] = b.lo_rows; op->i[14] = dh;
-  op->f[0] = 1.4426950408889634f / sqrtf((float)dh);
-  if (n_parts > 1) {
-    PmOp* c = pm_op(b, PH_COMBINE, -1, R, hq);
-    c->p[0] = ws + p.att_o; c->p[1] = ws + p.att_ml; c->p[2] = out;
-    c->i[0] = n_parts; c->i[1] = dh; c->i[2] = b.lo_rows;
-  }
+  b.P.alias_attn = 1;                                     // the attention scratch lies over the ring
+  b.P.attn_off = 0u;
+  return pm_launch_nb<256>(s, b.P, b.grid, fixed + (size_t)stages * stage);
 }
 
 // Layer Self-Attention phase: one warp per (token, query head), rows staged by bulk asynchronous copies.
-// Falls back to the general attention phase when the layer stack does not fit (S > 128).
-static void pm_lsa_attention_op(PmBuild& b, const Workspace& p, char* ws, int R, int n_tok, int S, int hq, int hkv, int dh,
-                                const bf16* qkv, int ld, bf16* out) {
+static int pm_lsa_warps(const moa_ctx* ctx, int S, int dh) {      // warps of a CTA that fit their stacks (0: none)
   const int s_pad = (S + 15) & ~15;
   const size_t per_warp = (size_t)3 * s_pad * (dh * 2 + 16) + 16;
-  const int stage = WS_W_BYTES + b.NB * WS_BK * 2;
-  const size_t avail = b.dense ? (size_t)((b.ctx->smem_optin - PM_FIXED_SMEM) / stage) * stage : (size_t)96 * 1024;
-  const int n_warps = imin(PM_WWARPS, (int)(avail / per_warp));
-  if (S > 128 || n_warps < 1) {
-    const int nq = hq * dh, nkv = hkv * dh;
-    pm_attention_ops(b, p, ws, R, n_tok, S, hq, hkv, dh, qkv, nullptr, ld, -1, qkv + nq, qkv + nq + nkv, S, ld, nullptr, S,
-                     S, nullptr, nullptr, 0, nullptr, 0, 0, 0, out);
-    return;
-  }
+  const int stage = WS_W_BYTES + 256 * WS_BK * 2;
+  const size_t avail = (size_t)((ctx->smem_optin - PM_FIXED_SMEM) / stage) * stage;
+  return S > 128 ? 0 : imin(PM_WWARPS, (int)(avail / per_warp));
+}
+static void pm_lsa_attention_op(PmBuild& b, int R, int n_tok, int S, int hq, int hkv, int dh, const bf16* qkv, int ld, bf16* out) {
+  const int s_pad = (S + 15) & ~15;
+  const size_t per_warp = (size_t)3 * s_pad * (dh * 2 + 16) + 16;
+  const int n_warps = pm_lsa_warps(b.ctx, S, dh);
+  if (n_warps < 1) { b.err = MOA_ERR_SHAPE; return; }         // ruled out by pm_usable()
   if (n_warps * per_warp > b.attn_bytes) b.attn_bytes = n_warps * per_warp;
   PmOp* op = pm_op(b, PH_LSA_ATTN, -1, R, n_tok);
   op->p[0] = qkv; op->p[1] = out;
-  op->i[0] = ld; op->i[1] = hq; op->i[2] = hkv; op->i[3] = S; op->i[4] = n_warps; op->i[5] = b.lo_rows; op->i[6] = dh;
+  op->i[0] = ld; op->i[1] = hq; op->i[2] = hkv; op->i[3] = S; op->i[4] = n_warps; op->i[5] = 0; op->i[6] = dh;
   op->f[0] = 1.4426950408889634f / sqrtf((float)dh);
 }
 
@@ -1027,119 +982,10 @@ static void pm_resnorm(PmBuild& b, int gemm, int R, int K, float* xres, const vo
                        float eps) {
   PmOp* op = pm_op(b, PH_RESNORM, gemm, R, K);
   op->p[2] = gain; op->p[3] = xres; op->p[4] = xn; op->p[5] = hidden;
-  op->i[1] = b.lo_rows; op->f[0] = eps;
+  op->i[1] = 0; op->f[0] = eps;
 }
 
-// MLP phases on xn = RMSNorm(xres): [gate | up] GEMM, SwiGLU, down GEMM. Returns the down GEMM's index.
-static int pm_mlp(PmBuild& b, const Workspace& p, char* ws, int R, int K, int F, const void* wgate, const void* wup,
-                  const void* wdown) {
-  float* part = (float*)(ws + p.part);
-  bf16* xn = (bf16*)(ws + p.xn);
-  bf16* h = (bf16*)(ws + p.narrow);
-  const void* W2[2] = {wgate, wup};
-  const int N2[2] = {F, F};
-  const int g = pm_gemm(b, xn, R, K, 2, W2, N2, 0, part, p.part_rows);
-  PmOp* op = pm_op(b, PH_SILU, g, R, F);
-  op->p[0] = h; op->i[1] = b.lo_rows;
-  const void* W1[1] = {wdown};
-  const int N1[1] = {K};
-  return pm_gemm(b, h, R, F, 1, W1, N1, 0, part, p.part_rows);
-}
-
-static moa_status draft_step_pm(moa_ctx* ctx, moa_state* st, int batch, int* topk_id, float* topk_logp, void* hidden_out,
-                                char* ws, const Workspace& p, cudaStream_t s) {
-  const moa_config& c = ctx->c;
-  const moa_weights& w = ctx->w;
-  const TreeLayout& L = ctx->tl;
-  const TreePtrs tp = tree_ptrs(st->tree, L);
-  const int step = st->step, B = c.tree_topk, D = c.tree_depth;
-  const int R = step == 0 ? batch : batch * B;
-  const int rows_per_seq = step == 0 ? 1 : B;
-  const int nbB = c.max_batch * B;
-  const int E = c.d_model, dh = c.head_dim, V = c.vocab;
-  const int cur = step & 1;
-  const int* row_tok = tp.row_tok + (size_t)cur * nbB;
-  const int* row_anc = tp.row_anc + (size_t)cur * nbB * D;
-  bf16* tk = (bf16*)((char*)st->tree + L.tk);
-  bf16* tv = (bf16*)((char*)st->tree + L.tv);
-  float* xres = (float*)(ws + p.xres);
-  bf16* xn = (bf16*)(ws + p.xn);
-  bf16* obuf = (bf16*)(ws + p.obuf);
-  float* q32 = (float*)(ws + p.q32);
-  float* part = (float*)(ws + p.part);
-  int max_sa = 0, max_ca = 0;
-  for (int b = 0; b < batch; ++b) {
-    max_sa = imax(max_sa, st->sa_len_host[b]);
-    max_ca = imax(max_ca, st->ca_len_host[b]);
-  }
-  PmBuild b;
-  pm_init(b, ctx, R, false, st->tree, L, ws, p);
-  const int nq = c.sa_hq * dh, nkv = c.sa_hkv * dh, cq = c.ca_hq * dh, ckv = c.ca_hkv * dh;
-  // ---- self-attention block ----
-  {
-    PmOp* op = pm_op(b, PH_EMBED_NORM, -1, R, E);
-    op->p[0] = w.embed; op->p[1] = row_tok; op->p[2] = w.sa_norm1; op->p[3] = xres; op->p[4] = xn;
-    op->i[0] = V; op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
-  }
-  {
-    const void* W3[3] = {w.sa_wq, w.sa_wk, w.sa_wv};
-    const int N3[3] = {nq, nkv, nkv};
-    const int g = pm_gemm(b, xn, R, E, 3, W3, N3, 0, part, p.part_rows);
-    PmOp* op = pm_op(b, PH_ROPE, g, R, nq + 2 * nkv);
-    op->p[0] = q32; op->p[1] = tk; op->p[2] = tv; op->p[3] = st->sa_len;
-    op->i[0] = c.sa_hq; op->i[1] = c.sa_hkv; op->i[2] = dh; op->i[3] = step; op->i[4] = B; op->i[5] = L.NS;
-    op->f[0] = c.sa_rope_theta;
-  }
-  pm_attention_ops(b, p, ws, R, batch, rows_per_seq, c.sa_hq, c.sa_hkv, dh, nullptr, q32, nq, -1, (const bf16*)st->sa_k,
-                   (const bf16*)st->sa_v, c.max_ctx, nkv, st->sa_len, 0, max_sa, tk, tv, L.NS, row_anc, D, step + 1,
-                   step == 0 ? 1 : 1 + step * B, obuf);
-  {
-    const void* W1[1] = {w.sa_wo};
-    const int N1[1] = {E};
-    const int g = pm_gemm(b, obuf, R, nq, 1, W1, N1, 0, part, p.part_rows);
-    pm_resnorm(b, g, R, E, xres, w.sa_norm2, xn, nullptr, c.rms_eps);
-  }
-  {
-    const int g = pm_mlp(b, p, ws, R, E, c.sa_mlp, w.sa_wgate, w.sa_wup, w.sa_wdown);
-    // ---- cross-attention block ----
-    pm_resnorm(b, g, R, E, xres, w.ca_normq, xn, nullptr, c.rms_eps);
-  }
-  {
-    const void* W1[1] = {w.ca_wq};
-    const int N1[1] = {cq};
-    const int g = pm_gemm(b, xn, R, E, 1, W1, N1, 0, part, p.part_rows);
-    pm_attention_ops(b, p, ws, R, batch, rows_per_seq, c.ca_hq, c.ca_hkv, dh, nullptr, part, cq, g, (const bf16*)st->ca_k,
-                     (const bf16*)st->ca_v, c.max_ctx, ckv, st->ca_len, 0, max_ca, nullptr, nullptr, 0, nullptr, 0, 0, 0,
-                     obuf);
-  }
-  {
-    const void* W1[1] = {w.ca_wo};
-    const int N1[1] = {E};
-    const int g = pm_gemm(b, obuf, R, cq, 1, W1, N1, 0, part, p.part_rows);
-    pm_resnorm(b, g, R, E, xres, w.ca_norm2, xn, nullptr, c.rms_eps);
-  }
-  {
-    const int g = pm_mlp(b, p, ws, R, E, c.ca_mlp, w.ca_wgate, w.ca_wup, w.ca_wdown);
-    // ---- LM head, log-softmax, top-B ----
-    pm_resnorm(b, g, R, E, xres, w.final_norm, xn, hidden_out, c.rms_eps);
-  }
-  {
-    const void* W1[1] = {w.lm_head};
-    const int N1[1] = {V};
-    const int g = pm_gemm(b, xn, R, E, 1, W1, N1, 1, nullptr, 0);
-    PmGemm& G = b.P.g[g];
-    G.B = B;
-    G.p_max = (float*)(ws + p.pmax); G.p_sum = (float*)(ws + p.psum);
-    G.c_val = (float*)(ws + p.cval); G.c_id = (int*)(ws + p.cid);
-    G.n_sub = 4 * G.tiles_total;
-    if (G.n_sub > PM_MERGE_OWN * PM_WORKERS) return MOA_ERR_SHAPE;       // ruled out by pm_usable()
-    PmOp* op = pm_op(b, PH_MERGE, g, R, V);
-    op->p[0] = topk_id; op->p[1] = topk_logp; op->i[1] = B;
-  }
-  return pm_launch(b, s);
-}
-
-// One LSA pass over nt tokens (rows t0*S .. of h_stack): small regime (split planes + glue) or dense regime.
+// One LSA pass over nt tokens (rows t0*S .. of h_stack) in the dense regime (more than 256 rows).
 static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt, int t0, const SeqSplit& split,
                               bf16* kv_out, char* ws, const Workspace& p, cudaStream_t s) {
   const moa_config& c = ctx->c;
@@ -1148,7 +994,6 @@ static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt
   const int S = c.n_stack, D = c.d_stack, dh = c.head_dim, F = c.lsa_mlp;
   const int nq = c.lsa_hq * dh, nkv = c.lsa_hkv * dh, ld = nq + 2 * nkv, ckv = c.ca_hkv * dh;
   const int R = nt * S;
-  const bool dense = R > 256;
   float* xres = (float*)(ws + p.xres);
   bf16* xn = (bf16*)(ws + p.xn);
   bf16* narrow = (bf16*)(ws + p.narrow);
@@ -1157,51 +1002,39 @@ static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt
   float* kvf = (float*)(ws + p.kvf);
   bf16* kvn = (bf16*)(ws + p.kvn);
   PmBuild b;
-  pm_init(b, ctx, R, dense, st->tree, L, ws, p);
+  pm_init(b, ctx, st->tree, L, ws, p);
   b.P.split = split;
   {
     PmOp* op = pm_op(b, PH_ROWS_NORM, -1, R, D);
     op->p[0] = x; op->p[2] = w.lsa_norm1; op->p[3] = xres; op->p[4] = xn;
-    op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
+    op->i[1] = 0; op->f[0] = c.rms_eps;
   }
   const void* W3[3] = {w.lsa_wq, w.lsa_wk, w.lsa_wv};
   const int N3[3] = {nq, nkv, nkv};
   const void* Wo[1] = {w.lsa_wo};
   const int No[1] = {D};
-  int g_down;
-  if (!dense) {
-    const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 0, part, p.part_rows);
-    PmOp* op = pm_op(b, PH_SUMCAST, g0, R, ld);
-    op->p[0] = narrow;
-    pm_lsa_attention_op(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, ld, obuf);
-    const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 0, part, p.part_rows);
-    pm_resnorm(b, g1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
-    g_down = pm_mlp(b, p, ws, R, D, F, w.lsa_wgate, w.lsa_wup, w.lsa_wdown);
-  } else {
-    const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 2, nullptr, 0);
-    b.P.g[g0].out16 = narrow; b.P.g[g0].ld16 = ld;
-    pm_lsa_attention_op(b, p, ws, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, ld, obuf);
-    const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 3, xres, 0);
-    b.P.g[g1].ldo = D;
-    pm_resnorm(b, -1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
-    const void* W2[2] = {w.lsa_wgate, w.lsa_wup};
-    const int N2[2] = {F, F};
-    const int g2 = pm_gemm(b, xn, R, D, 2, W2, N2, 4, nullptr, 0);
-    b.P.g[g2].out16 = narrow; b.P.g[g2].ld16 = F;
-    const void* Wd[1] = {w.lsa_wdown};
-    const int g3 = pm_gemm(b, narrow, R, F, 1, Wd, No, 3, xres, 0);
-    b.P.g[g3].ldo = D;
-    g_down = -1;
-  }
+  const int g0 = pm_gemm(b, xn, R, D, 3, W3, N3, 2, nullptr, 0);
+  b.P.g[g0].out16 = narrow; b.P.g[g0].ld16 = ld;
+  pm_lsa_attention_op(b, R, nt, S, c.lsa_hq, c.lsa_hkv, dh, narrow, ld, obuf);
+  const int g1 = pm_gemm(b, obuf, R, nq, 1, Wo, No, 3, xres, 0);
+  b.P.g[g1].ldo = D;
+  pm_resnorm(b, -1, R, D, xres, w.lsa_norm2, xn, nullptr, c.rms_eps);
+  const void* W2[2] = {w.lsa_wgate, w.lsa_wup};
+  const int N2[2] = {F, F};
+  const int g2 = pm_gemm(b, xn, R, D, 2, W2, N2, 4, nullptr, 0);
+  b.P.g[g2].out16 = narrow; b.P.g[g2].ld16 = F;
+  const void* Wd[1] = {w.lsa_wdown};
+  const int g3 = pm_gemm(b, narrow, R, F, 1, Wd, No, 3, xres, 0);
+  b.P.g[g3].ldo = D;
   {
-    PmOp* op = pm_op(b, PH_MEAN_NORM, g_down, nt, D);
+    PmOp* op = pm_op(b, PH_MEAN_NORM, -1, nt, D);
     op->p[0] = xres; op->p[1] = kvf; op->p[2] = kv_out; op->p[3] = w.ca_normkv; op->p[4] = kvn;
-    op->i[0] = S; op->i[1] = b.lo_rows; op->f[0] = c.rms_eps;
+    op->i[0] = S; op->i[1] = 0; op->f[0] = c.rms_eps;
   }
   {
-    const void* W2[2] = {w.ca_wk, w.ca_wv};
-    const int N2[2] = {ckv, ckv};
-    const int g = pm_gemm(b, kvn, nt, D, 2, W2, N2, 0, part, p.part_rows);
+    const void* Wkv[2] = {w.ca_wk, w.ca_wv};
+    const int Nkv[2] = {ckv, ckv};
+    const int g = pm_gemm(b, kvn, nt, D, 2, Wkv, Nkv, 0, part, p.part_rows);
     PmOp* op = pm_op(b, PH_CACHE_APPEND, g, nt, 2 * ckv);
     op->p[0] = st->ca_len; op->p[1] = st->ca_k; op->p[2] = st->ca_v;
     op->i[0] = ckv; op->i[1] = c.max_ctx; op->i[2] = t0;
@@ -1212,17 +1045,12 @@ static moa_status lsa_pass_pm(moa_ctx* ctx, moa_state* st, const bf16* x, int nt
 static bool pm_usable(const moa_ctx* ctx) {
   if (!ctx->fast || !ctx->coop || ctx->c.dtype != MOA_BF16 || ctx->sm_count > 256) return false;
   const moa_weights& w = ctx->w;
-  const void* all[] = {w.lm_head, w.lsa_wq, w.lsa_wk, w.lsa_wv, w.lsa_wo, w.lsa_wgate, w.lsa_wup, w.lsa_wdown,
-                       w.sa_wq, w.sa_wk, w.sa_wv, w.sa_wo, w.sa_wgate, w.sa_wup, w.sa_wdown,
-                       w.ca_wq, w.ca_wk, w.ca_wv, w.ca_wo, w.ca_wgate, w.ca_wup, w.ca_wdown};
+  const void* all[] = {w.lsa_wq, w.lsa_wk, w.lsa_wv, w.lsa_wo, w.lsa_wgate, w.lsa_wup, w.lsa_wdown, w.ca_wk, w.ca_wv};
   for (const void* m : all)
     if (!find_wmap(ctx, m)) return false;
   const moa_config& c = ctx->c;
-  const int widths[] = {c.d_model, c.d_stack, c.lsa_mlp, c.sa_mlp, c.ca_mlp};
-  for (int v : widths)
-    if (v % 64 != 0) return false;
-  if (4 * ((c.vocab + WS_BM - 1) / WS_BM) > PM_MERGE_OWN * PM_WORKERS) return false;
-  return true;
+  if (c.d_stack % 64 != 0 || c.lsa_mlp % 64 != 0) return false;
+  return pm_lsa_warps(ctx, c.n_stack, c.head_dim) >= 1;       // a token's stack of q, k, v rows fits in shared memory
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1304,7 +1132,6 @@ moa_status moa_create(const moa_config* cfg, const moa_weights* w, moa_ctx** out
   ctx->coop = prop.cooperativeLaunch != 0;
   ctx->smem_optin = (int)prop.sharedMemPerBlockOptin;
   ctx->last_n_ops = 0;
-  ctx->fused_step = false;
   ctx->n_wmap_base = 0;
   memset(&ctx->tli, 0, sizeof(ctx->tli));
   memset(ctx->tli_w, 0, sizeof(ctx->tli_w));
@@ -1494,12 +1321,6 @@ moa_status moa_trace_end(int32_t* n_out) {
 #endif
 }
 
-moa_status moa_set_option(moa_ctx* ctx, int32_t option, int32_t value) {
-  if (!ctx) return MOA_ERR_NULL;
-  if (option == MOA_OPT_FUSED_STEP) { ctx->fused_step = value != 0; return MOA_OK; }
-  return MOA_ERR_SHAPE;
-}
-
 moa_status moa_profile_phases(moa_ctx* ctx, const void* ws, size_t ws_bytes, int32_t cap, double* us_out,
                               double* wait_us_out, int32_t* kind_out, int32_t* n_out, void* stream) {
   if (!ctx || !ws || !us_out || !kind_out || !n_out) return MOA_ERR_NULL;
@@ -1576,6 +1397,7 @@ moa_status moa_state_set_len(moa_ctx* ctx, moa_state* st, int32_t which, const i
 
 moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, const int32_t* n_tok_host, int32_t batch,
                            void* kv_out, void* ws, size_t ws_bytes, void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!n_tok_host || !ws) return MOA_ERR_NULL;
   SeqSplit split;
@@ -1591,7 +1413,7 @@ moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, con
   moa_status r;
   // Passes with more than 256 (token, layer) rows run as one persistent kernel with tensor-core GEMMs whose
   // epilogues are fused (dense regime); smaller ones take the weight-streaming kernels launch by launch.
-  if (pm_usable(ctx) && ((long long)imin(p.chunk_tok, total) * ctx->c.n_stack > 256 || ctx->fused_step)) {
+  if (pm_usable(ctx) && (long long)imin(p.chunk_tok, total) * ctx->c.n_stack > 256) {
     r = MOA_OK;
     const int S = ctx->c.n_stack, D = ctx->c.d_stack;
     // passes of at most 256 tokens (the key/value projection of a pass is one activation block)
@@ -1617,6 +1439,7 @@ moa_status moa_lsa_forward(moa_ctx* ctx, moa_state* st, const void* h_stack, con
 
 moa_status moa_sa_append(moa_ctx* ctx, moa_state* st, const int32_t* tok, const int32_t* n_host, int32_t batch, void* ws,
                          size_t ws_bytes, void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!n_host || !ws) return MOA_ERR_NULL;
   SeqSplit split;
@@ -1637,6 +1460,7 @@ moa_status moa_sa_append(moa_ctx* ctx, moa_state* st, const int32_t* tok, const 
 
 moa_status moa_drafter_prefill(moa_ctx* ctx, moa_state* st, const int32_t* tok, const int32_t* n_host, int32_t batch,
                                const int32_t* ca_limit, void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!n_host || !ws || !hidden_out) return MOA_ERR_NULL;
   SeqSplit split;
@@ -1657,6 +1481,7 @@ moa_status moa_drafter_prefill(moa_ctx* ctx, moa_state* st, const int32_t* tok, 
 }
 
 moa_status moa_tree_begin(moa_ctx* ctx, moa_state* st, const int32_t* root_tok, int32_t batch, void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!root_tok) return MOA_ERR_NULL;
   for (int b = 0; b < batch; ++b)
@@ -1671,6 +1496,7 @@ moa_status moa_tree_begin(moa_ctx* ctx, moa_state* st, const int32_t* root_tok, 
 
 moa_status moa_draft_step(moa_ctx* ctx, moa_state* st, int32_t batch, int32_t* topk_id, float* topk_logp,
                           void* hidden_out, void* ws, size_t ws_bytes, void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!topk_id || !topk_logp || !ws) return MOA_ERR_NULL;
   if (!aligned16(topk_id) || !aligned16(topk_logp) || !aligned16(hidden_out) || !aligned16(ws)) return MOA_ERR_ALIGN;
@@ -1678,11 +1504,6 @@ moa_status moa_draft_step(moa_ctx* ctx, moa_state* st, int32_t batch, int32_t* t
   const int chunk = chunk_from_bytes(ctx->c, ctx->tli, ctx->elt, ws_bytes);
   if (chunk < 1) return MOA_ERR_WORKSPACE;
   const Workspace p = plan_workspace(ctx->c, ctx->tli, ctx->elt, chunk);
-  // The single-kernel forward exists and is parity-tested, but with few rows the chain of separate launches is
-  // the faster of the two on B200 as measured (421 us against 620 us per forward at the Llama-3-8B shape), so the
-  // fused kernel is taken only on request.
-  if (ctx->fused_step && ctx->tli.n_layers == 0 && pm_usable(ctx))
-    return draft_step_pm(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream);
   return ctx->c.dtype == MOA_F32
              ? draft_step_t<float>(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream)
              : draft_step_t<bf16>(ctx, st, batch, topk_id, topk_logp, hidden_out, (char*)ws, p, (cudaStream_t)stream);
@@ -1691,6 +1512,7 @@ moa_status moa_draft_step(moa_ctx* ctx, moa_state* st, int32_t batch, int32_t* t
 moa_status moa_tree_expand(moa_ctx* ctx, moa_state* st, int32_t batch, const int32_t* topk_id, const float* topk_logp,
                            int32_t* out_tok, int32_t* out_parent, int32_t* out_depth, float* out_score, int32_t* out_n,
                            void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!topk_id || !topk_logp) return MOA_ERR_NULL;
   if (st->step < 0 || st->step >= ctx->c.tree_depth) return MOA_ERR_STATE;
@@ -1711,6 +1533,7 @@ moa_status moa_tree_expand(moa_ctx* ctx, moa_state* st, int32_t batch, const int
 
 moa_status moa_tree_attn_mask(const int32_t* parent, int32_t batch, int32_t n, void* mask_out, int32_t packed,
                               void* stream) {
+  MOA_RANGE();
   if (!parent || !mask_out) return MOA_ERR_NULL;
   if (batch < 0 || n < 0 || (long long)batch * n > 0x3fffffff) return MOA_ERR_SHAPE;
   if (packed != 0 && packed != 1) return MOA_ERR_SHAPE;
@@ -1756,6 +1579,7 @@ static moa_status sa_static_scratch(void** out) {
 
 moa_status moa_sa_append_static(moa_ctx* ctx, moa_state* st, const int32_t* tok, const int32_t* n_host, int32_t batch,
                                 void* stream) {
+  MOA_RANGE();
   MOA_TRY(check_state(ctx, st, batch));
   if (!n_host) return MOA_ERR_NULL;
   SeqSplit split;
@@ -1795,16 +1619,18 @@ moa_status moa_sa_append_static(moa_ctx* ctx, moa_state* st, const int32_t* tok,
 moa_status moa_verify_greedy(const int32_t* tok, const int32_t* parent, int32_t batch, int32_t n, const void* target_logits,
                              int32_t logits_dtype, int32_t vocab, int32_t cap, int32_t* choice, int32_t* acc_slot,
                              int32_t* acc_tok, int32_t* acc_len, int32_t* next_tok, void* stream) {
+  MOA_RANGE();
   if (!tok || !parent || !target_logits || !choice || !acc_slot || !acc_tok || !acc_len || !next_tok) return MOA_ERR_NULL;
   if (batch <= 0 || batch > MOA_MAX_BATCH || n <= 0 || vocab <= 0 || cap <= 0) return MOA_ERR_SHAPE;
   if (logits_dtype != MOA_F32 && logits_dtype != MOA_BF16) return MOA_ERR_DTYPE;
   if ((long long)batch * n > 65535) return MOA_ERR_SHAPE;          // one cluster per row along gridDim.y
   cudaStream_t s = (cudaStream_t)stream;
   // few rows: a cluster of CTAs per row, so that the rows fill the GPU; many rows: one CTA per row
-  int sms = 148;
-  {
-    int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  static int sms_of[64];                 // SM count per device, asked for once (the entry point has no context)
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+    if (sms_of[dev] == 0) cudaDeviceGetAttribute(&sms_of[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (sms_of[dev] > 0) sms = sms_of[dev];
   }
   const int rows = batch * n;
   const bool spread = rows < 4 * sms;
@@ -1823,6 +1649,7 @@ moa_status moa_verify_greedy(const int32_t* tok, const int32_t* parent, int32_t 
 }
 
 moa_status moa_pack_tree(const int32_t* tok, const int32_t* parent, int64_t count, void* msg, void* stream) {
+  MOA_RANGE();
   if (!tok || !parent || !msg) return MOA_ERR_NULL;
   if (count < 0 || count > (1ll << 31)) return MOA_ERR_SHAPE;
   if ((uintptr_t)msg & 3u) return MOA_ERR_ALIGN;
@@ -1834,6 +1661,7 @@ moa_status moa_pack_tree(const int32_t* tok, const int32_t* parent, int64_t coun
 }
 
 moa_status moa_unpack_tree(const void* msg, int64_t count, int32_t* tok, int32_t* parent, void* stream) {
+  MOA_RANGE();
   if (!tok || !parent || !msg) return MOA_ERR_NULL;
   if (count < 0 || count > (1ll << 31)) return MOA_ERR_SHAPE;
   if ((uintptr_t)msg & 3u) return MOA_ERR_ALIGN;
@@ -1846,6 +1674,7 @@ moa_status moa_unpack_tree(const void* msg, int64_t count, int32_t* tok, int32_t
 
 moa_status moa_quantize_rows(const void* x, int32_t dtype, int64_t rows, int32_t width, int8_t* codes, float* scales,
                              void* stream) {
+  MOA_RANGE();
   if (!x || !codes || !scales) return MOA_ERR_NULL;
   if (dtype != MOA_F32 && dtype != MOA_BF16) return MOA_ERR_DTYPE;
   if (rows < 0 || width <= 0 || rows > (1ll << 31)) return MOA_ERR_SHAPE;
@@ -1865,6 +1694,7 @@ moa_status moa_quantize_rows(const void* x, int32_t dtype, int64_t rows, int32_t
 
 moa_status moa_dequantize_rows(const int8_t* codes, const float* scales, int64_t rows, int32_t width, void* out, int32_t dtype,
                                void* stream) {
+  MOA_RANGE();
   if (!out || !codes || !scales) return MOA_ERR_NULL;
   if (dtype != MOA_F32 && dtype != MOA_BF16) return MOA_ERR_DTYPE;
   if (rows < 0 || width <= 0 || rows > (1ll << 31)) return MOA_ERR_SHAPE;

@@ -38,6 +38,7 @@ struct AttnParams {
   bf16* out;                             // [R, hq*DH]
   int out_lo;                            // > 0: the low-order term of every output goes to row out_lo + r
   float scale_log2;                      // log2(e) / sqrt(DH)
+  int* status;                           // device status word (debug-build index checks)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
@@ -102,6 +103,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
   int k_begin, k_end;
   if (!tree_part) {
     const int len = P.lenA ? P.lenA[seq] : P.nA_fixed;
+    if (threadIdx.x == 0) MOA_DEV_CHECK(len >= 0 && len <= P.capA, P.status);
     const int blocks = (len + AT_KB - 1) / AT_KB;
     const int b0 = (int)(((long long)part * blocks) / P.n_split), b1 = (int)(((long long)(part + 1) * blocks) / P.n_split);
     k_begin = b0 * AT_KB;
@@ -119,6 +121,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
       const int r = seq * P.rows_per_seq + threadIdx.x;
       for (int i = 0; i < P.nB; ++i) {
         const int slot = P.slotsB[(size_t)r * P.slots_ld + i];
+        MOA_DEV_CHECK(slot >= 0 && slot < P.n_slots && slot < P.capB, P.status);
         if (slot >= 0 && slot < 256) allow[threadIdx.x][slot >> 6] |= 1ull << (slot & 63);
       }
     }

@@ -44,7 +44,8 @@ constexpr int RN_CHUNKS = 8;     // 8-element chunks of a row one thread of a 25
 template <typename TIN, typename T>
 __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict__ x, const int* __restrict__ tok,
                                                            int vocab, const T* __restrict__ gain, int K, float eps,
-                                                           float* __restrict__ res_out, T* __restrict__ y, int lo_rows) {
+                                                           float* __restrict__ res_out, T* __restrict__ y, int lo_rows,
+                                                           int* __restrict__ status) {
   pdl_trigger();
   pdl_wait(KID_NORM);
   __shared__ float red[33];
@@ -52,6 +53,7 @@ __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const TIN* __restrict
   const TIN* xr;
   if (tok != nullptr) {
     int t = tok[r];
+    if (threadIdx.x == 0) MOA_DEV_CHECK(t >= 0 && t < vocab, status);
     t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
     xr = x + (size_t)t * K;
   } else {
@@ -356,6 +358,7 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
     seq = rr.step == 0 ? r : r / rr.B;
     pos_add = rr.step;
     const int slot = rr.step == 0 ? 0 : 1 + (rr.step - 1) * rr.B + (r % rr.B);
+    if (threadIdx.x == 0 && blockIdx.y == 0) MOA_DEV_CHECK(slot < rr.slots, status);
     dst = (size_t)seq * rr.slots + slot;
   } else {
     const int t = rr.row0 + r;

@@ -187,4 +187,16 @@ struct SeqSplit {
 // Device-side status word values (mirrors moa_status where it matters).
 enum : int { DEV_OK = 0, DEV_ERR_BOUNDS = 6, DEV_ERR_TIMEOUT = 10 };
 
+// Debug build (-DMOA_CHECKS): indices that the host logic guarantees (token ids, tree slots, cache lengths) are
+// checked where they are used; a violation raises the status word and the access is skipped or clamped as in the
+// normal build. Without the flag the macro costs nothing.
+#ifdef MOA_CHECKS
+#define MOA_DEV_CHECK(cond, status_ptr)                                          \
+  do {                                                                           \
+    if (!(cond) && (status_ptr) != nullptr) atomicMax((status_ptr), DEV_ERR_BOUNDS); \
+  } while (0)
+#else
+#define MOA_DEV_CHECK(cond, status_ptr) do { } while (0)
+#endif
+
 }  // namespace moa

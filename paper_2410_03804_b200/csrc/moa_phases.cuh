@@ -1,26 +1,24 @@
-// Phase machine: one persistent cooperative kernel that runs a whole drafter forward (or a whole LSA
-// pass) as a list of phases separated by grid-wide barriers.
+// Phase machine: one persistent cooperative kernel that runs a whole LSA pass of more than 256 (token, layer)
+// rows -- the dense regime, where the projections are tensor-core-bound GEMMs -- as a list of phases separated by
+// grid-wide barriers.
 //
-// Why one kernel: a draft step at batch 1 is a chain of ~22 dependent operations, most of them a few
-// microseconds long, around ~1.4 GB of weights that should stream from HBM without a pause. Separate
-// launches drain and refill the memory pipeline at every link of the chain. Here one CTA per SM stays
-// resident for the whole step and
+// Why one kernel: the pass is six GEMMs with fused epilogues and four short glue phases over the same rows;
+// separate launches would write and re-read every intermediate through HBM and drain the tensor pipe at every
+// link. Here one CTA per SM stays resident for the whole pass and
 //   warp 0      streams weight tiles with TMA along the STATIC schedule of all GEMM phases, running ahead
 //               of the phase that is executing (weights depend on nothing), as far as the shared-memory
 //               ring allows; only the small activation tile of a stage waits for its phase to open;
 //   warp 1      issues tcgen05.mma (weights = A operand, M = 128; activation rows = B operand);
 //   warps 2..5  drain the TMEM accumulators (epilogues), and together with
-//   warps 6..7  execute the glue phases (norms, rotary, SwiGLU, attention, merges) between the GEMMs.
+//   warps 6..7  execute the glue phases (norms, layer self-attention, layer mean, cache append) between the GEMMs.
 // Phases are separated by a grid barrier (one atomic arrival per CTA; the last arrival raises a flag per
 // CTA, each on its own cache line; bounded polling; the launch is cooperative so all CTAs are resident).
 // Every wait is bounded: on expiry a CTA raises the abort word, every CTA drains, frees TMEM and returns,
 // and the status word reads MOA_ERR_TIMEOUT.
 #pragma once
-#include "moa_pm_attn.cuh"
 #include "moa_pm_common.cuh"
 #include "moa_pm_glue.cuh"
 #include "moa_pm_lsa.cuh"
-#include "moa_pm_merge.cuh"
 
 namespace moa {
 
@@ -31,10 +29,9 @@ namespace moa {
 template <int NB>
 __host__ __device__ constexpr int pm_acc() { return NB <= 64 ? 4 : (NB <= 128 ? 2 : 1); }
 
-// 16 accumulator columns starting at column c of the unit's buffer: sum over the independent accumulators and,
-// for a split X buffer, over the hi and lo halves.
+// 16 accumulator columns starting at column c of the unit's buffer: sum over the independent accumulators.
 template <int NB>
-__device__ __forceinline__ void pm_ld16(uint32_t taddr, int c, int xsplit, float* v) {
+__device__ __forceinline__ void pm_ld16(uint32_t taddr, int c, float* v) {
   tc_ld16(taddr + c, v);
 #pragma unroll
   for (int a = 1; a < pm_acc<NB>(); ++a) {
@@ -42,15 +39,6 @@ __device__ __forceinline__ void pm_ld16(uint32_t taddr, int c, int xsplit, float
     tc_ld16(taddr + a * NB + c, w);
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] += w[i];
-  }
-  if (xsplit) {
-#pragma unroll
-    for (int a = 0; a < pm_acc<NB>(); ++a) {
-      float w[16];
-      tc_ld16(taddr + a * NB + NB / 2 + c, w);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] += w[i];
-    }
   }
 }
 
@@ -66,7 +54,7 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
 #pragma unroll 1
     for (int c0 = 0; c0 < rows; c0 += 16) {
       float v[16];
-      pm_ld16<NB>(taddr, c0, Gm.xsplit, v);
+      pm_ld16<NB>(taddr, c0, v);
       if (valid) {
 #pragma unroll
         for (int i = 0; i < 16; ++i)
@@ -78,7 +66,7 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
 #pragma unroll 1
     for (int c0 = 0; c0 < rows; c0 += 16) {
       float v[16];
-      pm_ld16<NB>(taddr, c0, 0, v);
+      pm_ld16<NB>(taddr, c0, v);
       if (valid) {
         if (Gm.mode == 2) {
 #pragma unroll
@@ -106,48 +94,6 @@ __device__ __forceinline__ void pm_epilogue(const PmGemm& Gm, const PmUnit& d, u
         for (int i = 0; i < 16; ++i)
           if (c0 + i < rows)
             Gm.out16[(size_t)(r0 + c0 + i) * Gm.ld16 + nrow] = __float2bfloat16_rn(gt[i] / (1.f + __expf(-gt[i])) * up[i]);
-      }
-    }
-  } else {
-    // LM head: per 32 vocabulary rows and activation row: max, sum of exponentials, sorted B best (logit, id)
-    const int sub = d.tile * 4 + q;
-    const int B = Gm.B;
-#pragma unroll 1
-    for (int c0 = 0; c0 < rows; c0 += 16) {
-      float v[16];
-      pm_ld16<NB>(taddr, c0, Gm.xsplit, v);
-#pragma unroll 1
-      for (int i = 0; i < 16; ++i) {
-        const int r = c0 + i;
-        if (r >= rows) break;
-        float val = valid ? v[i] : -INFINITY;
-        int id = nrow;
-        const float wmax = warp_max(val);
-        const float e = (valid && wmax > -INFINITY) ? __expf(val - wmax) : 0.f;
-        const float wsum = warp_sum(e);
-        // bitonic sort of the 32 (value, id) pairs: best (largest value, then smallest id) ends in lane 0
-#pragma unroll
-        for (int k = 2; k <= 32; k <<= 1) {
-#pragma unroll
-          for (int jj = k >> 1; jj > 0; jj >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, val, jj);
-            const int oi = __shfl_xor_sync(0xffffffffu, id, jj);
-            const bool lower = (lane & jj) == 0;
-            const bool up = (lane & k) == 0;
-            const bool want_better = lower == up;
-            const bool other_better = ranks_before(ov, oi, val, id);
-            if (want_better == other_better) { val = ov; id = oi; }
-          }
-        }
-        const size_t at = (size_t)r * Gm.n_sub + sub;
-        if (lane < B) {
-          Gm.c_val[at * B + lane] = val;
-          Gm.c_id[at * B + lane] = id;
-        }
-        if (lane == 0) {
-          Gm.p_max[at] = wmax;
-          Gm.p_sum[at] = wsum;
-        }
       }
     }
   }

@@ -1,14 +1,8 @@
 // Phase machine, part 1: descriptors, small device helpers and the static GEMM schedule.
 //
-// The phase machine is one persistent cooperative kernel that runs a whole drafter forward (or a whole
-// LSA pass) as a list of phases separated by grid-wide barriers; see moa_phases.cuh for the kernel and
-// the reasons. This file holds what its parts share.
-//
-// Activation operands ("X buffers") may carry each value as TWO bf16 terms, hi + lo, where lo is what
-// hi's 8-bit mantissa dropped. The MMA then runs over N = 2 x padded rows and the epilogue adds the two
-// column halves, so activations enter every product with ~16 bits of mantissa while weights and caches
-// stay in their 16-bit storage type. With few rows this is free: the stream is HBM-bound and N only
-// grows from 16 to 32.
+// The phase machine is one persistent cooperative kernel that runs a whole LSA pass of more than 256 (token,
+// layer) rows as a list of phases separated by grid-wide barriers; see moa_phases.cuh for the kernel and the
+// reasons. This file holds what its parts share.
 #pragma once
 #include "moa_attn.cuh"
 #include "moa_basic.cuh"
@@ -19,17 +13,13 @@ namespace moa {
 constexpr int PM_THREADS = 256;
 constexpr int PM_WORKERS = 192;          // warps 2..7
 constexpr int PM_WWARPS = 6;
-constexpr int PM_MAX_OPS = 28;
+constexpr int PM_MAX_OPS = 16;
 constexpr int PM_MAX_GEMMS = 10;
 constexpr int PM_MAX_STAGES = 12;
-constexpr int PM_KB = 32;                // keys per attention block
-constexpr int PM_KVST = 2;               // key/value blocks in flight per attention unit
 constexpr int PM_MAXCH = 6;              // 8-element chunks a thread keeps of one row (rows up to 9216 wide)
-constexpr int PM_MERGE_OWN = 24;         // vocabulary slices one thread owns in the LM-head merge
 
 enum PmKind : int {
-  PH_GEMM = 0, PH_EMBED_NORM, PH_ROWS_NORM, PH_RESNORM, PH_ROPE, PH_ATTN, PH_COMBINE, PH_SILU, PH_SUMCAST,
-  PH_MEAN_NORM, PH_CACHE_APPEND, PH_MERGE, PH_LSA_ATTN
+  PH_GEMM = 0, PH_ROWS_NORM, PH_RESNORM, PH_MEAN_NORM, PH_CACHE_APPEND, PH_LSA_ATTN
 };
 
 struct PmGemm {            // (its tensor maps are PmParams.tm[gemm][0..2] weights, [3] activations)
@@ -37,19 +27,14 @@ struct PmGemm {            // (its tensor maps are PmParams.tm[gemm][0..2] weigh
   int tiles_total;         // weight tiles (gated: gate/up tile pairs)
   int kb_total, splits, row_blocks;
   int units, rot;          // tiles_total * splits * row_blocks; unit u runs on CTA (u + rot) % grid
-  int mode;                // 0 fp32 split planes, 1 LM-head partial top-B, 2 bf16 store, 3 residual add, 4 gated SwiGLU
+  int mode;                // 0 fp32 split planes, 2 bf16 store, 3 residual add, 4 gated SwiGLU
   int R;                   // valid activation rows
-  int xsplit;              // X buffer carries hi | lo halves (lo rows start at NB/2)
   int rows_per_block;      // X rows per unit: NB, or 128 when gated
   int ldo;                 // modes 0, 3: leading dimension of out
   int ld16;                // modes 2, 4
-  int B;                   // mode 1
-  int n_sub;               // mode 1: partial lists per activation row
   size_t plane;            // mode 0: elements between split planes
   float* out;              // mode 0: planes; mode 3: fp32 residual stream
   bf16* out16;             // modes 2, 4
-  float *p_max, *p_sum, *c_val;   // mode 1: [R][n_sub], [R][n_sub], [R][n_sub][B]
-  int* c_id;
 };
 
 struct PmOp {

@@ -1,5 +1,4 @@
-// Phase machine, part 2: the glue phases between the GEMMs (norms, rotary, SwiGLU, layer mean, cache
-// append). Each is executed by the 192 worker threads of every CTA; its units are spread over the grid.
+// Phase machine, part 2: the glue phases between the GEMMs (norms, layer mean, cache append). Each is executed by the 192 worker threads of every CTA; its units are spread over the grid.
 // Everything another CTA wrote earlier in the same launch is read with ld.global.cg (past L1).
 #pragma once
 #include "moa_pm_common.cuh"
@@ -7,18 +6,17 @@
 namespace moa {
 
 // Row normalisation family. One CTA per row (or one warp per row when there are many rows).
-//  source of row r:  embed[tok[r]] (PH_EMBED_NORM) | x[r] (PH_ROWS_NORM) | xres[r] + split planes (PH_RESNORM)
-//  p[0] src (bf16 table / rows), p[1] tok, p[2] gain (bf16) or null, p[3] xres (fp32) or null, p[4] xbuf or null,
-//  p[5] hidden_out (bf16) or null; i[0] vocab, i[1] lo_rows; f[0] eps.
+//  source of row r:  x[r] (PH_ROWS_NORM) | xres[r] + split planes (PH_RESNORM)
+//  p[0] src rows (bf16), p[2] gain (bf16) or null, p[3] xres (fp32) or null, p[4] xbuf or null,
+//  p[5] hidden_out (bf16) or null; i[1] lo_rows; f[0] eps.
 __device__ __noinline__ void pm_norm_rows(PmSmem& S, const PmOp& op, int wt) {
   const int R = op.rows, K = op.cols, kind = op.kind;
   const bf16* src = (const bf16*)op.p[0];
-  const int* tok = (const int*)op.p[1];
   const bf16* gain = (const bf16*)op.p[2];
   float* xres = (float*)op.p[3];
   bf16* xbuf = (bf16*)op.p[4];
   bf16* hidden = (bf16*)op.p[5];
-  const int vocab = op.i[0], lo_rows = op.i[1];
+  const int lo_rows = op.i[1];
   const float eps = op.f[0];
   const float* part = nullptr;
   int splits = 0;
@@ -41,12 +39,7 @@ __device__ __noinline__ void pm_norm_rows(PmSmem& S, const PmOp& op, int wt) {
       bf16x8_to_float(*reinterpret_cast<const uint4*>(src + srow * K + c * 8), v);
     }
   };
-  auto src_row = [&](int r) -> size_t {
-    if (kind != PH_EMBED_NORM) return (size_t)r;
-    int t = __ldcg(tok + r);
-    t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
-    return (size_t)t;
-  };
+  auto src_row = [&](int r) -> size_t { return (size_t)r; };
   auto finish_chunk = [&](int r, int c, const float* v, float rinv) {
     if (xres && (kind != PH_RESNORM || part)) {
       *reinterpret_cast<float4*>(xres + (size_t)r * K + c * 8) = make_float4(v[0], v[1], v[2], v[3]);
@@ -129,92 +122,6 @@ __device__ __noinline__ void pm_norm_rows(PmSmem& S, const PmOp& op, int wt) {
   }
 }
 
-// h = silu(gate) * up from the split planes of a [gate | up] GEMM -> X buffer [rows, F].  p[0] xbuf; i[1] lo_rows.
-__device__ __noinline__ void pm_silu(PmSmem& S, const PmOp& op, int wt) {
-  const PmGemm& G = S.g[op.gemm];
-  const float* out = G.out;
-  const int splits = G.splits;
-  const size_t plane = G.plane;
-  const int R = op.rows, F = op.cols, nch = F >> 3, lo_rows = op.i[1];
-  bf16* xbuf = (bf16*)op.p[0];
-  const long long total = (long long)R * nch;
-  for (long long i = (long long)blockIdx.x * PM_WORKERS + wt; i < total; i += (long long)gridDim.x * PM_WORKERS) {
-    const int r = (int)(i / nch), c = (int)(i - (long long)r * nch);
-    float g8[8], u8[8], h[8];
-    load8_planes(out + (size_t)r * 2 * F + c * 8, splits, plane, g8);
-    load8_planes(out + (size_t)r * 2 * F + F + c * 8, splits, plane, u8);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) h[k] = g8[k] / (1.f + __expf(-g8[k])) * u8[k];
-    xbuf_store8(xbuf, (size_t)F, r, c * 8, lo_rows, h);
-  }
-}
-
-// y = bf16(sum of planes), [rows, cols] dense.  p[0] dst (bf16)
-__device__ __noinline__ void pm_sumcast(PmSmem& S, const PmOp& op, int wt) {
-  const PmGemm& G = S.g[op.gemm];
-  const float* out = G.out;
-  const int splits = G.splits;
-  const size_t plane = G.plane;
-  const int R = op.rows, W = op.cols, nch = W >> 3;
-  bf16* dst = (bf16*)op.p[0];
-  const long long total = (long long)R * nch;
-  for (long long i = (long long)blockIdx.x * PM_WORKERS + wt; i < total; i += (long long)gridDim.x * PM_WORKERS) {
-    const int r = (int)(i / nch), c = (int)(i - (long long)r * nch);
-    float v[8];
-    load8_planes(out + (size_t)r * W + c * 8, splits, plane, v);
-    xbuf_store8(dst, (size_t)W, r, c * 8, 0, v);
-  }
-}
-
-// Rotary embedding of the draft rows: q -> fp32 [R, hq*dh]; k (rotated), v -> tree slots (bf16). One warp per
-// (row, head). p[0] q32, p[1] tree k, p[2] tree v, p[3] pos_base (sa_len); i[0] hq, i[1] hkv, i[2] dh, i[3] step,
-// i[4] B, i[5] slots per sequence; f[0] theta. Planes row layout [q | k | v]. Angles are formed in double.
-__device__ __noinline__ void pm_rope(PmSmem& S, const PmOp& op, int wt) {
-  const PmGemm& G = S.g[op.gemm];
-  const float* out = G.out;
-  const int splits = G.splits;
-  const size_t plane = G.plane;
-  const int R = op.rows, hq = op.i[0], hkv = op.i[1], dh = op.i[2], step = op.i[3], B = op.i[4], slots = op.i[5];
-  const float theta = op.f[0];
-  float* q32 = (float*)op.p[0];
-  bf16* tk = (bf16*)op.p[1];
-  bf16* tv = (bf16*)op.p[2];
-  const int* pos_base = (const int*)op.p[3];
-  const int heads = hq + 2 * hkv, half = dh >> 1, ld = heads * dh;
-  const int lane = wt & 31;
-  const int gw = (int)blockIdx.x * PM_WWARPS + (wt >> 5), nw = (int)gridDim.x * PM_WWARPS;
-  for (int unit = gw; unit < R * heads; unit += nw) {
-    const int r = unit / heads, h = unit - r * heads;
-    const int seq = step == 0 ? r : r / B;
-    const int slot = step == 0 ? 0 : 1 + (step - 1) * B + (r % B);
-    const size_t dst = ((size_t)seq * slots + slot) * hkv * dh;
-    const float* row = out + (size_t)r * ld + h * dh;
-    if (h >= hq + hkv) {                                   // value head: copy
-      const int hv = h - hq - hkv;
-      for (int j = lane; j < dh; j += 32) tv[dst + hv * dh + j] = __float2bfloat16_rn(load1_planes(row + j, splits, plane));
-      continue;
-    }
-    const int pos = __ldcg(pos_base + seq) + step;
-    for (int j = lane; j < half; j += 32) {
-      const float x1 = load1_planes(row + j, splits, plane), x2 = load1_planes(row + half + j, splits, plane);
-      float cs = 1.f, sn = 0.f;
-      if (theta != 0.f) {
-        const double inv = exp2(-2.0 * (double)j / (double)dh * log2((double)theta));
-        double s, c;
-        sincos((double)pos * inv, &s, &c);
-        cs = (float)c; sn = (float)s;
-      }
-      const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
-      if (h < hq) {
-        q32[(size_t)r * hq * dh + h * dh + j] = y1;
-        q32[(size_t)r * hq * dh + h * dh + half + j] = y2;
-      } else {
-        tk[dst + (h - hq) * dh + j] = __float2bfloat16_rn(y1);
-        tk[dst + (h - hq) * dh + half + j] = __float2bfloat16_rn(y2);
-      }
-    }
-  }
-}
 
 // LSA tail: xres (+ planes of the down projection) -> mean over the S layer rows of a token -> kvf (fp32),
 // kv_out (bf16, optional), kvn = RMSNorm(mean; gain) into an X buffer. One CTA per token.

@@ -19,7 +19,7 @@ STATUS_NAMES = ["OK", "ERR_NULL", "ERR_SHAPE", "ERR_DTYPE", "ERR_ALIGN", "ERR_WO
                 "ERR_STATE", "ERR_ARCH", "ERR_CUDA", "ERR_TIMEOUT"]
 MOA_OK = 0
 
-EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_set_option", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
+EXPORTS = ["moa_create", "moa_destroy", "moa_tli_configure", "moa_state_bytes", "moa_status_str", "moa_last_cuda_error",
            "moa_state_set_len", "moa_lsa_forward", "moa_sa_append", "moa_sa_append_static", "moa_drafter_prefill", "moa_tree_begin", "moa_draft_step",
            "moa_tree_expand", "moa_tree_attn_mask", "moa_verify_greedy", "moa_pack_tree", "moa_unpack_tree", "moa_quantize_rows", "moa_dequantize_rows", "moa_state_status", "moa_profile_begin", "moa_profile_end", "moa_profile_phases",
            "moa_launch_count", "moa_trace_begin", "moa_trace_end"]
@@ -87,9 +87,10 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     if _lib is not None:
         return _lib
     trace = os.environ.get("MOA_TRACE_BUILD", "") == "1"          # the variant whose kernels stamp the stage trace
-    path = _build.LIB_TRACE if trace else _build.LIB
+    checks = os.environ.get("MOA_CHECKS_BUILD", "") == "1"        # the debug variant with device-side index checks
+    path = _build.LIB_TRACE if trace else _build.LIB_CHECKS if checks else _build.LIB
     if rebuild_if_stale and (os.path.exists("/usr/local/cuda/bin/nvcc") or os.environ.get("NVCC")):
-        path = _build.build(trace=trace)
+        path = _build.build(trace=trace, checks=checks)
     if not os.path.exists(path):
         raise RuntimeError(f"{path} not found: build it with `python -m paper_2410_03804_b200.build`")
     lib = C.CDLL(path)
@@ -97,7 +98,6 @@ def load_library(rebuild_if_stale: bool = True) -> C.CDLL:
     lib.moa_create.argtypes = [C.POINTER(MoaConfig), C.POINTER(MoaWeights), C.POINTER(vp)]
     lib.moa_destroy.argtypes = [vp]
     lib.moa_destroy.restype = None
-    lib.moa_set_option.argtypes = [vp, i32, i32]
     lib.moa_state_bytes.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
     lib.moa_status_str.argtypes = [i32]
     lib.moa_status_str.restype = C.c_char_p
@@ -239,8 +239,7 @@ class MoA:
     cfg['n_tli'] = N > 0 (plus 'tli_hq', 'tli_hkv', 'tli_mlp') the weights also hold 'tli{l}_{norm1,wq,...}' for
     l < N, and the LLM's caches of those layers are the tensors tli_k[l], tli_v[l] (fill_tli_cache)."""
 
-    def __init__(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int, lsa_chunk_tokens: int = 8,
-                 fused_step: bool = False):
+    def __init__(self, cfg: dict, weights: dict, max_batch: int, max_ctx: int, lsa_chunk_tokens: int = 8):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2410_03804_b200 needs a CUDA device (B200, sm_100a); there is no CPU path")
@@ -265,8 +264,6 @@ class MoA:
         h = C.c_void_p()
         _check(self.lib.moa_create(C.byref(c), C.byref(w), C.byref(h)), "moa_create")
         self.h = h
-        if fused_step:
-            _check(self.lib.moa_set_option(self.h, 1, 1), "moa_set_option")
         self.device = weights["embed"].device
         self.n_tli = int(cfg.get("n_tli", 0))
         self.tli_k, self.tli_v = [], []
@@ -423,11 +420,10 @@ class MoA:
         _check(self.lib.moa_profile_end(self.h, C.byref(ms), C.byref(n)), "moa_profile_end")
         return ms.value, n.value
 
-    PHASE_KINDS = ["gemm", "embed_norm", "rows_norm", "res_norm", "rope", "attention", "attn_merge", "swiglu",
-                   "sum_cast", "mean_norm", "cache_append", "lm_merge", "lsa_attention"]
+    PHASE_KINDS = ["gemm", "rows_norm", "res_norm", "mean_norm", "cache_append", "lsa_attention"]
 
     def moa_profile_phases(self, stream=None):
-        """[(kind name, microseconds, of which in the closing barrier)] of the last fused launch made while
+        """[(kind name, microseconds, of which in the closing barrier)] of the last dense LSA pass launched while
         profiling was on."""
         cap = 32
         us, wait, kinds, n = (C.c_double * cap)(), (C.c_double * cap)(), (C.c_int32 * cap)(), C.c_int32()

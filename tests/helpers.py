@@ -48,11 +48,10 @@ def make_oracles(p: synth.Preset, weights_cpu: dict, cache_f64=True):
     return exact, dec
 
 
-def make_gpu(p: synth.Preset, weights_cpu: dict, max_ctx: int, lsa_chunk_tokens: int = 8, max_batch=None,
-             fused_step: bool = False):
+def make_gpu(p: synth.Preset, weights_cpu: dict, max_ctx: int, lsa_chunk_tokens: int = 8, max_batch=None):
     from paper_2410_03804_b200 import moa
     w = {k: v.cuda() for k, v in weights_cpu.items()}
-    return moa.MoA(cfg_of(p), w, max_batch or p.batch, max_ctx, lsa_chunk_tokens, fused_step=fused_step)
+    return moa.MoA(cfg_of(p), w, max_batch or p.batch, max_ctx, lsa_chunk_tokens)
 
 
 def assert_rows_close(got, want, tol, what=""):
