@@ -47,9 +47,17 @@ def algorithmic_bytes(p) -> dict:
     return dict(step=(sa_w + ca_w + lm + caches + tli) * e, lm_head=lm * e, lsa=(lsa_w + lsa_in) * e)
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch (wstream_gemm_kernel<32>, mode 1) from the ncu
-# capture summarised in profiles/lm_head_wstream_c2.md; set back to None when that kernel changes.
-LM_HEAD_TRAFFIC = {"c2": 1051208704 + 3780352}
+def lm_head_traffic(name: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one LM-head launch from the tracked ncu summary
+    profiles/lm_head_traffic.json (which names the commit the counters were taken on), or None when there is no
+    entry for this workload."""
+    path = os.path.join(ROOT, "profiles", "lm_head_traffic.json")
+    try:
+        with open(path) as f:
+            e = json.load(f).get(name)
+        return None if e is None else int(e["dram_bytes_read"]) + int(e["dram_bytes_write"])
+    except (OSError, ValueError, KeyError):
+        return None
 
 
 class ClockSampler:
@@ -135,9 +143,12 @@ class OracleSampler:
         self.tli = [tuple(t[0].float().numpy().astype(np.float64) for t in synth.make_tli_cache(one, l, self.ctx))
                     for l in range(p.n_tli)]
 
-    def sample(self, rows: int = 2, lsa_tok: int = 1):
-        """Returns (cycle_seconds_estimate, cores, description)."""
+    def sample(self, rows: int = None, lsa_tok: int = None):
+        """Times the cycle's whole LSA token set of one sequence and the forwards of its first two tree levels (1 + B
+        rows) unless told otherwise, and scales to a cycle. Returns (cycle_seconds_estimate, cores, description)."""
         p, synth = self.p, self.synth
+        rows = 1 + p.tree_topk if rows is None else rows
+        lsa_tok = p.lsa_tokens if lsa_tok is None else lsa_tok
         caK, caV, saK, saV = self.caches
         h = synth.make_h_stack(p, lsa_tok).float().numpy()
         t0 = time.perf_counter()
@@ -150,13 +161,13 @@ class OracleSampler:
         t_row = (time.perf_counter() - t0) / rows
         n_rows = p.batch * (1 + p.tree_topk * (p.tree_depth - 1))
         cycle = p.batch * p.lsa_tokens * t_lsa + n_rows * t_row
-        what = (f"{lsa_tok} LSA token(s) ({t_lsa:.2f} s each) + {rows} drafter forward rows ({t_row:.2f} s each) of {p.name}"
-                f" with {self.ctx}-entry caches, scaled to one cycle = {p.batch * p.lsa_tokens} LSA tokens + {n_rows} rows;"
+        what = (f"timed: {lsa_tok} LSA token(s) ({t_lsa:.2f} s each) + {rows} drafter forward rows ({t_row:.2f} s each) of {p.name}"
+                f" with {self.ctx}-entry caches; extrapolated to one cycle = {p.batch * p.lsa_tokens} LSA tokens + {n_rows} rows;"
                 f" weights widened to fp64 beforehand")
         return cycle, self.cores, what
 
 
-def oracle_sample(p, rows: int = 2, lsa_tok: int = 1):
+def oracle_sample(p, rows: int = None, lsa_tok: int = None):
     return OracleSampler(p).sample(rows, lsa_tok)
 
 
@@ -164,7 +175,7 @@ def run_reference(args, p):
     sampler = OracleSampler(p)                       # set-up is not timed
     t_all = []
     for _ in range(args.warmup + args.steps):
-        cycle, cores, what = sampler.sample(rows=1, lsa_tok=1)     # one bounded sample per step
+        cycle, cores, what = sampler.sample()     # one bounded sample per step: the LSA token set + two tree levels
         t_all.append(cycle)
     t = statistics.mean(t_all[args.warmup:]) if len(t_all) > args.warmup else t_all[-1]
     D, m = p.tree_depth, p.tree_keep
@@ -173,7 +184,8 @@ def run_reference(args, p):
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": workload_config(p),
-            "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what},
+            "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what,
+                             "extrapolated": True},
             "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "drafted_tokens_per_sec": p.batch * m / t}
     print(json.dumps(line))
@@ -490,6 +502,16 @@ def main():
     sampler.start()
     ms = timed(run_dev, args.steps)
     ms_e2e = timed(run_e2e, args.steps)
+    # the same block replayed ten more times with an event pair around every cycle: spread of the per-cycle time
+    n_dist = max(10 * args.steps, 200)
+    dist_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_dist)]
+    torch.cuda.synchronize()
+    for a, b in dist_ev:
+        a.record()
+        run_dev()
+        b.record()
+    torch.cuda.synchronize()
+    cyc = sorted(a.elapsed_time(b) for a, b in dist_ev)
     # the dominant kernel (LM head), bracketed by CUDA events on the launching stream: same cycles, launched on
     # the stream (events cannot be read inside a graph), directly after the timed replays
     g.moa_profile_begin()
@@ -553,10 +575,12 @@ def main():
         "gpu_launches": launches,
         "launch_mode": "cuda graph replay of one recorded cycle" if use_graph else "stream launches",
         "ms_per_step_stream_launches": ms_stream / args.steps,
+        "cycle_ms_distribution": {"n": n_dist, "median": cyc[n_dist // 2], "p10": cyc[n_dist // 10], "p90": cyc[(9 * n_dist) // 10],
+                                  "what": "every cycle between its own event pair, same launch mode, right after the timed block"},
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "lm_head", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}",
-                     "traffic": LM_HEAD_TRAFFIC.get(p.name),
+                     "traffic": lm_head_traffic(p.name),
                      "launches_timed": lm_n, "avg_launch_us": lm_avg_s * 1e6,
                      "timed_over": "the same cycles launched on the stream right after the timed replays",
                      "algorithmic_bytes_per_launch": ab["lm_head"]},
@@ -581,7 +605,8 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cyc, cores, what = oracle_sample(p)
-        line["cpu_baseline"] = {"value": D / cyc, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what}
+        line["cpu_baseline"] = {"value": D / cyc, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": what,
+                                "extrapolated": True}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
