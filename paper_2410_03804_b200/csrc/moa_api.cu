@@ -10,6 +10,7 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include "moa_attn.cuh"
+#include "moa_attn_tc.cuh"
 #include "moa_basic.cuh"
 #include "moa_codec.cuh"
 #include "moa_phases.cuh"
@@ -30,7 +31,7 @@ struct NvtxRange {
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256 };
+enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256, TC_MIN_KEYS = 4096 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -393,6 +394,66 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     const int nwarps = imin(8, (Qn + 15) / 16);
     P.q_tiles = (Qn + nwarps * 16 - 1) / (nwarps * 16);
     const int has_tree = (kB != nullptr && nB > 0) ? 1 : 0;
+    P.part_o = (float*)(ws + p.att_o);
+    P.part_ml = (float*)(ws + p.att_ml);
+    P.out = (bf16*)out;
+    P.out_lo = lo_rows_of(sizeof(T), R);
+    P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    // Long dense caches (fp32 queries, head size 128, no per-row limits): the cache segment on the tcgen05 kernel, one CTA
+    // per SM; the tree segment, if any, as one more part from the split-KV kernel; merged together.
+    if (q32 && dh == 128 && !lim.active() && ctx->fast && Qn <= 128 && posA_ld == hkv * dh && kA != nullptr &&
+        max_len >= TC_MIN_KEYS) {
+      const int blocks = (max_len + TC_KB - 1) / TC_KB;
+      int n_split = imax(1, imin(blocks, ctx->sm_count / imax(1, nseq * hkv)));
+      const long long per_part = (long long)R * hq;
+      while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
+      if (n_split + has_tree > 1 && per_part * (n_split + has_tree) > p.att_units) return MOA_ERR_WORKSPACE;
+      AttnTcParams TP;
+      memset(&TP, 0, sizeof(TP));
+      P.n_split = n_split;
+      P.n_parts = n_split + has_tree;
+      TP.a = P;
+      const int cache_rows = ctx->c.max_batch * capA;
+      if (!encode_map(ctx, &TP.tmK, kA, cache_rows, hkv * dh, TC_KB) || !encode_map(ctx, &TP.tmV, vA, cache_rows, hkv * dh, TC_KB))
+        return MOA_ERR_CUDA;
+      static bool tc_attr = false;
+      if (!tc_attr) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+        if (e != cudaSuccess) {
+          snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+          return MOA_ERR_CUDA;
+        }
+        tc_attr = true;
+      }
+      launch_pdl(attn_tc_kernel, dim3(n_split, hkv, nseq), dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
+      MOA_CHECK_LAUNCH();
+      if (has_tree) {                         // the tree segment alone: its single part is stored behind the cache parts
+        AttnParams T2 = P;
+        T2.n_split = 0;
+        T2.part_base = n_split;
+        static bool t_attr = false;
+        const int smem = 2 * nwarps * 16 * 128 * 2 + 4 * AT_KB * 128 * 2;
+        if (!t_attr) {
+          cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               2 * 8 * 16 * 128 * 2 + 4 * AT_KB * 128 * 2);
+          if (e != cudaSuccess) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+            return MOA_ERR_CUDA;
+          }
+          t_attr = true;
+        }
+        launch_pdl(attn_split_kernel<128, true, true>, dim3(1, hkv * P.q_tiles, nseq), dim3(nwarps * 32), smem, s, T2);
+        MOA_CHECK_LAUNCH();
+      }
+      if (P.n_parts > 1) {
+        const int n_rh = nseq * rows_per_seq * hq;
+        const int share = P.n_parts >= CB_SHARE_FROM ? 1 : 0;
+        launch_pdl(attn_combine_kernel<128>, dim3(share ? n_rh : (n_rh + CB_WARPS - 1) / CB_WARPS), dim3(CB_WARPS * 32), 0, s, P.part_o,
+                   P.part_ml, P.n_parts, n_rh, share, P.out, P.out_lo, P.hq);
+        MOA_CHECK_LAUNCH();
+      }
+      return MOA_OK;
+    }
     const int blocks = imax(1, (max_len + AT_KB - 1) / AT_KB);
     // cache parts plus the tree part fill one wave of two CTAs per SM: a few CTAs more would run alone afterwards
     int n_split = imax(1, imin(blocks, (2 * ctx->sm_count) / imax(1, nseq * hkv * P.q_tiles) - has_tree));
@@ -401,11 +462,6 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     if (per_part * (n_split + has_tree) > p.att_units && n_split + has_tree > 1) return MOA_ERR_WORKSPACE;
     P.n_split = n_split;
     P.n_parts = n_split + has_tree;
-    P.part_o = (float*)(ws + p.att_o);
-    P.part_ml = (float*)(ws + p.att_ml);
-    P.out = (bf16*)out;
-    P.out_lo = lo_rows_of(sizeof(T), R);
-    P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
     // fp32 queries and the probabilities are split into two bf16 terms each
     if (q32)
       return dh == 128 ? launch_attn_split<128, true, true>(s, P, nseq, nwarps) : launch_attn_split<64, true, true>(s, P, nseq, nwarps);

@@ -424,3 +424,50 @@ def test_lsa_tokens_are_independent_and_incremental_equals_full(dtype):
         got = run(parts, chunk)
         for a, b, what in zip(got, full, ("kv", "CA K rows", "CA V rows")):
             H.assert_rows_close(a, b, tol, f"{what}: parts {parts[:3]}.. chunk {chunk} vs one call")
+
+
+def test_long_caches_take_the_tensor_core_attention_with_ragged_lengths():
+    """Caches of more than 4096 positions run their cache segment on the tcgen05 attention kernel (keys streamed by
+    TMA, scores and the output accumulator in TMEM); the tree segment stays on the split-KV kernel and the parts are
+    merged. Two sequences with different lengths, one of them with an empty self-attention prefix (key ranges of
+    zero blocks), lengths that are not multiples of the 64-position block."""
+    p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=1031, lsa_hq=2, lsa_hkv=2,
+                     lsa_mlp=128, sa_hq=4, sa_hkv=1, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=448, ctx=5000, batch=2,
+                     tree_topk=4, tree_depth=3, tree_keep=9, head_dim=128)
+    w = synth.make_weights(p)
+    g = H.make_gpu(p, w, max_ctx=5056)
+    exact, dec = H.make_oracles(p, w)
+    caK, caV = synth.make_cache(p, "ca")
+    saK, saV = synth.make_cache(p, "sa")
+    g.fill_cache("ca", caK.cuda(), caV.cuda())
+    g.fill_cache("sa", saK.cuda(), saV.cuda())
+    lens_ca, lens_sa = [5000, 4101], [4990, 0]
+    g.moa_state_set_len("ca", lens_ca)
+    g.moa_state_set_len("sa", lens_sa)
+    root = synth.make_root(p)
+    g.moa_tree_begin(root.cuda())
+    B, D = p.tree_topk, p.tree_depth
+
+    def trees_of(dr, forced):
+        return [O.draft_tree(dr, int(root[b]), H.np32(saK[b, :lens_sa[b]]), H.np32(saV[b, :lens_sa[b]]),
+                             H.np32(caK[b, :lens_ca[b]]), H.np32(caV[b, :lens_ca[b]]), B, D, p.tree_keep,
+                             forced=None if forced is None else forced[b]) for b in range(2)]
+    td = trees_of(dec, None)
+    forced = [[([r["ids"] for r in rows], [r["logp"] for r in rows]) for rows in td[b][1]] for b in range(2)]
+    tx = trees_of(exact, forced)
+    tol = H.tol_of(p)
+    worst = 0.0
+    for s in range(D):
+        ids, lp, hid = g.moa_draft_step(want_hidden=True)
+        ids, lp, hid = ids.cpu().numpy(), lp.cpu().numpy(), H.np32(hid.cpu())
+        rs = 1 if s == 0 else B
+        f_ids, f_lp = np.zeros((2 * rs, B), np.int32), np.zeros((2 * rs, B), np.float32)
+        for b in range(2):
+            for r in range(rs):
+                worst = max(worst, H.assert_rows_close(hid[b * rs + r][None], tx[b][1][s][r]["o_hat"][None], tol, f"hidden s{s} b{b} r{r}"))
+                H.check_topk(ids[b * rs + r], lp[b * rs + r], td[b][1][s][r]["z"], tol, H.tie_window(p, td[b][1][s][r]["z"]))
+                f_ids[b * rs + r], f_lp[b * rs + r] = td[b][1][s][r]["ids"], td[b][1][s][r]["logp"]
+        g.moa_tree_expand(torch.from_numpy(f_ids).cuda(), torch.from_numpy(f_lp).cuda())
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 0
+    print(f"[long caches, tensor-core attention] worst hidden {worst:.2e}")
