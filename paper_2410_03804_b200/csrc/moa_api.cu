@@ -402,12 +402,13 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     // Long dense caches (fp32 queries, head size 128, no per-row limits): the cache segment on the tcgen05 kernel, one CTA
     // per SM; the tree segment, if any, as one more part from the split-KV kernel; merged together.
     if (q32 && dh == 128 && !lim.active() && ctx->fast && Qn <= 128 && posA_ld == hkv * dh && kA != nullptr &&
-        max_len >= TC_MIN_KEYS) {
+        max_len >= TC_MIN_KEYS && n_slots <= 256) {
       const int blocks = (max_len + TC_KB - 1) / TC_KB;
+      const int reps = Qn <= 64 ? 2 : 1;              // few queries: two copies of each share a block's positions
       int n_split = imax(1, imin(blocks, ctx->sm_count / imax(1, nseq * hkv)));
       const long long per_part = (long long)R * hq;
       while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
-      if (n_split + has_tree > 1 && per_part * (n_split + has_tree) > p.att_units) return MOA_ERR_WORKSPACE;
+      if (per_part * (n_split + has_tree) > p.att_units) return MOA_ERR_WORKSPACE;
       AttnTcParams TP;
       memset(&TP, 0, sizeof(TP));
       P.n_split = n_split;
@@ -416,35 +417,23 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
       const int cache_rows = ctx->c.max_batch * capA;
       if (!encode_map(ctx, &TP.tmK, kA, cache_rows, hkv * dh, TC_KB) || !encode_map(ctx, &TP.tmV, vA, cache_rows, hkv * dh, TC_KB))
         return MOA_ERR_CUDA;
+      if (has_tree && (!encode_map(ctx, &TP.tmKB, kB, ctx->c.max_batch * capB, hkv * dh, TC_KB) ||
+                       !encode_map(ctx, &TP.tmVB, vB, ctx->c.max_batch * capB, hkv * dh, TC_KB)))
+        return MOA_ERR_CUDA;
       static bool tc_attr = false;
       if (!tc_attr) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
         if (e != cudaSuccess) {
           snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
           return MOA_ERR_CUDA;
         }
         tc_attr = true;
       }
-      launch_pdl(attn_tc_kernel, dim3(n_split, hkv, nseq), dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
+      const dim3 tgrid(hkv, nseq, n_split + has_tree);
+      if (reps == 2) launch_pdl(attn_tc_kernel<2>, tgrid, dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
+      else launch_pdl(attn_tc_kernel<1>, tgrid, dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
       MOA_CHECK_LAUNCH();
-      if (has_tree) {                         // the tree segment alone: its single part is stored behind the cache parts
-        AttnParams T2 = P;
-        T2.n_split = 0;
-        T2.part_base = n_split;
-        static bool t_attr = false;
-        const int smem = 2 * nwarps * 16 * 128 * 2 + 4 * AT_KB * 128 * 2;
-        if (!t_attr) {
-          cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               2 * 8 * 16 * 128 * 2 + 4 * AT_KB * 128 * 2);
-          if (e != cudaSuccess) {
-            snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-            return MOA_ERR_CUDA;
-          }
-          t_attr = true;
-        }
-        launch_pdl(attn_split_kernel<128, true, true>, dim3(1, hkv * P.q_tiles, nseq), dim3(nwarps * 32), smem, s, T2);
-        MOA_CHECK_LAUNCH();
-      }
       if (P.n_parts > 1) {
         const int n_rh = nseq * rows_per_seq * hq;
         const int share = P.n_parts >= CB_SHARE_FROM ? 1 : 0;

@@ -32,9 +32,7 @@ struct AttnParams {
   const bf16* kB; const bf16* vB; int capB;                // segment B: ((seq*capB + slot)*hkv + g)*DH
   const int* slotsB; int slots_ld; int nB; int n_slots;    // row's ancestor slots [nB]; slots in use
   int n_split;                           // splits of segment A
-  int n_parts;                           // parts per (row, head) in the part buffers: n_split + (segment B ? 1 : 0)
-  int part_base;                         // this launch's part p is stored as part part_base + p (non-zero when the cache
-                                         // segment's parts come from the tensor-core kernel and only segment B runs here)
+  int n_parts;                           // n_split + (segment B ? 1 : 0)
   int q_tiles;                           // query tiles per (seq, kv head)
   float* part_o; float* part_ml;         // [R*hq][n_parts][DH], [R*hq][n_parts][2]
   bf16* out;                             // [R, hq*DH]
@@ -379,7 +377,7 @@ __global__ void __launch_bounds__(256) attn_split_kernel(const AttnParams P) {
           *reinterpret_cast<uint32_t*>(dlo + i * 8 + tq * 2) = pack_bf16(a - __bfloat162float(ha), b - __bfloat162float(hb));
       }
     } else {
-      const size_t pidx = ((size_t)row * P.hq + head) * P.n_parts + P.part_base + part;
+      const size_t pidx = ((size_t)row * P.hq + head) * P.n_parts + part;
       float* dst = P.part_o + pidx * DH;
 #pragma unroll
       for (int i = 0; i < DH / 8; ++i)

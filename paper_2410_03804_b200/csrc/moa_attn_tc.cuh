@@ -9,14 +9,22 @@
 //   warp 1      one thread issues tcgen05.mma:  S = Q_hi K^T + Q_lo K^T   (A = Q, B = K, both K-major; fp32 in TMEM)
 //                                               O += P_hi V + P_lo V      (A = P from shared memory, K-major;
 //                                                                          B = V as it lies in the cache: MN-major)
-//   warps 2..5  softmax: thread t owns query row t (TMEM lane t): reads its 64 scores, keeps the running maximum
-//               and sum in the log2 domain, writes the probabilities as two bf16 terms into the swizzled P tiles.
+//   warps 2..9  softmax, two groups of four warps that take alternate blocks: a thread owns one query row (TMEM lane)
+//               of its group's blocks: reads its scores, keeps the running maximum and sum in the log2 domain, writes
+//               the probabilities as two bf16 terms into the swizzled P tiles. Each group has its own score buffer,
+//               P buffer and OUTPUT ACCUMULATOR in TMEM, so the groups are independent partial softmaxes (over the
+//               even and the odd blocks) that never wait for one another; they are merged once, at the end.
 // The output accumulator stays in TMEM for the whole key range; it is rescaled only when a row's maximum has grown
 // by more than 2^8 since the last rescale (probabilities then stay below 256, well inside fp32 / bf16 range), so
 // the rescale -- a TMEM load, multiply, store of the row -- happens a few times per range, not per block.
-// Each CTA leaves (max, sum, unnormalised output) per query for attn_combine_kernel, in the layout of the split-KV
-// kernel, so the tree part of a self-attention (masked per row, a few dozen slots) still runs there and the parts
-// are merged together. Queries arrive in fp32 and enter as two bf16 terms, as in the split-KV kernel.
+// A block's softmax is a chain of short dependent steps (TMEM load, maximum, exponentials, shared-memory stores,
+// fences), so one group per CTA would set the pace; two groups overlap their chains. Each CTA leaves (max, sum,
+// unnormalised output) per query for attn_combine_kernel, in the layout of the split-KV kernel. A self-attention's tree segment (the sequence's drafted slots, masked per row by
+// its ancestor list) is one more CTA of the same grid: same pipeline over the tree's keys / values, with the row's
+// slot bitmap applied to the scores. Queries arrive in fp32 and enter as two bf16 terms, as in the split-KV kernel.
+// With at most 64 queries per kv head (REPS = 2) every query occupies two rows of the tile, r and 64 + r, and each copy
+// takes half of a block's 64 positions (its probabilities for the other half are zero): the two copies are
+// independent partial softmaxes too (merged with the groups at the end), and twice as many lanes share the exponentials.
 // Every mbarrier wait is bounded; on expiry the CTA raises the abort flag, drains, frees TMEM and reports
 // DEV_ERR_TIMEOUT through the status word.
 #pragma once
@@ -28,17 +36,18 @@ namespace moa {
 constexpr int TC_KB = 64;                 // cache positions per block
 constexpr int TC_DH = 128;
 constexpr int TC_STAGES = 3;
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;            // TMA warp, MMA warp, two softmax groups of four warps
 constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // one query term: two 64-column chunks of [128 rows x 128 B]
 constexpr int TC_P_BYTES = 128 * TC_KB * 2;           // one probability term: [128 rows x 128 B]
 constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-column chunks of [64 rows x 128 B]
 constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + 2 * TC_P_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
+constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + 4 * TC_P_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
 constexpr float TC_RESCALE_LOG2 = 8.f;
 
 struct AttnTcParams {
   CUtensorMap tmK, tmV;      // cache [positions of all sequences, hkv * 128], box 64 columns x 64 positions, swizzle 128B
-  AttnParams a;              // queries (fp32), lengths, part buffers; n_parts counts the tree part too
+  CUtensorMap tmKB, tmVB;    // tree slots [slots of all sequences, hkv * 128], same box (used when a.n_parts > a.n_split)
+  AttnParams a;              // queries (fp32), lengths, part buffers; part a.n_split, if any, is the tree segment
 };
 
 // Shared-memory descriptor of an MN-major bf16 operand with the 128-byte swizzle: 64 elements along MN are contiguous
@@ -65,56 +74,71 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
       : "memory");
 }
 
+template <int REPS>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams P) {
+  constexpr int RPR = 128 / REPS;            // tile rows per copy of the queries
+  constexpr int NC = TC_KB / REPS;           // positions of a block one copy scores
   extern __shared__ uint8_t tc_smem_raw[];
   const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = tc_smem_raw + (base - smem_u32(tc_smem_raw));
-  constexpr uint32_t oQhi = 0, oQlo = TC_Q_BYTES, oPhi = 2 * TC_Q_BYTES, oPlo = oPhi + TC_P_BYTES, oKV = oPlo + TC_P_BYTES,
+  // P buffer j: hi term at oP + j * 2 * TC_P_BYTES, lo term TC_P_BYTES behind it
+  constexpr uint32_t oQhi = 0, oQlo = TC_Q_BYTES, oP = 2 * TC_Q_BYTES, oKV = oP + 4 * TC_P_BYTES,
                      oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
   const uint32_t bar0 = base + oBar;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
   auto sfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + i); };
   auto sempty_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + 2 + i); };
-  const uint32_t pfull_bar = bar0 + 8u * (2 * TC_STAGES + 4), pempty_bar = pfull_bar + 8u, qfull_bar = pfull_bar + 16u,
-                 ofull_bar = pfull_bar + 24u;
-  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (2 * TC_STAGES + 8));
+  auto pfull_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 4 + j); };
+  auto pempty_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 6 + j); };
+  const uint32_t qfull_bar = bar0 + 8u * (2 * TC_STAGES + 8), ofull_bar = qfull_bar + 8u;
+  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (2 * TC_STAGES + 10));
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const AttnParams& A = P.a;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int part = blockIdx.x, g = blockIdx.y, seq = blockIdx.z;
-  const int Qn = A.rows_per_seq * A.group;           // <= 128, checked by the host
+  const int g = blockIdx.x, seq = blockIdx.y, part = blockIdx.z;      // parts along z: the tree part's CTAs are launched last
+  const int Qn = A.rows_per_seq * A.group;           // <= 128 / REPS, checked by the host
   pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(sfull_bar(i), 1); mbar_init(sempty_bar(i), 128); }
-    mbar_init(pfull_bar, 128);
-    mbar_init(pempty_bar, 1);
-    mbar_init(qfull_bar, 128);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(sfull_bar(i), 1); mbar_init(sempty_bar(i), 128);
+      mbar_init(pfull_bar(i), 128); mbar_init(pempty_bar(i), 1);
+    }
+    mbar_init(qfull_bar, 256);
     mbar_init(ofull_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + 128u;          // S buffers at columns 0 and 64, O at 128..255
+  const uint32_t tS = tmem_base, tO = tmem_base + 128u;          // S buffers at columns 0 and 64, the groups' O at 128 and 256
 
   // the cache was written by earlier kernels of the stream, and so were the queries
   pdl_wait(KID_ATTN);
-  const int len = A.lenA ? A.lenA[seq] : A.nA_fixed;
-  const int blocks = (len + TC_KB - 1) / TC_KB;
-  const int b0 = (int)(((long long)part * blocks) / A.n_split), b1 = (int)(((long long)(part + 1) * blocks) / A.n_split);
-  const int k_begin = b0 * TC_KB, k_end = min(b1 * TC_KB, len);
-  const int n_blocks = b1 - b0;
+  const bool tree_part = part >= A.n_split;          // the grid's last CTA along x when the attention has a tree segment
+  int k_begin, k_end, n_blocks;
+  if (!tree_part) {
+    const int len = A.lenA ? A.lenA[seq] : A.nA_fixed;
+    const int blocks = (len + TC_KB - 1) / TC_KB;
+    const int b0 = (int)(((long long)part * blocks) / A.n_split), b1 = (int)(((long long)(part + 1) * blocks) / A.n_split);
+    k_begin = b0 * TC_KB;
+    k_end = min(b1 * TC_KB, len);
+    n_blocks = b1 - b0;
+  } else {
+    k_begin = 0;
+    k_end = min(A.n_slots, 256);                     // slot bitmaps hold 256 slots (the host checks)
+    n_blocks = (k_end + TC_KB - 1) / TC_KB;
+  }
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -126,11 +150,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(empty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
         mbar_expect_tx(full_bar(st), TC_STAGE_BYTES);
         const uint32_t dst = base + oKV + st * TC_STAGE_BYTES;
-        const int y = seq * A.capA + k_begin + b * TC_KB;
-        tma_load_2d(dst, &P.tmK, x0, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES / 2, &P.tmK, x0 + 64, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES, &P.tmV, x0, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES + TC_KV_BYTES / 2, &P.tmV, x0 + 64, y, full_bar(st));
+        const int y = seq * (tree_part ? A.capB : A.capA) + k_begin + b * TC_KB;
+        const CUtensorMap* tk = tree_part ? &P.tmKB : &P.tmK;
+        const CUtensorMap* tv = tree_part ? &P.tmVB : &P.tmV;
+        tma_load_2d(dst, tk, x0, y, full_bar(st));
+        tma_load_2d(dst + TC_KV_BYTES / 2, tk, x0 + 64, y, full_bar(st));
+        tma_load_2d(dst + TC_KV_BYTES, tv, x0, y, full_bar(st));
+        tma_load_2d(dst + TC_KV_BYTES + TC_KV_BYTES / 2, tv, x0 + 64, y, full_bar(st));
       }
     }
   } else if (warp == 1) {
@@ -163,46 +189,54 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       if (ok) ok = issue_s(0);
       for (int b = 0; b < n_blocks && ok; ++b) {
         if (b + 1 < n_blocks && !issue_s(b + 1)) { ok = false; break; }
-        if (!mbar_wait(pfull_bar, (uint32_t)b & 1u, abort_flag)) { ok = false; break; }
+        const int j = b & 1;
+        if (!mbar_wait(pfull_bar(j), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t paddr = base + oP + (uint32_t)j * 2u * TC_P_BYTES;
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16(tO, umma_desc_sw128(base + oPhi) + 2u * ks, umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O,
-                      (b > 0 || ks > 0) ? 1u : 0u);
+          tc_mma_bf16(tO + (uint32_t)(j * TC_DH), umma_desc_sw128(paddr) + 2u * ks, umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2),
+                      IDESC_O, (b > 1 || ks > 0) ? 1u : 0u);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16(tO, umma_desc_sw128(base + oPlo) + 2u * ks, umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
-        tc_commit(pempty_bar);                    // P may be overwritten, O may be rescaled
+          tc_mma_bf16(tO + (uint32_t)(j * TC_DH), umma_desc_sw128(paddr + TC_P_BYTES) + 2u * ks,
+                      umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
+        tc_commit(pempty_bar(j));                 // the group's P buffer may be overwritten and its O is at rest once this completes
         tc_commit(empty_bar(b % TC_STAGES));      // the stage's K and V are done with
       }
       if (ok) tc_commit(ofull_bar);
     }
   } else {
-    // ------------------------------ softmax: one thread per query row ------------------------------
+    // ------------------------------ softmax: group gi takes the blocks b with b % 2 == gi ------------------------------
+    const int wi = warp - 2;                           // 0..7
+    const int gi = wi >> 2;                            // group: its S buffer, P buffer, O accumulator and barriers have index gi
     const int quad = warp & 3;                         // TMEM lane quadrant of this warp
-    const int ql = quad * 32 + lane;                   // query row = TMEM lane
-    const int st_i = threadIdx.x - 64;                 // 0..127 among these threads
-    const bool valid = ql < Qn;
-    const bool warp_live = quad * 32 < Qn;             // at least one real query in this warp
-    const int row = seq * A.rows_per_seq + (valid ? ql / A.group : 0);
-    const int head = g * A.group + (valid ? ql % A.group : 0);
+    const int ql = quad * 32 + lane;                   // tile row = TMEM lane
+    const int st_i = threadIdx.x - 64;                 // 0..255 among the softmax threads
+    const int qi = ql % RPR, rep = ql / RPR;           // query of this row, and which copy of it
+    const int c_lo = rep * NC;                         // this copy's positions inside a block: c_lo .. c_lo + NC - 1
+    const bool valid = qi < Qn;
+    const bool warp_live = (quad * 32) % RPR < Qn;     // at least one real query in this warp
+    const int row = seq * A.rows_per_seq + (valid ? qi / A.group : 0);
+    const int head = g * A.group + (valid ? qi % A.group : 0);
     // ---- queries -> two bf16 terms in shared memory (rows beyond Qn are zero) ----
-    for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 128) {
+    for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 256) {
       float x[4][8];
       bool in[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 128;
-        const int r = i >> 4, c = i & 15;
-        in[u] = r < Qn;
+        const int i = i0 + u * 256;
+        const int r = (i >> 4) % RPR, c = i & 15;
+        in[u] = i < 128 * 16 && r < Qn;
         if (in[u])
           load8_planes(A.q32 + (size_t)(seq * A.rows_per_seq + r / A.group) * A.q_ld + (g * A.group + r % A.group) * TC_DH + c * 8,
                        A.q_splits, A.q_plane, x[u]);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 128;
+        const int i = i0 + u * 256;
+        if (i >= 128 * 16) continue;
         const int r = i >> 4, c = i & 15;
         uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
         if (in[u]) {
@@ -218,57 +252,79 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         *reinterpret_cast<uint4*>(bp + oQlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
     }
+    uint8_t* const phi = bp + oP + (uint32_t)gi * 2u * TC_P_BYTES;      // the group's P tile (hi term; lo TC_P_BYTES behind)
+    if (REPS > 1) {            // a copy's probabilities outside its own positions are zero, once and for all
+#pragma unroll
+      for (int c = 0; c < TC_KB; c += 8)
+        if (c < c_lo || c >= c_lo + NC) {
+          *reinterpret_cast<uint4*>(phi + sw128_off(ql, c)) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(phi + TC_P_BYTES + sw128_off(ql, c)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     mbar_arrive(qfull_bar);
 
+    // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per key block
+    unsigned long long allow[4] = {0ull, 0ull, 0ull, 0ull};
+    if (tree_part && valid) {
+      for (int i = 0; i < A.nB; ++i) {
+        const int slot = A.slotsB[(size_t)row * A.slots_ld + i];
+        MOA_DEV_CHECK(slot >= 0 && slot < A.n_slots && slot < A.capB, A.status);
+        if (slot >= 0 && slot < 256) allow[slot >> 6] |= 1ull << (slot & 63);
+      }
+    }
     float m_ref = -INFINITY, l_run = 0.f;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t tSg = tS + lane_addr + (uint32_t)(gi * TC_KB), tOg = tO + lane_addr + (uint32_t)(gi * TC_DH);
     bool ok = true;
-    for (int b = 0; b < n_blocks && ok; ++b) {
-      const int i = b & 1;
-      if (!mbar_wait(sfull_bar(i), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
+    for (int b = gi; b < n_blocks && ok; b += 2) {
+      const uint32_t k = (uint32_t)(b >> 1);            // how many blocks this group has done
+      if (!mbar_wait(sfull_bar(gi), k & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float s[TC_KB];
+      float s[NC];
       if (warp_live) {
 #pragma unroll
-        for (int c = 0; c < TC_KB; c += 16) tc_ld16(tS + lane_addr + (uint32_t)(i * TC_KB + c), s + c);
+        for (int c = 0; c < NC; c += 16) tc_ld16(tSg + (uint32_t)(c_lo + c), s + c);
       }
       tc_fence_before();
-      mbar_arrive(sempty_bar(i));
-      {
+      mbar_arrive(sempty_bar(gi));
+      const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
+      if (n_in < TC_KB) {
         // A ragged last block: positions beyond the range carry whatever the cache holds there. Their probabilities are
         // exactly zero, but zero times a non-finite stale value is not, so those V rows are cleared in shared memory
         // (the block has landed: its scores are complete).
-        const int n_keep = min(TC_KB, k_end - (k_begin + b * TC_KB));
-        if (n_keep < TC_KB) {
-          uint8_t* v = bp + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-          for (int j = st_i; j < (TC_KB - n_keep) * 16; j += 128) {
-            const int r = n_keep + (j >> 4), c16 = j & 15;                   // row, 16-byte piece of its 256 bytes
-            *reinterpret_cast<uint4*>(v + (c16 >> 3) * (TC_KV_BYTES / 2) + r * 128 + (c16 & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-          }
+        uint8_t* v = bp + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        for (int j = st_i & 127; j < (TC_KB - n_in) * 16; j += 128) {
+          const int r = n_in + (j >> 4), c16 = j & 15;                   // row, 16-byte piece of its 256 bytes
+          *reinterpret_cast<uint4*>(v + (c16 >> 3) * (TC_KV_BYTES / 2) + r * 128 + (c16 & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
         }
       }
       // block maximum of the raw scores (the scale is positive and goes into the exponent's multiply-add)
-      const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
       float mx = -INFINITY;
       if (warp_live) {
-        if (n_in == TC_KB) {
+        if (tree_part) {                                   // the row sees its ancestors' slots and its own only
+          const unsigned long long word = allow[b & 3] >> c_lo;
 #pragma unroll
-          for (int c = 0; c < TC_KB; ++c) mx = fmaxf(mx, s[c]);
+          for (int c = 0; c < NC; ++c) {
+            s[c] = (c_lo + c < n_in && ((word >> c) & 1ull)) ? s[c] : -INFINITY;
+            mx = fmaxf(mx, s[c]);
+          }
+        } else if (n_in == TC_KB) {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four chains instead of one
+#pragma unroll
+          for (int c = 0; c < NC; ++c) m4[c & 3] = fmaxf(m4[c & 3], s[c]);
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         } else {
 #pragma unroll
-          for (int c = 0; c < TC_KB; ++c) {
-            s[c] = c < n_in ? s[c] : -INFINITY;
+          for (int c = 0; c < NC; ++c) {
+            s[c] = c_lo + c < n_in ? s[c] : -INFINITY;
             mx = fmaxf(mx, s[c]);
           }
         }
       }
       const float m_blk = mx * A.scale_log2;
-      // PV of the block before this one must be done: P is free and O is at rest
-      if (!mbar_wait(pempty_bar, (uint32_t)(b - 1) & 1u, abort_flag)) { ok = false; break; }
-      tc_fence_after();
+      float f = 1.f;
       if (warp_live) {
-        float f = 1.f;
         if (m_ref == -INFINITY) {
           m_ref = m_blk;                                   // nothing accumulated yet for this row
         } else if (m_blk > m_ref + TC_RESCALE_LOG2) {
@@ -276,56 +332,100 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           m_ref = m_blk;
           l_run *= f;
         }
-        if (b > 0 && __any_sync(0xffffffffu, f != 1.f)) {  // rare: the row's output accumulator moves to the new reference
+      }
+      // the group's previous product has left the tensor cores: its P buffer is free and its O is at rest
+      if (!mbar_wait(pempty_bar(gi), (k & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      if (k > 0 && warp_live && __any_sync(0xffffffffu, f != 1.f)) {      // rare: a row's accumulator moves to a new reference
 #pragma unroll 1
-          for (int c = 0; c < TC_DH; c += 16) {
-            float o[16];
-            tc_ld16(tO + lane_addr + (uint32_t)c, o);
+        for (int c = 0; c < TC_DH; c += 16) {
+          float o[16];
+          tc_ld16(tOg + (uint32_t)c, o);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) o[e] *= f;
-            tc_st16(tO + lane_addr + (uint32_t)c, o);
-          }
-          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          for (int e = 0; e < 16; ++e) o[e] *= f;
+          tc_st16(tOg + (uint32_t)c, o);
         }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      }
+      if (warp_live) {
         const float msub = m_ref == -INFINITY ? 0.f : m_ref;
-        float rs = 0.f;
+        float rs[2] = {0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < TC_KB; c += 8) {
+        for (int c = 0; c < NC; c += 8) {
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float p0 = ex2_approx(fmaf(s[c + 2 * e], A.scale_log2, -msub)), p1 = ex2_approx(fmaf(s[c + 2 * e + 1], A.scale_log2, -msub));
-            rs += p0 + p1;
+            rs[0] += p0;
+            rs[1] += p1;
             const uint32_t h = pack_bf16(p0, p1);
             hi[e] = h;
             lo[e] = pack_bf16(p0 - __uint_as_float(h << 16), p1 - __uint_as_float(h & 0xffff0000u));
           }
-          const uint32_t off = sw128_off(ql, c);
-          *reinterpret_cast<uint4*>(bp + oPhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(bp + oPlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          const uint32_t off = sw128_off(ql, c_lo + c);
+          *reinterpret_cast<uint4*>(phi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(phi + TC_P_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
-        l_run += rs;
+        l_run += rs[0] + rs[1];
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
-      mbar_arrive(pfull_bar);
+      mbar_arrive(pfull_bar(gi));
     }
-    // ---- the range's result: (max, sum, unnormalised output) per query, or the normalised rows when this is the only part ----
+    // ---- merge of the CTA's partial softmaxes (2 groups x REPS copies per query), then the range's result: (max, sum,
+    //      unnormalised output) per query, or the normalised rows when this range is the attention's only part ----
     if (ok && n_blocks > 0) ok = mbar_wait(ofull_bar, 0u, abort_flag);
     tc_fence_after();
-    if (ok && warp_live) {
-      const size_t pidx = ((size_t)row * A.hq + head) * A.n_parts + part;
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-#pragma unroll 1
-      for (int c = 0; c < TC_DH; c += 16) {
-        float o[16];
-        if (n_blocks > 0) {
-          tc_ld16(tO + lane_addr + (uint32_t)c, o);
-        } else {
+    if (!ok) *abort_flag = 1;
+    // the key / value ring is free now: [sub-part][query][2] (max, sum), then two buffers of [sub-part][query][16] output columns
+    constexpr int NSP = 2 * REPS;
+    float* ml_x = reinterpret_cast<float*>(bp + oKV);
+    float* o_x = ml_x + NSP * RPR * 2;
+    const int sp = gi * REPS + rep;
+    const bool has_blocks = gi < n_blocks;                 // this group saw at least one block
+    ml_x[(sp * RPR + qi) * 2 + 0] = has_blocks ? m_ref : -INFINITY;
+    ml_x[(sp * RPR + qi) * 2 + 1] = has_blocks ? l_run : 0.f;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const bool dead = __shfl_sync(0xffffffffu, *abort_flag, 0) != 0;     // warp-uniform: the TMEM loads below are warp-wide
+    float M = -INFINITY;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) o[e] = 0.f;
+    for (int t = 0; t < NSP; ++t) M = fmaxf(M, ml_x[(t * RPR + qi) * 2]);
+    float L = 0.f;
+#pragma unroll
+    for (int t = 0; t < NSP; ++t) {
+      const float mt = ml_x[(t * RPR + qi) * 2];
+      L += mt == -INFINITY ? 0.f : ex2_approx(mt - M) * ml_x[(t * RPR + qi) * 2 + 1];
+    }
+    const float w_own = (!has_blocks || m_ref == -INFINITY) ? 0.f : ex2_approx(m_ref - M);
+    const size_t pidx = ((size_t)row * A.hq + head) * A.n_parts + part;
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+#pragma unroll 1
+    for (int c = 0; c < TC_DH; c += 16) {
+      float o[16];
+      if (has_blocks && warp_live && !dead) {
+        tc_ld16(tOg + (uint32_t)c, o);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] = 0.f;
+      }
+      float* mine = o_x + ((size_t)((c >> 4) & 1) * NSP * RPR + (size_t)sp * RPR + qi) * 16;
+#pragma unroll
+      for (int e = 0; e < 16; e += 4)
+        *reinterpret_cast<float4*>(mine + e) = w_own == 0.f ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                                            : make_float4(o[e] * w_own, o[e + 1] * w_own, o[e + 2] * w_own, o[e + 3] * w_own);
+      asm volatile("bar.sync 1, 256;" ::: "memory");       // (two buffers: the next chunk's writes do not meet this chunk's reads)
+      if (sp == 0 && valid) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[e] = 0.f;
+#pragma unroll
+        for (int t = 0; t < NSP; ++t) {                     // sub-parts added in a fixed order
+          const float* src = o_x + ((size_t)((c >> 4) & 1) * NSP * RPR + (size_t)t * RPR + qi) * 16;
+#pragma unroll
+          for (int e = 0; e < 16; e += 4) {
+            const float4 v4 = *reinterpret_cast<const float4*>(src + e);
+            o[e] += v4.x; o[e + 1] += v4.y; o[e + 2] += v4.z; o[e + 3] += v4.w;
+          }
         }
-        if (!valid) continue;
         if (A.n_parts == 1) {
           bf16* dst = A.out + ((size_t)row * A.hq + head) * TC_DH + c;
           bf16* dlo = A.out + ((size_t)(A.out_lo + row) * A.hq + head) * TC_DH + c;
@@ -349,10 +449,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
         }
       }
-      if (valid && A.n_parts > 1) {
-        A.part_ml[pidx * 2 + 0] = m_ref;           // log2 domain, as attn_combine_kernel expects
-        A.part_ml[pidx * 2 + 1] = l_run;
-      }
+    }
+    if (sp == 0 && valid && A.n_parts > 1) {
+      A.part_ml[pidx * 2 + 0] = M;               // log2 domain, as attn_combine_kernel expects
+      A.part_ml[pidx * 2 + 1] = L;
     }
   }
 
@@ -361,7 +461,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag && A.status) atomicMax(A.status, DEV_ERR_TIMEOUT);
 }
