@@ -404,7 +404,6 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     if (q32 && dh == 128 && !lim.active() && ctx->fast && Qn <= 128 && posA_ld == hkv * dh && kA != nullptr &&
         max_len >= TC_MIN_KEYS && n_slots <= 256) {
       const int blocks = (max_len + TC_KB - 1) / TC_KB;
-      const int reps = Qn <= 64 ? 2 : 1;              // few queries: two copies of each share a block's positions
       int n_split = imax(1, imin(blocks, ctx->sm_count / imax(1, nseq * hkv)));
       const long long per_part = (long long)R * hq;
       while (n_split > 1 && per_part * (n_split + has_tree) > p.att_units) --n_split;
@@ -422,8 +421,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
         return MOA_ERR_CUDA;
       static bool tc_attr = false;
       if (!tc_attr) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_BYTES);
         if (e != cudaSuccess) {
           snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
           return MOA_ERR_CUDA;
@@ -431,8 +429,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
         tc_attr = true;
       }
       const dim3 tgrid(hkv, nseq, n_split + has_tree);
-      if (reps == 2) launch_pdl(attn_tc_kernel<2>, tgrid, dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
-      else launch_pdl(attn_tc_kernel<1>, tgrid, dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
+      launch_pdl(attn_tc_kernel, tgrid, dim3(TC_THREADS), TC_SMEM_BYTES, s, TP);
       MOA_CHECK_LAUNCH();
       if (P.n_parts > 1) {
         const int n_rh = nseq * rows_per_seq * hq;

@@ -3,28 +3,29 @@
 // The split-KV kernel of moa_attn.cuh issues its products with mma.sync from a handful of warps, and at long
 // context (tens of thousands of cached positions per kv head) it is bound by that instruction stream, not by HBM.
 // Here one CTA per (sequence, kv head, key range) keeps all queries that share the kv head -- (rows of the
-// sequence) x (query heads of the group), at most 128 -- as the M = 128 operand in shared memory and streams the
-// cache through a TMA ring of 64-position blocks:
-//   warp 0      TMA producer: K block [64, 128] and V block [64, 128] per stage (128-byte swizzle)
-//   warp 1      one thread issues tcgen05.mma:  S = Q_hi K^T + Q_lo K^T   (A = Q, B = K, both K-major; fp32 in TMEM)
-//                                               O += P_hi V + P_lo V      (A = P from shared memory, K-major;
-//                                                                          B = V as it lies in the cache: MN-major)
+// sequence) x (query heads of the group), at most 128 -- as the M = 128 operand and streams the cache through a TMA
+// ring of 64-position blocks. Both products take their A operand from TENSOR MEMORY, so the only shared-memory
+// traffic of the tensor cores is the cache itself (with A in shared memory the 128-row query and probability tiles,
+// re-read for every block, cost more shared-memory bandwidth than the keys and values and set the pace):
+//   warp 0      TMA producer: K block [64, 128] and V block [64, 128] per stage (128-byte swizzle), six stages
+//   warp 1      one thread issues tcgen05.mma:  S = Q_hi K^T + Q_lo K^T   (A = Q in TMEM, B = K, K-major; fp32 in TMEM)
+//                                               O += P_hi V + P_lo V      (A = P in TMEM, B = V as it lies in the
+//                                                                          cache: MN-major)
 //   warps 2..9  softmax, two groups of four warps that take alternate blocks: a thread owns one query row (TMEM lane)
-//               of its group's blocks: reads its scores, keeps the running maximum and sum in the log2 domain, writes
-//               the probabilities as two bf16 terms into the swizzled P tiles. Each group has its own score buffer,
-//               P buffer and OUTPUT ACCUMULATOR in TMEM, so the groups are independent partial softmaxes (over the
-//               even and the odd blocks) that never wait for one another; they are merged once, at the end.
-// The output accumulator stays in TMEM for the whole key range; it is rescaled only when a row's maximum has grown
-// by more than 2^8 since the last rescale (probabilities then stay below 256, well inside fp32 / bf16 range), so
-// the rescale -- a TMEM load, multiply, store of the row -- happens a few times per range, not per block.
-// A block's softmax is a chain of short dependent steps (TMEM load, maximum, exponentials, shared-memory stores,
-// fences), so one group per CTA would set the pace; two groups overlap their chains. Each CTA leaves (max, sum,
-// unnormalised output) per query for attn_combine_kernel, in the layout of the split-KV kernel. A self-attention's tree segment (the sequence's drafted slots, masked per row by
-// its ancestor list) is one more CTA of the same grid: same pipeline over the tree's keys / values, with the row's
-// slot bitmap applied to the scores. Queries arrive in fp32 and enter as two bf16 terms, as in the split-KV kernel.
-// With at most 64 queries per kv head (REPS = 2) every query occupies two rows of the tile, r and 64 + r, and each copy
-// takes half of a block's 64 positions (its probabilities for the other half are zero): the two copies are
-// independent partial softmaxes too (merged with the groups at the end), and twice as many lanes share the exponentials.
+//               of its group's blocks: reads its 64 scores, keeps the running maximum and sum in the log2 domain, and
+//               writes the probabilities as two bf16 terms over the scores it has just read (P_hi | P_lo take the 64
+//               columns the fp32 scores took). Each group has its own score / probability buffer and its own OUTPUT
+//               ACCUMULATOR, so the groups are independent partial softmaxes (over the even and the odd blocks) that
+//               never wait for one another; they are merged once, at the end.
+// Tensor memory (512 columns): Q_hi 0..63, Q_lo 64..127 (bf16 pairs), S/P of group g at 128 + 64 g, O of group g at
+// 256 + 128 g. An output accumulator is rescaled only when a row's maximum has grown by more than 2^8 since its last
+// rescale (probabilities then stay below 256), so the rescale -- a TMEM load, multiply, store of the row -- happens a
+// few times per range, not per block. A block's softmax is a chain of short dependent steps, so one group per CTA
+// would set the pace; two groups overlap their chains.
+// Each CTA leaves (max, sum, unnormalised output) per query for attn_combine_kernel, in the layout of the split-KV
+// kernel. A self-attention's tree segment (the sequence's drafted slots, masked per row by its ancestor list) is one
+// more CTA of the same grid: same pipeline over the tree's keys / values, with the row's slot bitmap applied to the
+// scores. Queries arrive in fp32 and enter as two bf16 terms, as in the split-KV kernel.
 // Every mbarrier wait is bounded; on expiry the CTA raises the abort flag, drains, frees TMEM and reports
 // DEV_ERR_TIMEOUT through the status word.
 #pragma once
@@ -35,13 +36,12 @@ namespace moa {
 
 constexpr int TC_KB = 64;                 // cache positions per block
 constexpr int TC_DH = 128;
-constexpr int TC_STAGES = 3;
+constexpr int TC_STAGES = 6;
 constexpr int TC_THREADS = 320;            // TMA warp, MMA warp, two softmax groups of four warps
-constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // one query term: two 64-column chunks of [128 rows x 128 B]
-constexpr int TC_P_BYTES = 128 * TC_KB * 2;           // one probability term: [128 rows x 128 B]
 constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-column chunks of [64 rows x 128 B]
 constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + 4 * TC_P_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
+constexpr uint32_t TC_TM_Q = 0, TC_TM_S = 128, TC_TM_O = 256;       // tensor-memory columns (see above)
 constexpr float TC_RESCALE_LOG2 = 8.f;
 
 struct AttnTcParams {
@@ -60,9 +60,20 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t 
 // Instruction descriptor as umma_idesc_bf16, with B taken MN-major.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_bmn(int m, int n) { return umma_idesc_bf16(m, n) | (1u << 16); }
 
-// Byte offset of element (row, col) in a tile of 128-byte rows whose 16-byte chunks are XORed with row & 7.
-__device__ __forceinline__ uint32_t sw128_off(int row, int col) {
-  return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
+// tcgen05.mma with the A operand in tensor memory: row r of A in lane r, elements 2 j and 2 j + 1 of a row as the low and
+// high half of column j (a K = 16 step takes 8 columns).
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
 }
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
   asm volatile(
@@ -74,16 +85,11 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
       : "memory");
 }
 
-template <int REPS>
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams P) {
-  constexpr int RPR = 128 / REPS;            // tile rows per copy of the queries
-  constexpr int NC = TC_KB / REPS;           // positions of a block one copy scores
   extern __shared__ uint8_t tc_smem_raw[];
   const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = tc_smem_raw + (base - smem_u32(tc_smem_raw));
-  // P buffer j: hi term at oP + j * 2 * TC_P_BYTES, lo term TC_P_BYTES behind it
-  constexpr uint32_t oQhi = 0, oQlo = TC_Q_BYTES, oP = 2 * TC_Q_BYTES, oKV = oP + 4 * TC_P_BYTES,
-                     oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
+  constexpr uint32_t oKV = 0, oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
   const uint32_t bar0 = base + oBar;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
@@ -98,13 +104,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   const AttnParams& A = P.a;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x, seq = blockIdx.y, part = blockIdx.z;      // parts along z: the tree part's CTAs are launched last
-  const int Qn = A.rows_per_seq * A.group;           // <= 128 / REPS, checked by the host
+  const int Qn = A.rows_per_seq * A.group;           // <= 128, checked by the host
   pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(sfull_bar(i), 1); mbar_init(sempty_bar(i), 128);
+      mbar_init(sfull_bar(i), 1);
       mbar_init(pfull_bar(i), 128); mbar_init(pempty_bar(i), 1);
     }
     mbar_init(qfull_bar, 256);
@@ -121,7 +127,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base, tO = tmem_base + 128u;          // S buffers at columns 0 and 64, the groups' O at 128 and 256
 
   // the cache was written by earlier kernels of the stream, and so were the queries
   pdl_wait(KID_ATTN);
@@ -164,25 +169,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     if (lane == 0 && n_blocks > 0) {
       constexpr uint32_t IDESC_S = umma_idesc_bf16(128, TC_KB);
       constexpr uint32_t IDESC_O = umma_idesc_bf16_bmn(128, TC_DH);
+      const uint32_t tQ = tmem_base + TC_TM_Q;
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       tc_fence_after();
+      // S of block b into its group's buffer: the buffer held the group's probabilities of block b - 2, so that
+      // block's P V product must have been issued (it has: program order) -- the tensor pipe runs in issue order.
       auto issue_s = [&](int b) -> bool {
         const int st = b % TC_STAGES, i = b & 1;
         if (!mbar_wait(full_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
-        if (!mbar_wait(sempty_bar(i), ((uint32_t)(b >> 1) & 1u) ^ 1u, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t kaddr = base + oKV + st * TC_STAGE_BYTES;
+        const uint64_t kd = umma_desc_sw128(base + oKV + st * TC_STAGE_BYTES);
+        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);
 #pragma unroll
-        for (int ks = 0; ks < TC_DH / 16; ++ks) {
-          const uint64_t bd = umma_desc_sw128(kaddr + (ks >> 2) * (TC_KV_BYTES / 2)) + 2u * (ks & 3);
-          tc_mma_bf16(tS + (uint32_t)(i * TC_KB), umma_desc_sw128(base + oQhi + (ks >> 2) * (TC_Q_BYTES / 2)) + 2u * (ks & 3), bd, IDESC_S,
-                      ks > 0 ? 1u : 0u);
-        }
+        for (int ks = 0; ks < TC_DH / 16; ++ks)            // k-steps 0..3 in the first 64-column chunk of K, 4..7 in the second
+          tc_mma_bf16_ta(d, tQ + (uint32_t)(ks * 8), kd + (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3)), IDESC_S, ks > 0 ? 1u : 0u);
 #pragma unroll
-        for (int ks = 0; ks < TC_DH / 16; ++ks) {
-          const uint64_t bd = umma_desc_sw128(kaddr + (ks >> 2) * (TC_KV_BYTES / 2)) + 2u * (ks & 3);
-          tc_mma_bf16(tS + (uint32_t)(i * TC_KB), umma_desc_sw128(base + oQlo + (ks >> 2) * (TC_Q_BYTES / 2)) + 2u * (ks & 3), bd, IDESC_S, 1u);
-        }
+        for (int ks = 0; ks < TC_DH / 16; ++ks)
+          tc_mma_bf16_ta(d, tQ + 64u + (uint32_t)(ks * 8), kd + (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3)), IDESC_S, 1u);
         tc_commit(sfull_bar(i));
         return true;
       };
@@ -193,16 +196,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(pfull_bar(j), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        const uint32_t paddr = base + oP + (uint32_t)j * 2u * TC_P_BYTES;
+        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * TC_KB);       // P_hi in its first 32 columns, P_lo in the rest
+        const uint32_t d = tmem_base + TC_TM_O + (uint32_t)(j * TC_DH);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16(tO + (uint32_t)(j * TC_DH), umma_desc_sw128(paddr) + 2u * ks, umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2),
-                      IDESC_O, (b > 1 || ks > 0) ? 1u : 0u);
+          tc_mma_bf16_ta(d, pt + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, (b > 1 || ks > 0) ? 1u : 0u);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16(tO + (uint32_t)(j * TC_DH), umma_desc_sw128(paddr + TC_P_BYTES) + 2u * ks,
-                      umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
-        tc_commit(pempty_bar(j));                 // the group's P buffer may be overwritten and its O is at rest once this completes
+          tc_mma_bf16_ta(d, pt + 32u + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
+        tc_commit(pempty_bar(j));                 // the group's O is at rest once this completes
         tc_commit(empty_bar(b % TC_STAGES));      // the stage's K and V are done with
       }
       if (ok) tc_commit(ofull_bar);
@@ -210,58 +212,42 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   } else {
     // ------------------------------ softmax: group gi takes the blocks b with b % 2 == gi ------------------------------
     const int wi = warp - 2;                           // 0..7
-    const int gi = wi >> 2;                            // group: its S buffer, P buffer, O accumulator and barriers have index gi
+    const int gi = wi >> 2;                            // group: its S/P buffer, O accumulator and barriers have index gi
     const int quad = warp & 3;                         // TMEM lane quadrant of this warp
-    const int ql = quad * 32 + lane;                   // tile row = TMEM lane
+    const int ql = quad * 32 + lane;                   // query row = TMEM lane
     const int st_i = threadIdx.x - 64;                 // 0..255 among the softmax threads
-    const int qi = ql % RPR, rep = ql / RPR;           // query of this row, and which copy of it
-    const int c_lo = rep * NC;                         // this copy's positions inside a block: c_lo .. c_lo + NC - 1
-    const bool valid = qi < Qn;
-    const bool warp_live = (quad * 32) % RPR < Qn;     // at least one real query in this warp
-    const int row = seq * A.rows_per_seq + (valid ? qi / A.group : 0);
-    const int head = g * A.group + (valid ? qi % A.group : 0);
-    // ---- queries -> two bf16 terms in shared memory (rows beyond Qn are zero) ----
-    for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 256) {
-      float x[4][8];
-      bool in[4];
+    const bool valid = ql < Qn;
+    const bool warp_live = quad * 32 < Qn;             // at least one real query in this warp
+    const int row = seq * A.rows_per_seq + (valid ? ql / A.group : 0);
+    const int head = g * A.group + (valid ? ql % A.group : 0);
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    // ---- queries -> two bf16 terms in tensor memory: group gi writes head dimensions 64 gi .. 64 gi + 63 of its rows ----
+    if (warp_live) {
+      const float* qsrc = A.q32 + (size_t)row * A.q_ld + head * TC_DH + gi * 64;
+#pragma unroll 1
+      for (int c = 0; c < 64; c += 16) {
+        float x[16];
+        if (valid) {
+          load8_planes(qsrc + c, A.q_splits, A.q_plane, x);
+          load8_planes(qsrc + c + 8, A.q_splits, A.q_plane, x + 8);
+        } else {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 256;
-        const int r = (i >> 4) % RPR, c = i & 15;
-        in[u] = i < 128 * 16 && r < Qn;
-        if (in[u])
-          load8_planes(A.q32 + (size_t)(seq * A.rows_per_seq + r / A.group) * A.q_ld + (g * A.group + r % A.group) * TC_DH + c * 8,
-                       A.q_splits, A.q_plane, x[u]);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * 256;
-        if (i >= 128 * 16) continue;
-        const int r = i >> 4, c = i & 15;
-        uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
-        if (in[u]) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const bf16 h0 = __float2bfloat16_rn(x[u][2 * e]), h1 = __float2bfloat16_rn(x[u][2 * e + 1]);
-            hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-            lo[e] = pack_bf16(x[u][2 * e] - __bfloat162float(h0), x[u][2 * e + 1] - __bfloat162float(h1));
-          }
+          for (int e = 0; e < 16; ++e) x[e] = 0.f;
         }
-        const uint32_t off = (uint32_t)((c >> 3) * (TC_Q_BYTES / 2)) + sw128_off(r, (c & 7) * 8);
-        *reinterpret_cast<uint4*>(bp + oQhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(bp + oQlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-      }
-    }
-    uint8_t* const phi = bp + oP + (uint32_t)gi * 2u * TC_P_BYTES;      // the group's P tile (hi term; lo TC_P_BYTES behind)
-    if (REPS > 1) {            // a copy's probabilities outside its own positions are zero, once and for all
+        uint32_t hi[8], lo[8];
 #pragma unroll
-      for (int c = 0; c < TC_KB; c += 8)
-        if (c < c_lo || c >= c_lo + NC) {
-          *reinterpret_cast<uint4*>(phi + sw128_off(ql, c)) = make_uint4(0u, 0u, 0u, 0u);
-          *reinterpret_cast<uint4*>(phi + TC_P_BYTES + sw128_off(ql, c)) = make_uint4(0u, 0u, 0u, 0u);
+        for (int e = 0; e < 8; ++e) {
+          const bf16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
+          hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+          lo[e] = pack_bf16(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
         }
+        const uint32_t col = (uint32_t)((gi * 64 + c) / 2);
+        tc_st8(tmem_base + TC_TM_Q + lane_addr + col, hi);
+        tc_st8(tmem_base + TC_TM_Q + 64u + lane_addr + col, lo);
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
     mbar_arrive(qfull_bar);
 
     // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per key block
@@ -274,20 +260,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
     }
     float m_ref = -INFINITY, l_run = 0.f;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const uint32_t tSg = tS + lane_addr + (uint32_t)(gi * TC_KB), tOg = tO + lane_addr + (uint32_t)(gi * TC_DH);
+    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * TC_KB);
+    const uint32_t tOg = tmem_base + TC_TM_O + lane_addr + (uint32_t)(gi * TC_DH);
     bool ok = true;
     for (int b = gi; b < n_blocks && ok; b += 2) {
       const uint32_t k = (uint32_t)(b >> 1);            // how many blocks this group has done
       if (!mbar_wait(sfull_bar(gi), k & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float s[NC];
+      float s[TC_KB];
       if (warp_live) {
 #pragma unroll
-        for (int c = 0; c < NC; c += 16) tc_ld16(tSg + (uint32_t)(c_lo + c), s + c);
+        for (int c = 0; c < TC_KB; c += 16) tc_ld16(tSg + (uint32_t)c, s + c);
       }
-      tc_fence_before();
-      mbar_arrive(sempty_bar(gi));
       const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
       if (n_in < TC_KB) {
         // A ragged last block: positions beyond the range carry whatever the cache holds there. Their probabilities are
@@ -298,26 +282,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           const int r = n_in + (j >> 4), c16 = j & 15;                   // row, 16-byte piece of its 256 bytes
           *reinterpret_cast<uint4*>(v + (c16 >> 3) * (TC_KV_BYTES / 2) + r * 128 + (c16 & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       }
       // block maximum of the raw scores (the scale is positive and goes into the exponent's multiply-add)
       float mx = -INFINITY;
       if (warp_live) {
         if (tree_part) {                                   // the row sees its ancestors' slots and its own only
-          const unsigned long long word = allow[b & 3] >> c_lo;
+          const unsigned long long word = allow[b & 3];
 #pragma unroll
-          for (int c = 0; c < NC; ++c) {
-            s[c] = (c_lo + c < n_in && ((word >> c) & 1ull)) ? s[c] : -INFINITY;
+          for (int c = 0; c < TC_KB; ++c) {
+            s[c] = (c < n_in && ((word >> c) & 1ull)) ? s[c] : -INFINITY;
             mx = fmaxf(mx, s[c]);
           }
         } else if (n_in == TC_KB) {
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four chains instead of one
 #pragma unroll
-          for (int c = 0; c < NC; ++c) m4[c & 3] = fmaxf(m4[c & 3], s[c]);
+          for (int c = 0; c < TC_KB; ++c) m4[c & 3] = fmaxf(m4[c & 3], s[c]);
           mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         } else {
 #pragma unroll
-          for (int c = 0; c < NC; ++c) {
-            s[c] = c_lo + c < n_in ? s[c] : -INFINITY;
+          for (int c = 0; c < TC_KB; ++c) {
+            s[c] = c < n_in ? s[c] : -INFINITY;
             mx = fmaxf(mx, s[c]);
           }
         }
@@ -333,10 +318,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           l_run *= f;
         }
       }
-      // the group's previous product has left the tensor cores: its P buffer is free and its O is at rest
-      if (!mbar_wait(pempty_bar(gi), (k & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      if (k > 0 && warp_live && __any_sync(0xffffffffu, f != 1.f)) {      // rare: a row's accumulator moves to a new reference
+      if (k > 0 && warp_live && __any_sync(0xffffffffu, f != 1.f)) {
+        // rare: a row's accumulator moves to a new reference; the group's previous product must have left the tensor cores
+        if (!mbar_wait(pempty_bar(gi), (k & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll 1
         for (int c = 0; c < TC_DH; c += 16) {
           float o[16];
@@ -345,16 +330,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           for (int e = 0; e < 16; ++e) o[e] *= f;
           tc_st16(tOg + (uint32_t)c, o);
         }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
       if (warp_live) {
+        // probabilities as two bf16 terms over the scores just read: P_hi in columns 0..31 of the buffer, P_lo in 32..63
         const float msub = m_ref == -INFINITY ? 0.f : m_ref;
         float rs[2] = {0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < NC; c += 8) {
-          uint32_t hi[4], lo[4];
+        for (int c = 0; c < TC_KB; c += 16) {
+          uint32_t hi[8], lo[8];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
+          for (int e = 0; e < 8; ++e) {
             const float p0 = ex2_approx(fmaf(s[c + 2 * e], A.scale_log2, -msub)), p1 = ex2_approx(fmaf(s[c + 2 * e + 1], A.scale_log2, -msub));
             rs[0] += p0;
             rs[1] += p1;
@@ -362,26 +347,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
             hi[e] = h;
             lo[e] = pack_bf16(p0 - __uint_as_float(h << 16), p1 - __uint_as_float(h & 0xffff0000u));
           }
-          const uint32_t off = sw128_off(ql, c_lo + c);
-          *reinterpret_cast<uint4*>(phi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(phi + TC_P_BYTES + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          tc_st8(tSg + (uint32_t)(c / 2), hi);
+          tc_st8(tSg + 32u + (uint32_t)(c / 2), lo);
         }
         l_run += rs[0] + rs[1];
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       mbar_arrive(pfull_bar(gi));
     }
-    // ---- merge of the CTA's partial softmaxes (2 groups x REPS copies per query), then the range's result: (max, sum,
+    // ---- merge of the CTA's two partial softmaxes (one per group), then the range's result: (max, sum,
     //      unnormalised output) per query, or the normalised rows when this range is the attention's only part ----
     if (ok && n_blocks > 0) ok = mbar_wait(ofull_bar, 0u, abort_flag);
     tc_fence_after();
     if (!ok) *abort_flag = 1;
     // the key / value ring is free now: [sub-part][query][2] (max, sum), then two buffers of [sub-part][query][16] output columns
-    constexpr int NSP = 2 * REPS;
+    constexpr int NSP = 2, RPR = 128;
+    const int qi = ql;
     float* ml_x = reinterpret_cast<float*>(bp + oKV);
     float* o_x = ml_x + NSP * RPR * 2;
-    const int sp = gi * REPS + rep;
+    const int sp = gi;
     const bool has_blocks = gi < n_blocks;                 // this group saw at least one block
     ml_x[(sp * RPR + qi) * 2 + 0] = has_blocks ? m_ref : -INFINITY;
     ml_x[(sp * RPR + qi) * 2 + 1] = has_blocks ? l_run : 0.f;
