@@ -4,21 +4,23 @@
 // context (tens of thousands of cached positions per kv head) it is bound by that instruction stream, not by HBM.
 // Here one CTA per (sequence, kv head, key range) keeps all queries that share the kv head -- (rows of the
 // sequence) x (query heads of the group), at most 128 -- as the M = 128 operand and streams the cache through a TMA
-// ring of 64-position blocks. Both products take their A operand from TENSOR MEMORY, so the only shared-memory
-// traffic of the tensor cores is the cache itself (with A in shared memory the 128-row query and probability tiles,
-// re-read for every block, cost more shared-memory bandwidth than the keys and values and set the pace):
-//   warp 0      TMA producer: K block [64, 128] and V block [64, 128] per stage (128-byte swizzle), six stages
-//   warp 1      one thread issues tcgen05.mma:  S = Q_hi K^T + Q_lo K^T   (A = Q in TMEM, B = K, K-major; fp32 in TMEM)
+// ring of 64-position blocks:
+//   warp 0      TMA producer: K block [64, 128] and V block [64, 128] per stage (128-byte swizzle), five stages
+//   warp 1      one thread issues tcgen05.mma:  S_hi = Q_hi K^T, S_lo = Q_lo K^T  (A = Q in shared memory, B = K, both
+//                                                                          K-major; two fp32 accumulators in TMEM)
 //                                               O += P_hi V + P_lo V      (A = P in TMEM, B = V as it lies in the
 //                                                                          cache: MN-major)
+//               Products that accumulate into the same TMEM tile run one after the other at the tensor pipe's latency
+//               (about 90 cycles each with these small N), and that chain, not the math or the memory, sets a block's
+//               pace. So the two query terms go to two accumulators (two chains of 8 that interleave instead of one
+//               of 16; the softmax thread adds them).
 //   warps 2..9  softmax, two groups of four warps that take alternate blocks: a thread owns one query row (TMEM lane)
 //               of its group's blocks: reads its 64 scores, keeps the running maximum and sum in the log2 domain, and
 //               writes the probabilities as two bf16 terms over the scores it has just read (P_hi | P_lo take the 64
-//               columns the fp32 scores took). Each group has its own score / probability buffer and its own OUTPUT
+//               columns S_hi took). Each group has its own score / probability buffers and its own OUTPUT
 //               ACCUMULATOR, so the groups are independent partial softmaxes (over the even and the odd blocks) that
 //               never wait for one another; they are merged once, at the end.
-// Tensor memory (512 columns): Q_hi 0..63, Q_lo 64..127 (bf16 pairs), S/P of group g at 128 + 64 g, O of group g at
-// 256 + 128 g. An output accumulator is rescaled only when a row's maximum has grown by more than 2^8 since its last
+// Tensor memory (512 columns): S_hi (then P) of group g at 128 g, S_lo at 128 g + 64, O of group g at 256 + 128 g. An output accumulator is rescaled only when a row's maximum has grown by more than 2^8 since its last
 // rescale (probabilities then stay below 256), so the rescale -- a TMEM load, multiply, store of the row -- happens a
 // few times per range, not per block. A block's softmax is a chain of short dependent steps, so one group per CTA
 // would set the pace; two groups overlap their chains.
@@ -36,12 +38,13 @@ namespace moa {
 
 constexpr int TC_KB = 64;                 // cache positions per block
 constexpr int TC_DH = 128;
-constexpr int TC_STAGES = 6;
+constexpr int TC_STAGES = 5;
 constexpr int TC_THREADS = 320;            // TMA warp, MMA warp, two softmax groups of four warps
 constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-column chunks of [64 rows x 128 B]
 constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
-constexpr uint32_t TC_TM_Q = 0, TC_TM_S = 128, TC_TM_O = 256;       // tensor-memory columns (see above)
+constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // one query term: two 64-column chunks of [128 rows x 128 B]
+constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
+constexpr uint32_t TC_TM_S = 0, TC_TM_O = 256;        // tensor-memory columns (see above)
 constexpr float TC_RESCALE_LOG2 = 8.f;
 
 struct AttnTcParams {
@@ -60,6 +63,10 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t 
 // Instruction descriptor as umma_idesc_bf16, with B taken MN-major.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_bmn(int m, int n) { return umma_idesc_bf16(m, n) | (1u << 16); }
 
+// Byte offset of element (row, col) in a tile of 128-byte rows whose 16-byte chunks are XORed with row & 7.
+__device__ __forceinline__ uint32_t sw128_off(int row, int col) {
+  return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
+}
 // tcgen05.mma with the A operand in tensor memory: row r of A in lane r, elements 2 j and 2 j + 1 of a row as the low and
 // high half of column j (a K = 16 step takes 8 columns).
 __device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -89,7 +96,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   extern __shared__ uint8_t tc_smem_raw[];
   const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = tc_smem_raw + (base - smem_u32(tc_smem_raw));
-  constexpr uint32_t oKV = 0, oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
+  constexpr uint32_t oQhi = 0, oQlo = TC_Q_BYTES, oKV = 2 * TC_Q_BYTES, oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
   const uint32_t bar0 = base + oBar;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
@@ -169,23 +176,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     if (lane == 0 && n_blocks > 0) {
       constexpr uint32_t IDESC_S = umma_idesc_bf16(128, TC_KB);
       constexpr uint32_t IDESC_O = umma_idesc_bf16_bmn(128, TC_DH);
-      const uint32_t tQ = tmem_base + TC_TM_Q;
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       tc_fence_after();
-      // S of block b into its group's buffer: the buffer held the group's probabilities of block b - 2, so that
-      // block's P V product must have been issued (it has: program order) -- the tensor pipe runs in issue order.
+      const uint64_t qhd = umma_desc_sw128(base + oQhi), qld = umma_desc_sw128(base + oQlo);
+      // S of block b into its group's two accumulators. They held the group's probabilities of block b - 2, whose P V
+      // product has been issued before (program order): the tensor pipe runs in issue order.
       auto issue_s = [&](int b) -> bool {
         const int st = b % TC_STAGES, i = b & 1;
         if (!mbar_wait(full_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint64_t kd = umma_desc_sw128(base + oKV + st * TC_STAGE_BYTES);
-        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);
+        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * 128);
 #pragma unroll
-        for (int ks = 0; ks < TC_DH / 16; ++ks)            // k-steps 0..3 in the first 64-column chunk of K, 4..7 in the second
-          tc_mma_bf16_ta(d, tQ + (uint32_t)(ks * 8), kd + (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3)), IDESC_S, ks > 0 ? 1u : 0u);
-#pragma unroll
-        for (int ks = 0; ks < TC_DH / 16; ++ks)
-          tc_mma_bf16_ta(d, tQ + 64u + (uint32_t)(ks * 8), kd + (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3)), IDESC_S, 1u);
+        for (int ks = 0; ks < TC_DH / 16; ++ks) {          // k-steps 0..3 in the first 64-column chunk, 4..7 in the second
+          const uint64_t qo = (uint64_t)((ks >> 2) * (TC_Q_BYTES / 2 / 16) + 2 * (ks & 3));
+          const uint64_t ko = (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3));
+          tc_mma_bf16(d, qhd + qo, kd + ko, IDESC_S, ks > 0 ? 1u : 0u);           // the two chains interleave
+          tc_mma_bf16(d + 64u, qld + qo, kd + ko, IDESC_S, ks > 0 ? 1u : 0u);
+        }
         tc_commit(sfull_bar(i));
         return true;
       };
@@ -196,7 +204,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(pfull_bar(j), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * TC_KB);       // P_hi in its first 32 columns, P_lo in the rest
+        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * 128);         // P_hi in its first 32 columns, P_lo in the next 32
         const uint32_t d = tmem_base + TC_TM_O + (uint32_t)(j * TC_DH);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
@@ -221,33 +229,39 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     const int row = seq * A.rows_per_seq + (valid ? ql / A.group : 0);
     const int head = g * A.group + (valid ? ql % A.group : 0);
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    // ---- queries -> two bf16 terms in tensor memory: group gi writes head dimensions 64 gi .. 64 gi + 63 of its rows ----
-    if (warp_live) {
-      const float* qsrc = A.q32 + (size_t)row * A.q_ld + head * TC_DH + gi * 64;
-#pragma unroll 1
-      for (int c = 0; c < 64; c += 16) {
-        float x[16];
-        if (valid) {
-          load8_planes(qsrc + c, A.q_splits, A.q_plane, x);
-          load8_planes(qsrc + c + 8, A.q_splits, A.q_plane, x + 8);
-        } else {
+    // ---- queries -> two bf16 terms in shared memory (rows beyond Qn are zero) ----
+    for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 256) {
+      float x[4][8];
+      bool in[4];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) x[e] = 0.f;
-        }
-        uint32_t hi[8], lo[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const bf16 h0 = __float2bfloat16_rn(x[2 * e]), h1 = __float2bfloat16_rn(x[2 * e + 1]);
-          hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-          lo[e] = pack_bf16(x[2 * e] - __bfloat162float(h0), x[2 * e + 1] - __bfloat162float(h1));
-        }
-        const uint32_t col = (uint32_t)((gi * 64 + c) / 2);
-        tc_st8(tmem_base + TC_TM_Q + lane_addr + col, hi);
-        tc_st8(tmem_base + TC_TM_Q + 64u + lane_addr + col, lo);
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 256;
+        const int r = i >> 4, c = i & 15;
+        in[u] = i < 128 * 16 && r < Qn;
+        if (in[u])
+          load8_planes(A.q32 + (size_t)(seq * A.rows_per_seq + r / A.group) * A.q_ld + (g * A.group + r % A.group) * TC_DH + c * 8,
+                       A.q_splits, A.q_plane, x[u]);
       }
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 256;
+        if (i >= 128 * 16) continue;
+        const int r = i >> 4, c = i & 15;
+        uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
+        if (in[u]) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const bf16 h0 = __float2bfloat16_rn(x[u][2 * e]), h1 = __float2bfloat16_rn(x[u][2 * e + 1]);
+            hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+            lo[e] = pack_bf16(x[u][2 * e] - __bfloat162float(h0), x[u][2 * e + 1] - __bfloat162float(h1));
+          }
+        }
+        const uint32_t off = (uint32_t)((c >> 3) * (TC_Q_BYTES / 2)) + sw128_off(r, (c & 7) * 8);
+        *reinterpret_cast<uint4*>(bp + oQhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(bp + oQlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
     }
-    tc_fence_before();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     mbar_arrive(qfull_bar);
 
     // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per key block
@@ -260,7 +274,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
     }
     float m_ref = -INFINITY, l_run = 0.f;
-    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * TC_KB);
+    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * 128);      // S_hi (later P); S_lo 64 columns on
     const uint32_t tOg = tmem_base + TC_TM_O + lane_addr + (uint32_t)(gi * TC_DH);
     bool ok = true;
     for (int b = gi; b < n_blocks && ok; b += 2) {
@@ -270,7 +284,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       float s[TC_KB];
       if (warp_live) {
 #pragma unroll
-        for (int c = 0; c < TC_KB; c += 16) tc_ld16(tSg + (uint32_t)c, s + c);
+        for (int c = 0; c < TC_KB; c += 16) {
+          float t2[16];
+          tc_ld16(tSg + (uint32_t)c, s + c);
+          tc_ld16(tSg + 64u + (uint32_t)c, t2);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) s[c + e] += t2[e];
+        }
       }
       const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
       if (n_in < TC_KB) {
