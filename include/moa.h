@@ -51,7 +51,9 @@ typedef enum {
   MOA_ERR_STATE = 7,      /* calls out of order (e.g. draft step before moa_tree_begin) */
   MOA_ERR_ARCH = 8,       /* the current device is not compute capability 10.x */
   MOA_ERR_CUDA = 9,       /* a CUDA runtime call failed; see moa_last_cuda_error() */
-  MOA_ERR_TIMEOUT = 10    /* a bounded device-side wait expired */
+  MOA_ERR_TIMEOUT = 10,   /* a bounded device-side wait expired */
+  MOA_ERR_NONFINITE = 11  /* moa_state_status only: a tree expansion met a log-probability that is not a number (it
+                             ranked that candidate last); the drafted tree of that cycle is not to be trusted */
 } moa_status;
 
 typedef enum { MOA_F32 = 0, MOA_BF16 = 1 } moa_dtype;

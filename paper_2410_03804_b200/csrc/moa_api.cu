@@ -1113,6 +1113,7 @@ const char* moa_status_str(moa_status s) {
     case MOA_ERR_ARCH: return "device is not compute capability 10.x";
     case MOA_ERR_CUDA: return "CUDA error";
     case MOA_ERR_TIMEOUT: return "device-side wait timed out";
+    case MOA_ERR_NONFINITE: return "a log-probability was not a number";
   }
   return "unknown";
 }

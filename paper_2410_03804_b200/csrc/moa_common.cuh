@@ -185,7 +185,7 @@ struct SeqSplit {
 };
 
 // Device-side status word values (mirrors moa_status where it matters).
-enum : int { DEV_OK = 0, DEV_ERR_BOUNDS = 6, DEV_ERR_TIMEOUT = 10 };
+enum : int { DEV_OK = 0, DEV_ERR_BOUNDS = 6, DEV_ERR_TIMEOUT = 10, DEV_ERR_NONFINITE = 11 };
 
 // Debug build (-DMOA_CHECKS): indices that the host logic guarantees (token ids, tree slots, cache lengths) are
 // checked where they are used; a violation raises the status word and the access is skipped or clamped as in the

@@ -126,9 +126,20 @@ __global__ void __launch_bounds__(512) tree_expand_kernel(TreePtrs t, int B, int
   // 1. children: score and pool append
   for (int c = tid; c < C; c += blockDim.x) {
     const int r = c / B, j = c - r * B;
-    const int par = step == 0 ? -1 : frontier[r];
+    int par = step == 0 ? -1 : frontier[r];
+    if (step > 0 && (unsigned)par >= (unsigned)P) {     // a frontier entry is a pool index by construction
+      atomicMax(t.status, DEV_ERR_BOUNDS);
+      par = 0;
+    }
     const float ps = step == 0 ? 0.f : pool_score[par];
-    const float s = ps + topk_logp[(size_t)(row0 + r) * B + j];
+    float s = ps + topk_logp[(size_t)(row0 + r) * B + j];
+    // The ranks below are a permutation only under a total order, and a NaN compares false with everything: a
+    // log-probability that is not a number (a fault upstream) ranks last and is reported, instead of leaving
+    // frontier entries unwritten.
+    if (s != s) {
+      atomicMax(t.status, DEV_ERR_NONFINITE);
+      s = -INFINITY;
+    }
     c_score[c] = s;
     pool_tok[base + c] = topk_id[(size_t)(row0 + r) * B + j];
     pool_parent[base + c] = par;

@@ -56,6 +56,35 @@ def test_tree_expand_and_finalize_bit_exact(B, D, m, batch):
                           torch.zeros((batch * B, B), dtype=torch.float32).cuda())
 
 
+def test_tree_expand_reports_a_log_probability_that_is_not_a_number():
+    """The ranks of an expansion are a permutation only under a total order. A NaN among the log-probabilities (a fault
+    upstream of the tree) must rank last and raise status 11 instead of leaving frontier entries unwritten: every
+    parent stays a valid slot of the kept tree."""
+    B, D, m, batch = 4, 3, 8, 2
+    p, g = _tiny_model(B, D, m, batch)
+    rng = np.random.default_rng(7)
+    g.moa_tree_begin(torch.from_numpy(rng.integers(0, 1024, batch).astype(np.int32)).cuda())
+    outs = None
+    for s in range(D):
+        R = batch * (1 if s == 0 else B)
+        lp = -np.sort(rng.exponential(1.0, (R, B)), axis=-1).astype(np.float32)
+        if s < 2:
+            lp[0, :] = np.nan                       # a whole row at the first steps, one entry later
+        else:
+            lp[-1, 1] = np.nan
+        ids = rng.integers(0, 1024, (R, B)).astype(np.int32)
+        outs = g.moa_tree_expand(torch.from_numpy(ids).cuda(), torch.from_numpy(lp).cuda())
+    torch.cuda.synchronize()
+    assert g.moa_state_status() == 11
+    tok, parent, depth, score, n = [t.cpu().numpy() for t in outs]
+    for b in range(batch):
+        k = int(n[b])
+        assert 1 <= k <= m + 1
+        assert parent[b, 0] == -1 and np.all((parent[b, 1:k] >= 0) & (parent[b, 1:k] < np.arange(1, k)))
+        assert np.all(depth[b, 1:k] == depth[b, parent[b, 1:k]] + 1)
+        assert not np.isnan(score[b, :k]).any()
+
+
 def g_mask(parent_np, packed=False):
     from paper_2410_03804_b200 import moa
     t = torch.from_numpy(np.ascontiguousarray(parent_np.astype(np.int32))).cuda()
