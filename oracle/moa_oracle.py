@@ -534,9 +534,10 @@ def greedy_chain(dr: Drafter, prefix_toks, root_tok, caK, caV, K_draft, tliK=Non
 # client-server message codec (Section 4.2 "Client-Server"; message-size table in the appendix)
 # --------------------------------------------------------------------------
 def pack_tree(tok, parent):
-    """Client message: every draft-tree node as 3 bytes of token id (little endian) + 1 byte for its position
-    in the tree, 4 bytes per node, so a tree of M nodes is a 4M-byte message (the table's "4M").
-    Reading: the position byte is the parent's slot number (a tree is its parent list; slots are < 255); 255
+    """Client message (Section 4.2): a draft-tree node takes four bytes, three for the token id (little endian) and
+    the fourth for where the node sits in the tree, so a tree of M nodes is a message of 4M bytes, the size the
+    message-size table gives.
+    Reading: the fourth byte is the parent's slot number (a tree is its parent list; slots are < 255); 255
     marks "no parent" (the root, or an unused slot, whose token bytes are ff ff ff).
     tok, parent [n] -> uint8 [n, 4]."""
     n = len(tok)
