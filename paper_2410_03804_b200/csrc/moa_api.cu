@@ -375,7 +375,10 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
                             const float* q32, int q_splits, size_t q_plane, int q_ld, int R, int hq, int hkv, const T* kA, const T* vA, int capA, int posA_ld, const int* lenA,
                             int nA_fixed, int max_len, const T* kB, const T* vB, int capB, const int* slotsB,
                             int slots_ld, int nB, int n_slots, int rows_per_seq, T* out,
-                            RowLimit lim = RowLimit{nullptr, 0, 0}, void* status_word = nullptr) {
+                            RowLimit lim = RowLimit{nullptr, 0, 0}, void* status_word = nullptr, bool cache_settled = false) {
+  // cache_settled: segment A and its lengths were complete before the launch chain of this call began (a draft step: the
+  // caches are written by the append calls, which end with an ordinary launch), so a kernel may read them before it
+  // waits on its predecessor in the chain
   if (R <= 0) return MOA_OK;
   if (sizeof(T) == 2) {
     AttnParams P;
@@ -413,6 +416,7 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
       P.n_split = n_split;
       P.n_parts = n_split + has_tree;
       TP.a = P;
+      TP.early_cache = cache_settled ? 1 : 0;
       const int cache_rows = ctx->c.max_batch * capA;
       if (!encode_map(ctx, &TP.tmK, kA, cache_rows, hkv * dh, TC_KB) || !encode_map(ctx, &TP.tmV, vA, cache_rows, hkv * dh, TC_KB))
         return MOA_ERR_CUDA;
@@ -795,7 +799,7 @@ static moa_status tree_attn_layer(moa_ctx* ctx, moa_state* st, cudaStream_t s, c
   MOA_CHECK_LAUNCH();
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, a.hq, a.hkv, (const T*)a.ck, (const T*)a.cv, c.max_ctx, nkv,
                        st->sa_len, 0, max_len, (const T*)a.tk, (const T*)a.tv, L.NS, row_anc, D, step + 1,
-                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word));
+                       step == 0 ? 1 : 1 + step * B, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word, true));
   {
     const void* W1[1] = {a.wo};
     const int N1[1] = {E};
@@ -860,7 +864,7 @@ static moa_status draft_step_t(moa_ctx* ctx, moa_state* st, int batch, int* topk
   // bf16 path: the attention kernel reads the projection's split planes itself (fp32 queries, two bf16 terms)
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32 ? lo.part : nullptr, lo.splits, lo.plane, cq, R, c.ca_hq, c.ca_hkv,
                        (const T*)st->ca_k, (const T*)st->ca_v, c.max_ctx, ckv, st->ca_len, 0, max_ca, (const T*)nullptr,
-                       (const T*)nullptr, 0, nullptr, 0, 0, 0, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word));
+                       (const T*)nullptr, 0, nullptr, 0, 0, 0, rows_per_seq, obuf, RowLimit{nullptr, 0, 0}, status_word, true));
   {
     const void* W1[1] = {w.ca_wo};
     const int N1[1] = {E};

@@ -44,13 +44,15 @@ constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-
 constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;
 constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // one query term: two 64-column chunks of [128 rows x 128 B]
 constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
-constexpr uint32_t TC_TM_S = 0, TC_TM_O = 256;        // tensor-memory columns (see above)
+constexpr uint32_t TC_TM_Q = 0, TC_TM_S = 128, TC_TM_O = 256;   // tensor-memory columns (see above)
 constexpr float TC_RESCALE_LOG2 = 8.f;
 
 struct AttnTcParams {
   CUtensorMap tmK, tmV;      // cache [positions of all sequences, hkv * 128], box 64 columns x 64 positions, swizzle 128B
   CUtensorMap tmKB, tmVB;    // tree slots [slots of all sequences, hkv * 128], same box (used when a.n_parts > a.n_split)
   AttnParams a;              // queries (fp32), lengths, part buffers; part a.n_split, if any, is the tree segment
+  int early_cache;           // the cache segment (and its lengths) were complete before the chain this launch belongs to
+                             // began: its first blocks may be fetched before the wait on the preceding kernel
 };
 
 // Shared-memory descriptor of an MN-major bf16 operand with the 128-byte swizzle: 64 elements along MN are contiguous
@@ -63,10 +65,6 @@ __device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t 
 // Instruction descriptor as umma_idesc_bf16, with B taken MN-major.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16_bmn(int m, int n) { return umma_idesc_bf16(m, n) | (1u << 16); }
 
-// Byte offset of element (row, col) in a tile of 128-byte rows whose 16-byte chunks are XORed with row & 7.
-__device__ __forceinline__ uint32_t sw128_off(int row, int col) {
-  return (uint32_t)(row * 128 + ((((col >> 3) ^ (row & 7))) << 4) + (col & 7) * 2);
-}
 // tcgen05.mma with the A operand in tensor memory: row r of A in lane r, elements 2 j and 2 j + 1 of a row as the low and
 // high half of column j (a K = 16 step takes 8 columns).
 __device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -76,6 +74,27 @@ __device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem,
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// 64 consecutive columns of this thread's lane in one instruction
+__device__ __forceinline__ void tc_ld64(uint32_t taddr, float* v) {
+  uint32_t r[64];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]),
+        "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]),
+        "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]),
+        "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* r) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
@@ -101,7 +120,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
   auto sfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + i); };
-  auto sempty_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + 2 + i); };
   auto pfull_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 4 + j); };
   auto pempty_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 6 + j); };
   const uint32_t qfull_bar = bar0 + 8u * (2 * TC_STAGES + 8), ofull_bar = qfull_bar + 8u;
@@ -135,9 +153,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // the cache was written by earlier kernels of the stream, and so were the queries
-  pdl_wait(KID_ATTN);
-  const bool tree_part = part >= A.n_split;          // the grid's last CTA along x when the attention has a tree segment
+  // The queries and the tree slots come from the kernels just before this one. A cache segment that was complete
+  // before the chain began needs no wait: its producer warp sends the first ring of blocks at once and waits after.
+  const bool tree_part = part >= A.n_split;          // the grid's last CTA along z when the attention has a tree segment
+  const bool early = P.early_cache != 0 && !tree_part;
+  if (!(early && warp == 0)) pdl_wait(KID_ATTN);
   int k_begin, k_end, n_blocks;
   if (!tree_part) {
     const int len = A.lenA ? A.lenA[seq] : A.nA_fixed;
@@ -156,7 +176,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       const int x0 = g * TC_DH;
+      bool waited = !early;
       for (int b = 0; b < n_blocks; ++b) {
+        if (!waited && b >= TC_STAGES) { pdl_wait(KID_ATTN); waited = true; }
         const int st = b % TC_STAGES;
         const uint32_t k = (uint32_t)(b / TC_STAGES);
         if (!mbar_wait(empty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
@@ -170,6 +192,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         tma_load_2d(dst + TC_KV_BYTES, tv, x0, y, full_bar(st));
         tma_load_2d(dst + TC_KV_BYTES + TC_KV_BYTES / 2, tv, x0 + 64, y, full_bar(st));
       }
+      if (!waited) pdl_wait(KID_ATTN);
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -178,21 +201,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       constexpr uint32_t IDESC_O = umma_idesc_bf16_bmn(128, TC_DH);
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       tc_fence_after();
-      const uint64_t qhd = umma_desc_sw128(base + oQhi), qld = umma_desc_sw128(base + oQlo);
-      // S of block b into its group's two accumulators. They held the group's probabilities of block b - 2, whose P V
-      // product has been issued before (program order): the tensor pipe runs in issue order.
+      // S of block b into its group's score accumulator: both query terms, A from tensor memory (the shared-memory
+      // operand path then carries the keys only), one chain of 16 products. The accumulator held the group's
+      // probabilities of block b - 2, whose P V product has been issued before (program order): the tensor pipe runs
+      // in issue order.
       auto issue_s = [&](int b) -> bool {
         const int st = b % TC_STAGES, i = b & 1;
         if (!mbar_wait(full_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint64_t kd = umma_desc_sw128(base + oKV + st * TC_STAGE_BYTES);
-        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * 128);
+        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * 64);
 #pragma unroll
-        for (int ks = 0; ks < TC_DH / 16; ++ks) {          // k-steps 0..3 in the first 64-column chunk, 4..7 in the second
-          const uint64_t qo = (uint64_t)((ks >> 2) * (TC_Q_BYTES / 2 / 16) + 2 * (ks & 3));
+        for (int ks = 0; ks < TC_DH / 16; ++ks) {          // k-steps 0..3 in the first 64-column chunk of K, 4..7 in the second
           const uint64_t ko = (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3));
-          tc_mma_bf16(d, qhd + qo, kd + ko, IDESC_S, ks > 0 ? 1u : 0u);           // the two chains interleave
-          tc_mma_bf16(d + 64u, qld + qo, kd + ko, IDESC_S, ks > 0 ? 1u : 0u);
+          tc_mma_bf16_ta(d, tmem_base + TC_TM_Q + (uint32_t)(ks * 8), kd + ko, IDESC_S, ks > 0 ? 1u : 0u);
+          tc_mma_bf16_ta(d, tmem_base + TC_TM_Q + 64u + (uint32_t)(ks * 8), kd + ko, IDESC_S, 1u);
         }
         tc_commit(sfull_bar(i));
         return true;
@@ -204,7 +227,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (!mbar_wait(pfull_bar(j), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * 128);         // P_hi in its first 32 columns, P_lo in the next 32
+        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * 64);          // P_hi in its first 32 columns, P_lo in the next 32
         const uint32_t d = tmem_base + TC_TM_O + (uint32_t)(j * TC_DH);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
@@ -256,12 +279,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
             lo[e] = pack_bf16(x[u][2 * e] - __bfloat162float(h0), x[u][2 * e + 1] - __bfloat162float(h1));
           }
         }
-        const uint32_t off = (uint32_t)((c >> 3) * (TC_Q_BYTES / 2)) + sw128_off(r, (c & 7) * 8);
+        // staging: rows of 256 bytes, 16-byte piece c of row r at piece c ^ (r & 15) (a thread reads back its own row)
+        const uint32_t off = (uint32_t)(r * 256 + ((c ^ (r & 15)) << 4));
         *reinterpret_cast<uint4*>(bp + oQhi + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
         *reinterpret_cast<uint4*>(bp + oQlo + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    // each term into tensor memory as the A operand of the score products: row = lane, elements 2 j and 2 j + 1 of the
+    // row in column j. Group 0 writes the high-order term, group 1 the low-order one.
+    {
+      const uint8_t* src = bp + (gi == 0 ? oQhi : oQlo) + ql * 256;
+      const uint32_t tq = tmem_base + TC_TM_Q + lane_addr + (uint32_t)(gi * 64);
+#pragma unroll
+      for (int c = 0; c < 16; c += 2) {
+        const uint4 a0 = *reinterpret_cast<const uint4*>(src + (((c) ^ (ql & 15)) << 4));
+        const uint4 a1 = *reinterpret_cast<const uint4*>(src + (((c + 1) ^ (ql & 15)) << 4));
+        const uint32_t w8[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        tc_st8(tq + (uint32_t)(c * 4), w8);
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
     mbar_arrive(qfull_bar);
 
     // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per key block
@@ -274,7 +313,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
     }
     float m_ref = -INFINITY, l_run = 0.f;
-    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * 128);      // S_hi (later P); S_lo 64 columns on
+    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * 64);       // S (64 columns), then P over it
     const uint32_t tOg = tmem_base + TC_TM_O + lane_addr + (uint32_t)(gi * TC_DH);
     bool ok = true;
     for (int b = gi; b < n_blocks && ok; b += 2) {
@@ -282,16 +321,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       if (!mbar_wait(sfull_bar(gi), k & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       float s[TC_KB];
-      if (warp_live) {
-#pragma unroll
-        for (int c = 0; c < TC_KB; c += 16) {
-          float t2[16];
-          tc_ld16(tSg + (uint32_t)c, s + c);
-          tc_ld16(tSg + 64u + (uint32_t)c, t2);
-#pragma unroll
-          for (int e = 0; e < 16; ++e) s[c + e] += t2[e];
-        }
-      }
+      if (warp_live) tc_ld64(tSg, s);                   // one load of the row's 64 scores, one wait
       const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
       if (n_in < TC_KB) {
         // A ragged last block: positions beyond the range carry whatever the cache holds there. Their probabilities are
