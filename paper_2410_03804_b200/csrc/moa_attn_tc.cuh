@@ -4,30 +4,28 @@
 // context (tens of thousands of cached positions per kv head) it is bound by that instruction stream, not by HBM.
 // Here one CTA per (sequence, kv head, key range) keeps all queries that share the kv head -- (rows of the
 // sequence) x (query heads of the group), at most 128 -- as the M = 128 operand and streams the cache through a TMA
-// ring of 64-position blocks:
-//   warp 0      TMA producer: K block [64, 128] and V block [64, 128] per stage (128-byte swizzle), five stages
-//   warp 1      one thread issues tcgen05.mma:  S_hi = Q_hi K^T, S_lo = Q_lo K^T  (A = Q in shared memory, B = K, both
-//                                                                          K-major; two fp32 accumulators in TMEM)
-//                                               O += P_hi V + P_lo V      (A = P in TMEM, B = V as it lies in the
-//                                                                          cache: MN-major)
-//               Products that accumulate into the same TMEM tile run one after the other at the tensor pipe's latency
-//               (about 90 cycles each with these small N), and that chain, not the math or the memory, sets a block's
-//               pace. So the two query terms go to two accumulators (two chains of 8 that interleave instead of one
-//               of 16; the softmax thread adds them).
-//   warps 2..9  softmax, two groups of four warps that take alternate blocks: a thread owns one query row (TMEM lane)
-//               of its group's blocks: reads its 64 scores, keeps the running maximum and sum in the log2 domain, and
-//               writes the probabilities as two bf16 terms over the scores it has just read (P_hi | P_lo take the 64
-//               columns S_hi took). Each group has its own score / probability buffers and its own OUTPUT
-//               ACCUMULATOR, so the groups are independent partial softmaxes (over the even and the odd blocks) that
-//               never wait for one another; they are merged once, at the end.
-// Tensor memory (512 columns): S_hi (then P) of group g at 128 g, S_lo at 128 g + 64, O of group g at 256 + 128 g. An output accumulator is rescaled only when a row's maximum has grown by more than 2^8 since its last
-// rescale (probabilities then stay below 256), so the rescale -- a TMEM load, multiply, store of the row -- happens a
-// few times per range, not per block. A block's softmax is a chain of short dependent steps, so one group per CTA
-// would set the pace; two groups overlap their chains.
+// ring of 128-position blocks:
+//   warp 0      TMA producer: K block [128, 128] and V block [128, 128] per stage (128-byte swizzle), three stages
+//   warp 1      one thread issues tcgen05.mma:  S = Q_hi K^T + Q_lo K^T   (A = Q in TENSOR MEMORY, B = K, K-major,
+//                                                                          N = 128: one chain of 16 products)
+//                                               O += P_hi V + P_lo V      (A = P in tensor memory, B = V as it lies in
+//                                                                          the cache: MN-major)
+//               The tensor pipe sets the pace: a product costs about 50 cycles at N = 64 and 64 at N = 128 whatever
+//               its operands' source, so blocks of 128 positions halve the cost of the scores per position.
+//   warps 2..9  softmax: two threads per query row (tensor-memory lane), one per half of the block's 128 scores. A
+//               thread reads its 64 scores, the two exchange their maxima through shared memory, keep the running
+//               reference maximum and their part of the sum in the log2 domain, and write the probabilities as two
+//               bf16 terms over the scores (P_hi takes the first 64 columns of the score buffer, P_lo the other 64).
+// Tensor memory (512 columns): Q_hi | Q_lo at 0 (64 columns each: two bf16 per column), two score / probability buffers
+// at 128 and 256 (the scores of block b + 1 are formed while the softmax of block b runs), the output accumulator at
+// 384. The output accumulator is rescaled only when a row's maximum has grown by more than 2^8 since its last rescale
+// (probabilities then stay below 256), so the rescale -- a TMEM load, multiply, store of the row -- happens a few
+// times per range, not per block.
 // Each CTA leaves (max, sum, unnormalised output) per query for attn_combine_kernel, in the layout of the split-KV
-// kernel. A self-attention's tree segment (the sequence's drafted slots, masked per row by its ancestor list) is one
-// more CTA of the same grid: same pipeline over the tree's keys / values, with the row's slot bitmap applied to the
-// scores. Queries arrive in fp32 and enter as two bf16 terms, as in the split-KV kernel.
+// kernel (or the normalised rows when the range is the attention's only part). A self-attention's tree segment (the
+// sequence's drafted slots, masked per row by its ancestor list) is one more CTA of the same grid: same pipeline over
+// the tree's keys / values, with the row's slot bitmap applied to the scores. Queries arrive in fp32 and enter as two
+// bf16 terms, as in the split-KV kernel.
 // Every mbarrier wait is bounded; on expiry the CTA raises the abort flag, drains, frees TMEM and reports
 // DEV_ERR_TIMEOUT through the status word.
 #pragma once
@@ -36,15 +34,16 @@
 
 namespace moa {
 
-constexpr int TC_KB = 64;                 // cache positions per block
+constexpr int TC_KB = 128;                // cache positions per block
 constexpr int TC_DH = 128;
-constexpr int TC_STAGES = 5;
-constexpr int TC_THREADS = 320;            // TMA warp, MMA warp, two softmax groups of four warps
-constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-column chunks of [64 rows x 128 B]
-constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // one query term: two 64-column chunks of [128 rows x 128 B]
-constexpr int TC_SMEM_BYTES = 2 * TC_Q_BYTES + TC_STAGES * TC_STAGE_BYTES + 1024 + 256;
-constexpr uint32_t TC_TM_Q = 0, TC_TM_S = 128, TC_TM_O = 256;   // tensor-memory columns (see above)
+constexpr int TC_STAGES = 3;
+constexpr int TC_THREADS = 320;            // TMA warp, MMA warp, eight softmax warps (two per tensor-memory lane quadrant)
+constexpr int TC_KV_BYTES = TC_KB * TC_DH * 2;        // K (or V) block: two 64-column chunks of [128 rows x 128 B]
+constexpr int TC_STAGE_BYTES = 2 * TC_KV_BYTES;       // 64 KB
+constexpr int TC_Q_BYTES = 128 * TC_DH * 2;           // staging of one query term; the two terms lie over the last stage
+constexpr int TC_X_BYTES = 2 * 2 * 128 * 4;           // row maxima exchanged between the two threads of a row
+constexpr int TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + TC_X_BYTES + 1024 + 256;
+constexpr uint32_t TC_TM_Q = 0, TC_TM_S = 128, TC_TM_O = 384;   // tensor-memory columns (see above)
 constexpr float TC_RESCALE_LOG2 = 8.f;
 
 struct AttnTcParams {
@@ -111,20 +110,36 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
       : "memory");
 }
 
+// Barrier 1 over the 256 softmax threads that also ORs a flag: every thread gets the same answer, so a failed wait
+// anywhere takes all of them out of their loop at the same barrier (nobody is left waiting at the next one).
+__device__ __forceinline__ bool tc_bar_any(bool mine) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, 256, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(any)
+      : "r"((uint32_t)(mine ? 1u : 0u))
+      : "memory");
+  return any != 0u;
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams P) {
   extern __shared__ uint8_t tc_smem_raw[];
   const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = tc_smem_raw + (base - smem_u32(tc_smem_raw));
-  constexpr uint32_t oQhi = 0, oQlo = TC_Q_BYTES, oKV = 2 * TC_Q_BYTES, oBar = oKV + TC_STAGES * TC_STAGE_BYTES;
+  constexpr uint32_t oKV = 0, oQhi = (TC_STAGES - 1) * TC_STAGE_BYTES, oQlo = oQhi + TC_Q_BYTES;
+  constexpr uint32_t oX = TC_STAGES * TC_STAGE_BYTES, oBar = oX + TC_X_BYTES;
   const uint32_t bar0 = base + oBar;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
   auto sfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + i); };
-  auto pfull_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 4 + j); };
-  auto pempty_bar = [&](int j) { return bar0 + 8u * (2 * TC_STAGES + 6 + j); };
-  const uint32_t qfull_bar = bar0 + 8u * (2 * TC_STAGES + 8), ofull_bar = qfull_bar + 8u;
-  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (2 * TC_STAGES + 10));
+  auto pfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + 2 + i); };
+  const uint32_t pempty_bar = bar0 + 8u * (2 * TC_STAGES + 4), qfull_bar = pempty_bar + 8u, ofull_bar = qfull_bar + 8u;
+  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (2 * TC_STAGES + 7));
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+  float* xm = reinterpret_cast<float*>(bp + oX);       // [buffer][half][row]
 
   const AttnParams& A = P.a;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -134,10 +149,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(sfull_bar(i), 1);
-      mbar_init(pfull_bar(i), 128); mbar_init(pempty_bar(i), 1);
-    }
+    for (int i = 0; i < 2; ++i) { mbar_init(sfull_bar(i), 1); mbar_init(pfull_bar(i), 256); }
+    mbar_init(pempty_bar, 1);
     mbar_init(qfull_bar, 256);
     mbar_init(ofull_bar, 1);
     *abort_flag = 0;
@@ -154,7 +167,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   const uint32_t tmem_base = *tmem_slot;
 
   // The queries and the tree slots come from the kernels just before this one. A cache segment that was complete
-  // before the chain began needs no wait: its producer warp sends the first ring of blocks at once and waits after.
+  // before the chain began needs no wait: its producer warp sends its first blocks at once and waits after.
   const bool tree_part = part >= A.n_split;          // the grid's last CTA along z when the attention has a tree segment
   const bool early = P.early_cache != 0 && !tree_part;
   if (!(early && warp == 0)) pdl_wait(KID_ATTN);
@@ -177,9 +190,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     if (lane == 0) {
       const int x0 = g * TC_DH;
       bool waited = !early;
-      for (int b = 0; b < n_blocks; ++b) {
-        if (!waited && b >= TC_STAGES) { pdl_wait(KID_ATTN); waited = true; }
+      bool ok = true;
+      for (int b = 0; b < n_blocks && ok; ++b) {
         const int st = b % TC_STAGES;
+        if (st == TC_STAGES - 1 && b < TC_STAGES) {
+          // the last stage holds the query staging until the queries are in tensor memory
+          if (!waited) { pdl_wait(KID_ATTN); waited = true; }
+          if (!mbar_wait(qfull_bar, 0u, abort_flag)) break;
+        }
         const uint32_t k = (uint32_t)(b / TC_STAGES);
         if (!mbar_wait(empty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
         mbar_expect_tx(full_bar(st), TC_STAGE_BYTES);
@@ -201,16 +219,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       constexpr uint32_t IDESC_O = umma_idesc_bf16_bmn(128, TC_DH);
       bool ok = mbar_wait(qfull_bar, 0u, abort_flag);
       tc_fence_after();
-      // S of block b into its group's score accumulator: both query terms, A from tensor memory (the shared-memory
-      // operand path then carries the keys only), one chain of 16 products. The accumulator held the group's
-      // probabilities of block b - 2, whose P V product has been issued before (program order): the tensor pipe runs
-      // in issue order.
+      // S of block b into score buffer b & 1: both query terms, A from tensor memory, one chain of 16 products. The
+      // buffer held the probabilities of block b - 2, whose P V product has been issued before (program order): the
+      // tensor pipe runs in issue order.
       auto issue_s = [&](int b) -> bool {
         const int st = b % TC_STAGES, i = b & 1;
         if (!mbar_wait(full_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint64_t kd = umma_desc_sw128(base + oKV + st * TC_STAGE_BYTES);
-        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * 64);
+        const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);
 #pragma unroll
         for (int ks = 0; ks < TC_DH / 16; ++ks) {          // k-steps 0..3 in the first 64-column chunk of K, 4..7 in the second
           const uint64_t ko = (uint64_t)((ks >> 2) * (TC_KV_BYTES / 2 / 16) + 2 * (ks & 3));
@@ -223,27 +240,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       if (ok) ok = issue_s(0);
       for (int b = 0; b < n_blocks && ok; ++b) {
         if (b + 1 < n_blocks && !issue_s(b + 1)) { ok = false; break; }
-        const int j = b & 1;
-        if (!mbar_wait(pfull_bar(j), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
+        const int i = b & 1;
+        if (!mbar_wait(pfull_bar(i), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(j * 64);          // P_hi in its first 32 columns, P_lo in the next 32
-        const uint32_t d = tmem_base + TC_TM_O + (uint32_t)(j * TC_DH);
+        const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);       // P_hi in its first 64 columns, P_lo in the next 64
+        const uint32_t d = tmem_base + TC_TM_O;
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16_ta(d, pt + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, (b > 1 || ks > 0) ? 1u : 0u);
+          tc_mma_bf16_ta(d, pt + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, (b > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
         for (int ks = 0; ks < TC_KB / 16; ++ks)
-          tc_mma_bf16_ta(d, pt + 32u + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
-        tc_commit(pempty_bar(j));                 // the group's O is at rest once this completes
+          tc_mma_bf16_ta(d, pt + 64u + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
+        tc_commit(pempty_bar);                    // O is at rest once this completes
         tc_commit(empty_bar(b % TC_STAGES));      // the stage's K and V are done with
       }
       if (ok) tc_commit(ofull_bar);
     }
   } else {
-    // ------------------------------ softmax: group gi takes the blocks b with b % 2 == gi ------------------------------
+    // ------------------------------ softmax: two threads per query row, one per half of a block's 128 scores ------------------------------
     const int wi = warp - 2;                           // 0..7
-    const int gi = wi >> 2;                            // group: its S/P buffer, O accumulator and barriers have index gi
+    const int half = wi >> 2;                          // which 64 scores of a block (and which 64 output columns at the end)
     const int quad = warp & 3;                         // TMEM lane quadrant of this warp
     const int ql = quad * 32 + lane;                   // query row = TMEM lane
     const int st_i = threadIdx.x - 64;                 // 0..255 among the softmax threads
@@ -252,7 +269,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     const int row = seq * A.rows_per_seq + (valid ? ql / A.group : 0);
     const int head = g * A.group + (valid ? ql % A.group : 0);
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    // ---- queries -> two bf16 terms in shared memory (rows beyond Qn are zero) ----
+    // ---- queries -> two bf16 terms, staged in shared memory (rows beyond Qn are zero) ----
     for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 256) {
       float x[4][8];
       bool in[4];
@@ -287,10 +304,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
     // each term into tensor memory as the A operand of the score products: row = lane, elements 2 j and 2 j + 1 of the
-    // row in column j. Group 0 writes the high-order term, group 1 the low-order one.
+    // row in column j. The threads of half 0 write the high-order term, those of half 1 the low-order one.
     {
-      const uint8_t* src = bp + (gi == 0 ? oQhi : oQlo) + ql * 256;
-      const uint32_t tq = tmem_base + TC_TM_Q + lane_addr + (uint32_t)(gi * 64);
+      const uint8_t* src = bp + (half == 0 ? oQhi : oQlo) + ql * 256;
+      const uint32_t tq = tmem_base + TC_TM_Q + lane_addr + (uint32_t)(half * 64);
 #pragma unroll
       for (int c = 0; c < 16; c += 2) {
         const uint4 a0 = *reinterpret_cast<const uint4*>(src + (((c) ^ (ql & 15)) << 4));
@@ -300,10 +317,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the staging bytes become a ring stage
     tc_fence_before();
     mbar_arrive(qfull_bar);
 
-    // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per key block
+    // tree segment: bit per slot this row may see (its ancestors and itself), 64 slots per word
     unsigned long long allow[4] = {0ull, 0ull, 0ull, 0ull};
     if (tree_part && valid) {
       for (int i = 0; i < A.nB; ++i) {
@@ -313,50 +331,57 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       }
     }
     float m_ref = -INFINITY, l_run = 0.f;
-    const uint32_t tSg = tmem_base + TC_TM_S + lane_addr + (uint32_t)(gi * 64);       // S (64 columns), then P over it
-    const uint32_t tOg = tmem_base + TC_TM_O + lane_addr + (uint32_t)(gi * TC_DH);
-    bool ok = true;
-    for (int b = gi; b < n_blocks && ok; b += 2) {
-      const uint32_t k = (uint32_t)(b >> 1);            // how many blocks this group has done
-      if (!mbar_wait(sfull_bar(gi), k & 1u, abort_flag)) { ok = false; break; }
+    const uint32_t tOh = tmem_base + TC_TM_O + lane_addr + (uint32_t)(half * 64);     // this thread's half of the output columns
+    bool ok = true;          // false once any softmax thread has seen a wait fail; changes only at a barrier, for all at once
+    bool fail = false;       // this thread's own failed waits since the last barrier
+    for (int b = 0; b < n_blocks; ++b) {
+      const int i = b & 1;
+      if (!mbar_wait(sfull_bar(i), (uint32_t)(b >> 1) & 1u, abort_flag)) fail = true;
       tc_fence_after();
-      float s[TC_KB];
-      if (warp_live) tc_ld64(tSg, s);                   // one load of the row's 64 scores, one wait
-      const int n_in = min(TC_KB, k_end - (k_begin + b * TC_KB));       // positions of this block inside the range
-      if (n_in < TC_KB) {
+      const uint32_t tS = tmem_base + TC_TM_S + lane_addr + (uint32_t)(i * TC_KB);
+      float s[64];
+      if (warp_live) tc_ld64(tS + (uint32_t)(half * 64), s);        // this thread's 64 scores: one load, one wait
+      const int n_blk = min(TC_KB, k_end - (k_begin + b * TC_KB));      // positions of this block inside the range
+      const int n_in = max(0, min(64, n_blk - half * 64));              // of them in this thread's half
+      if (n_blk < TC_KB) {
         // A ragged last block: positions beyond the range carry whatever the cache holds there. Their probabilities are
         // exactly zero, but zero times a non-finite stale value is not, so those V rows are cleared in shared memory
         // (the block has landed: its scores are complete).
         uint8_t* v = bp + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        for (int j = st_i & 127; j < (TC_KB - n_in) * 16; j += 128) {
-          const int r = n_in + (j >> 4), c16 = j & 15;                   // row, 16-byte piece of its 256 bytes
+        for (int j = st_i; j < (TC_KB - n_blk) * 16; j += 256) {
+          const int r = n_blk + (j >> 4), c16 = j & 15;                  // row, 16-byte piece of its 256 bytes
           *reinterpret_cast<uint4*>(v + (c16 >> 3) * (TC_KV_BYTES / 2) + r * 128 + (c16 & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       }
-      // block maximum of the raw scores (the scale is positive and goes into the exponent's multiply-add)
+      // maximum of this thread's raw scores (the scale is positive and goes into the exponent's multiply-add)
       float mx = -INFINITY;
       if (warp_live) {
         if (tree_part) {                                   // the row sees its ancestors' slots and its own only
-          const unsigned long long word = allow[b & 3];
+          const unsigned long long word = allow[(2 * b + half) & 3];
 #pragma unroll
-          for (int c = 0; c < TC_KB; ++c) {
+          for (int c = 0; c < 64; ++c) {
             s[c] = (c < n_in && ((word >> c) & 1ull)) ? s[c] : -INFINITY;
             mx = fmaxf(mx, s[c]);
           }
-        } else if (n_in == TC_KB) {
+        } else if (n_in == 64) {
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four chains instead of one
 #pragma unroll
-          for (int c = 0; c < TC_KB; ++c) m4[c & 3] = fmaxf(m4[c & 3], s[c]);
+          for (int c = 0; c < 64; ++c) m4[c & 3] = fmaxf(m4[c & 3], s[c]);
           mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         } else {
 #pragma unroll
-          for (int c = 0; c < TC_KB; ++c) {
+          for (int c = 0; c < 64; ++c) {
             s[c] = c < n_in ? s[c] : -INFINITY;
             mx = fmaxf(mx, s[c]);
           }
         }
       }
+      // the row's two threads exchange their maxima (buffers alternate, so one barrier per block is enough); behind the
+      // barrier both have their scores in registers, and the probabilities may overwrite either half of the buffer
+      xm[(i * 2 + half) * 128 + ql] = mx;
+      if (tc_bar_any(fail || *abort_flag != 0)) { ok = false; break; }
+      mx = fmaxf(mx, xm[(i * 2 + (half ^ 1)) * 128 + ql]);
       const float m_blk = mx * A.scale_log2;
       float f = 1.f;
       if (warp_live) {
@@ -368,25 +393,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           l_run *= f;
         }
       }
-      if (k > 0 && warp_live && __any_sync(0xffffffffu, f != 1.f)) {
-        // rare: a row's accumulator moves to a new reference; the group's previous product must have left the tensor cores
-        if (!mbar_wait(pempty_bar(gi), (k & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+      if (b > 0 && warp_live && __any_sync(0xffffffffu, f != 1.f)) {
+        // rare: a row's accumulator moves to a new reference; the previous product must have left the tensor cores
+        if (!mbar_wait(pempty_bar, ((uint32_t)b & 1u) ^ 1u, abort_flag)) fail = true;   // seen by all at the next barrier
         tc_fence_after();
 #pragma unroll 1
-        for (int c = 0; c < TC_DH; c += 16) {
+        for (int c = 0; c < 64 && !fail; c += 16) {
           float o[16];
-          tc_ld16(tOg + (uint32_t)c, o);
+          tc_ld16(tOh + (uint32_t)c, o);
 #pragma unroll
           for (int e = 0; e < 16; ++e) o[e] *= f;
-          tc_st16(tOg + (uint32_t)c, o);
+          tc_st16(tOh + (uint32_t)c, o);
         }
       }
       if (warp_live) {
-        // probabilities as two bf16 terms over the scores just read: P_hi in columns 0..31 of the buffer, P_lo in 32..63
+        // probabilities as two bf16 terms over the scores: P_hi in columns 0..63 of the buffer (two positions per column),
+        // P_lo in 64..127; this thread's 64 positions take 32 columns of each
         const float msub = m_ref == -INFINITY ? 0.f : m_ref;
         float rs[2] = {0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < TC_KB; c += 16) {
+        for (int c = 0; c < 64; c += 16) {
           uint32_t hi[8], lo[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
@@ -397,97 +423,68 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
             hi[e] = h;
             lo[e] = pack_bf16(p0 - __uint_as_float(h << 16), p1 - __uint_as_float(h & 0xffff0000u));
           }
-          tc_st8(tSg + (uint32_t)(c / 2), hi);
-          tc_st8(tSg + 32u + (uint32_t)(c / 2), lo);
+          tc_st8(tS + (uint32_t)(half * 32 + c / 2), hi);
+          tc_st8(tS + 64u + (uint32_t)(half * 32 + c / 2), lo);
         }
         l_run += rs[0] + rs[1];
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
       tc_fence_before();
-      mbar_arrive(pfull_bar(gi));
+      mbar_arrive(pfull_bar(i));
     }
-    // ---- merge of the CTA's two partial softmaxes (one per group), then the range's result: (max, sum,
-    //      unnormalised output) per query, or the normalised rows when this range is the attention's only part ----
-    if (ok && n_blocks > 0) ok = mbar_wait(ofull_bar, 0u, abort_flag);
+    // ---- the range's result: (max, sum, unnormalised output) per query, or the normalised rows when this range is the
+    //      attention's only part; each of the row's two threads takes 64 output columns ----
+    if (ok && n_blocks > 0 && !mbar_wait(ofull_bar, 0u, abort_flag)) fail = true;
     tc_fence_after();
-    if (!ok) *abort_flag = 1;
-    // the key / value ring is free now: [sub-part][query][2] (max, sum), then two buffers of [sub-part][query][16] output columns
-    constexpr int NSP = 2, RPR = 128;
-    const int qi = ql;
-    float* ml_x = reinterpret_cast<float*>(bp + oKV);
-    float* o_x = ml_x + NSP * RPR * 2;
-    const int sp = gi;
-    const bool has_blocks = gi < n_blocks;                 // this group saw at least one block
-    ml_x[(sp * RPR + qi) * 2 + 0] = has_blocks ? m_ref : -INFINITY;
-    ml_x[(sp * RPR + qi) * 2 + 1] = has_blocks ? l_run : 0.f;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    const bool dead = __shfl_sync(0xffffffffu, *abort_flag, 0) != 0;     // warp-uniform: the TMEM loads below are warp-wide
-    float M = -INFINITY;
-#pragma unroll
-    for (int t = 0; t < NSP; ++t) M = fmaxf(M, ml_x[(t * RPR + qi) * 2]);
-    float L = 0.f;
-#pragma unroll
-    for (int t = 0; t < NSP; ++t) {
-      const float mt = ml_x[(t * RPR + qi) * 2];
-      L += mt == -INFINITY ? 0.f : ex2_approx(mt - M) * ml_x[(t * RPR + qi) * 2 + 1];
-    }
-    const float w_own = (!has_blocks || m_ref == -INFINITY) ? 0.f : ex2_approx(m_ref - M);
+    if (!ok || fail) *abort_flag = 1;
+    (void)tc_bar_any(false);                               // every exchange read of the loop is behind us
+    xm[half * 128 + ql] = l_run;
+    const bool dead = tc_bar_any(!ok || fail || *abort_flag != 0);       // the same for all: the TMEM loads below are warp-wide
+    const float L = l_run + xm[(half ^ 1) * 128 + ql];
+    const bool seen = n_blocks > 0 && m_ref != -INFINITY;
     const size_t pidx = ((size_t)row * A.hq + head) * A.n_parts + part;
-    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const float inv = (seen && L > 0.f) ? 1.f / L : 0.f;
 #pragma unroll 1
-    for (int c = 0; c < TC_DH; c += 16) {
+    for (int c = 0; c < 64; c += 16) {
       float o[16];
-      if (has_blocks && warp_live && !dead) {
-        tc_ld16(tOg + (uint32_t)c, o);
+      if (n_blocks > 0 && warp_live && !dead) {
+        tc_ld16(tOh + (uint32_t)c, o);
       } else {
 #pragma unroll
         for (int e = 0; e < 16; ++e) o[e] = 0.f;
       }
-      float* mine = o_x + ((size_t)((c >> 4) & 1) * NSP * RPR + (size_t)sp * RPR + qi) * 16;
-#pragma unroll
-      for (int e = 0; e < 16; e += 4)
-        *reinterpret_cast<float4*>(mine + e) = w_own == 0.f ? make_float4(0.f, 0.f, 0.f, 0.f)
-                                                            : make_float4(o[e] * w_own, o[e + 1] * w_own, o[e + 2] * w_own, o[e + 3] * w_own);
-      asm volatile("bar.sync 1, 256;" ::: "memory");       // (two buffers: the next chunk's writes do not meet this chunk's reads)
-      if (sp == 0 && valid) {
+      if (!valid) continue;
+      if (!seen) {
 #pragma unroll
         for (int e = 0; e < 16; ++e) o[e] = 0.f;
+      }
+      const int col = half * 64 + c;
+      if (A.n_parts == 1) {
+        bf16* dst = A.out + ((size_t)row * A.hq + head) * TC_DH + col;
+        bf16* dlo = A.out + ((size_t)(A.out_lo + row) * A.hq + head) * TC_DH + col;
+        uint32_t hi[8], lo[8];
 #pragma unroll
-        for (int t = 0; t < NSP; ++t) {                     // sub-parts added in a fixed order
-          const float* src = o_x + ((size_t)((c >> 4) & 1) * NSP * RPR + (size_t)t * RPR + qi) * 16;
-#pragma unroll
-          for (int e = 0; e < 16; e += 4) {
-            const float4 v4 = *reinterpret_cast<const float4*>(src + e);
-            o[e] += v4.x; o[e + 1] += v4.y; o[e + 2] += v4.z; o[e + 3] += v4.w;
-          }
+        for (int e = 0; e < 8; ++e) {
+          const float a0 = o[2 * e] * inv, a1 = o[2 * e + 1] * inv;
+          const bf16 h0 = __float2bfloat16_rn(a0), h1 = __float2bfloat16_rn(a1);
+          hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
+          lo[e] = pack_bf16(a0 - __bfloat162float(h0), a1 - __bfloat162float(h1));
         }
-        if (A.n_parts == 1) {
-          bf16* dst = A.out + ((size_t)row * A.hq + head) * TC_DH + c;
-          bf16* dlo = A.out + ((size_t)(A.out_lo + row) * A.hq + head) * TC_DH + c;
-          uint32_t hi[8], lo[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const float a0 = o[2 * e] * inv, a1 = o[2 * e + 1] * inv;
-            const bf16 h0 = __float2bfloat16_rn(a0), h1 = __float2bfloat16_rn(a1);
-            hi[e] = pack_bf16(__bfloat162float(h0), __bfloat162float(h1));
-            lo[e] = pack_bf16(a0 - __bfloat162float(h0), a1 - __bfloat162float(h1));
-          }
-          *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(dst + 8) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-          if (A.out_lo > 0) {
-            *reinterpret_cast<uint4*>(dlo) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-            *reinterpret_cast<uint4*>(dlo + 8) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-          }
-        } else {
-          float* dst = A.part_o + pidx * TC_DH + c;
-#pragma unroll
-          for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(dst + 8) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        if (A.out_lo > 0) {
+          *reinterpret_cast<uint4*>(dlo) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(dlo + 8) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
         }
+      } else {
+        float* dst = A.part_o + pidx * TC_DH + col;
+#pragma unroll
+        for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
       }
     }
-    if (sp == 0 && valid && A.n_parts > 1) {
-      A.part_ml[pidx * 2 + 0] = M;               // log2 domain, as attn_combine_kernel expects
-      A.part_ml[pidx * 2 + 1] = L;
+    if (half == 0 && valid && A.n_parts > 1) {
+      A.part_ml[pidx * 2 + 0] = seen ? m_ref : -INFINITY;      // log2 domain, as attn_combine_kernel expects
+      A.part_ml[pidx * 2 + 1] = seen ? L : 0.f;
     }
   }
 
