@@ -129,15 +129,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   extern __shared__ uint8_t tc_smem_raw[];
   const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = tc_smem_raw + (base - smem_u32(tc_smem_raw));
-  constexpr uint32_t oKV = 0, oQhi = (TC_STAGES - 1) * TC_STAGE_BYTES, oQlo = oQhi + TC_Q_BYTES;
+  // Key and value blocks have rings of their own (a key block is free again once its scores are formed, a block time
+  // before its value block): K0 K1 V0 V1 K2 V2. The last pair doubles as the query staging area at start-up.
+  auto k_off = [&](int st) { return (uint32_t)(st < TC_STAGES - 1 ? st * TC_KV_BYTES : 2 * (TC_STAGES - 1) * TC_KV_BYTES); };
+  auto v_off = [&](int st) { return (uint32_t)(st < TC_STAGES - 1 ? (TC_STAGES - 1 + st) * TC_KV_BYTES : (2 * (TC_STAGES - 1) + 1) * TC_KV_BYTES); };
+  constexpr uint32_t oQhi = 2 * (TC_STAGES - 1) * TC_KV_BYTES, oQlo = oQhi + TC_Q_BYTES;
   constexpr uint32_t oX = TC_STAGES * TC_STAGE_BYTES, oBar = oX + TC_X_BYTES;
   const uint32_t bar0 = base + oBar;
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
-  auto sfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + i); };
-  auto pfull_bar = [&](int i) { return bar0 + 8u * (2 * TC_STAGES + 2 + i); };
-  const uint32_t pempty_bar = bar0 + 8u * (2 * TC_STAGES + 4), qfull_bar = pempty_bar + 8u, ofull_bar = qfull_bar + 8u;
-  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (2 * TC_STAGES + 7));
+  auto kfull_bar = [&](int s) { return bar0 + 8u * s; };
+  auto kempty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
+  auto vfull_bar = [&](int s) { return bar0 + 8u * (2 * TC_STAGES + s); };
+  auto vempty_bar = [&](int s) { return bar0 + 8u * (3 * TC_STAGES + s); };
+  auto sfull_bar = [&](int i) { return bar0 + 8u * (4 * TC_STAGES + i); };
+  auto pfull_bar = [&](int i) { return bar0 + 8u * (4 * TC_STAGES + 2 + i); };
+  const uint32_t pempty_bar = bar0 + 8u * (4 * TC_STAGES + 4), qfull_bar = pempty_bar + 8u, ofull_bar = qfull_bar + 8u;
+  uint32_t* tmem_slot = (uint32_t*)(bp + oBar + 8 * (4 * TC_STAGES + 7));
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   float* xm = reinterpret_cast<float*>(bp + oX);       // [buffer][half][row]
 
@@ -148,7 +154,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
   pdl_trigger();
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < TC_STAGES; ++s) {
+      mbar_init(kfull_bar(s), 1); mbar_init(kempty_bar(s), 1);
+      mbar_init(vfull_bar(s), 1); mbar_init(vempty_bar(s), 1);
+    }
     for (int i = 0; i < 2; ++i) { mbar_init(sfull_bar(i), 1); mbar_init(pfull_bar(i), 256); }
     mbar_init(pempty_bar, 1);
     mbar_init(qfull_bar, 256);
@@ -199,16 +208,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           if (!mbar_wait(qfull_bar, 0u, abort_flag)) break;
         }
         const uint32_t k = (uint32_t)(b / TC_STAGES);
-        if (!mbar_wait(empty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
-        mbar_expect_tx(full_bar(st), TC_STAGE_BYTES);
-        const uint32_t dst = base + oKV + st * TC_STAGE_BYTES;
         const int y = seq * (tree_part ? A.capB : A.capA) + k_begin + b * TC_KB;
         const CUtensorMap* tk = tree_part ? &P.tmKB : &P.tmK;
         const CUtensorMap* tv = tree_part ? &P.tmVB : &P.tmV;
-        tma_load_2d(dst, tk, x0, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES / 2, tk, x0 + 64, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES, tv, x0, y, full_bar(st));
-        tma_load_2d(dst + TC_KV_BYTES + TC_KV_BYTES / 2, tv, x0 + 64, y, full_bar(st));
+        if (!mbar_wait(kempty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
+        mbar_expect_tx(kfull_bar(st), TC_KV_BYTES);
+        tma_load_2d(base + k_off(st), tk, x0, y, kfull_bar(st));
+        tma_load_2d(base + k_off(st) + TC_KV_BYTES / 2, tk, x0 + 64, y, kfull_bar(st));
+        if (!mbar_wait(vempty_bar(st), (k & 1u) ^ 1u, abort_flag)) break;
+        mbar_expect_tx(vfull_bar(st), TC_KV_BYTES);
+        tma_load_2d(base + v_off(st), tv, x0, y, vfull_bar(st));
+        tma_load_2d(base + v_off(st) + TC_KV_BYTES / 2, tv, x0 + 64, y, vfull_bar(st));
       }
       if (!waited) pdl_wait(KID_ATTN);
     }
@@ -224,9 +234,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       // tensor pipe runs in issue order.
       auto issue_s = [&](int b) -> bool {
         const int st = b % TC_STAGES, i = b & 1;
-        if (!mbar_wait(full_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
+        if (!mbar_wait(kfull_bar(st), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) return false;
         tc_fence_after();
-        const uint64_t kd = umma_desc_sw128(base + oKV + st * TC_STAGE_BYTES);
+        const uint64_t kd = umma_desc_sw128(base + k_off(st));
         const uint32_t d = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);
 #pragma unroll
         for (int ks = 0; ks < TC_DH / 16; ++ks) {          // k-steps 0..3 in the first 64-column chunk of K, 4..7 in the second
@@ -235,6 +245,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
           tc_mma_bf16_ta(d, tmem_base + TC_TM_Q + 64u + (uint32_t)(ks * 8), kd + ko, IDESC_S, 1u);
         }
         tc_commit(sfull_bar(i));
+        tc_commit(kempty_bar(st));                // the keys are done with once the scores are formed
         return true;
       };
       if (ok) ok = issue_s(0);
@@ -242,8 +253,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         if (b + 1 < n_blocks && !issue_s(b + 1)) { ok = false; break; }
         const int i = b & 1;
         if (!mbar_wait(pfull_bar(i), (uint32_t)(b >> 1) & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(vfull_bar(b % TC_STAGES), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t vaddr = base + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t vaddr = base + v_off(b % TC_STAGES);
         const uint32_t pt = tmem_base + TC_TM_S + (uint32_t)(i * TC_KB);       // P_hi in its first 64 columns, P_lo in the next 64
         const uint32_t d = tmem_base + TC_TM_O;
 #pragma unroll
@@ -253,7 +265,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
         for (int ks = 0; ks < TC_KB / 16; ++ks)
           tc_mma_bf16_ta(d, pt + 64u + (uint32_t)(ks * 8), umma_desc_mn_sw128(vaddr + ks * 2048, TC_KV_BYTES / 2), IDESC_O, 1u);
         tc_commit(pempty_bar);                    // O is at rest once this completes
-        tc_commit(empty_bar(b % TC_STAGES));      // the stage's K and V are done with
+        tc_commit(vempty_bar(b % TC_STAGES));     // the values are done with
       }
       if (ok) tc_commit(ofull_bar);
     }
@@ -270,22 +282,49 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
     const int head = g * A.group + (valid ? ql % A.group : 0);
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     // ---- queries -> two bf16 terms, staged in shared memory (rows beyond Qn are zero) ----
+    // Every thread takes eight 8-element pieces (piece i = row i / 16, column piece i % 16), four at a time. The loads
+    // of a batch are unconditional (rows beyond Qn read the last real row and are discarded) and go out together, two
+    // split-K planes at a time, so a batch costs one memory round trip per two planes instead of one per piece.
     for (int i0 = st_i; i0 < 128 * 16; i0 += 4 * 256) {
       float x[4][8];
+      const float* src[4];
       bool in[4];
+      const bool batch_live = (i0 - st_i) / 16 < Qn;             // the batch's lowest row: uniform over the threads
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int i = i0 + u * 256;
         const int r = i >> 4, c = i & 15;
-        in[u] = i < 128 * 16 && r < Qn;
-        if (in[u])
-          load8_planes(A.q32 + (size_t)(seq * A.rows_per_seq + r / A.group) * A.q_ld + (g * A.group + r % A.group) * TC_DH + c * 8,
-                       A.q_splits, A.q_plane, x[u]);
+        in[u] = r < Qn;
+        const int rc = in[u] ? r : Qn - 1;
+        src[u] = A.q32 + (size_t)(seq * A.rows_per_seq + rc / A.group) * A.q_ld + (g * A.group + rc % A.group) * TC_DH + c * 8;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[u][e] = 0.f;
+      }
+      if (batch_live) {
+        for (int sp = 0; sp < A.q_splits; sp += 2) {
+          const bool two = sp + 1 < A.q_splits;
+          float4 a0[4], b0[4], a1[4], b1[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float* p0 = src[u] + (size_t)sp * A.q_plane;
+            const float* p1 = src[u] + (size_t)(two ? sp + 1 : sp) * A.q_plane;
+            a0[u] = ldcg4(p0); b0[u] = ldcg4(p0 + 4);
+            a1[u] = ldcg4(p1); b1[u] = ldcg4(p1 + 4);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {                            // planes added in index order
+            x[u][0] += a0[u].x; x[u][1] += a0[u].y; x[u][2] += a0[u].z; x[u][3] += a0[u].w;
+            x[u][4] += b0[u].x; x[u][5] += b0[u].y; x[u][6] += b0[u].z; x[u][7] += b0[u].w;
+            if (two) {
+              x[u][0] += a1[u].x; x[u][1] += a1[u].y; x[u][2] += a1[u].z; x[u][3] += a1[u].w;
+              x[u][4] += b1[u].x; x[u][5] += b1[u].y; x[u][6] += b1[u].z; x[u][7] += b1[u].w;
+            }
+          }
+        }
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int i = i0 + u * 256;
-        if (i >= 128 * 16) continue;
         const int r = i >> 4, c = i & 15;
         uint32_t hi[4] = {0u, 0u, 0u, 0u}, lo[4] = {0u, 0u, 0u, 0u};
         if (in[u]) {
@@ -345,9 +384,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attn_tc_kernel(const __grid_con
       const int n_in = max(0, min(64, n_blk - half * 64));              // of them in this thread's half
       if (n_blk < TC_KB) {
         // A ragged last block: positions beyond the range carry whatever the cache holds there. Their probabilities are
-        // exactly zero, but zero times a non-finite stale value is not, so those V rows are cleared in shared memory
-        // (the block has landed: its scores are complete).
-        uint8_t* v = bp + oKV + (b % TC_STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        // exactly zero, but zero times a non-finite stale value is not, so those V rows are cleared in shared memory,
+        // once the block's values have landed (its scores being complete says nothing about them).
+        if (!mbar_wait(vfull_bar(b % TC_STAGES), (uint32_t)(b / TC_STAGES) & 1u, abort_flag)) fail = true;
+        uint8_t* v = bp + v_off(b % TC_STAGES);
         for (int j = st_i; j < (TC_KB - n_blk) * 16; j += 256) {
           const int r = n_blk + (j >> 4), c16 = j & 15;                  // row, 16-byte piece of its 256 bytes
           *reinterpret_cast<uint4*>(v + (c16 >> 3) * (TC_KV_BYTES / 2) + r * 128 + (c16 & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
