@@ -31,7 +31,7 @@ struct NvtxRange {
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256, TC_MIN_KEYS = 4096 };
+enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256, TC_MIN_KEYS = 2048 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
