@@ -402,8 +402,9 @@ static moa_status attention(moa_ctx* ctx, cudaStream_t s, char* ws, const Worksp
     P.out = (bf16*)out;
     P.out_lo = lo_rows_of(sizeof(T), R);
     P.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
-    // Long dense caches (fp32 queries, head size 128, no per-row limits): the cache segment on the tcgen05 kernel, one CTA
-    // per SM; the tree segment, if any, as one more part from the split-KV kernel; merged together.
+    // Long dense caches (fp32 queries, head size 128, no per-row limits): the tcgen05 kernel, one CTA per (kv head,
+    // sequence, key range) and one more per sequence for the tree segment, if any; the parts are merged by the same
+    // kernel as the split-KV parts.
     if (q32 && dh == 128 && !lim.active() && ctx->fast && Qn <= 128 && posA_ld == hkv * dh && kA != nullptr &&
         max_len >= TC_MIN_KEYS && n_slots <= 256) {
       const int blocks = (max_len + TC_KB - 1) / TC_KB;
