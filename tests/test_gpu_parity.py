@@ -426,22 +426,32 @@ def test_lsa_tokens_are_independent_and_incremental_equals_full(dtype):
             H.assert_rows_close(a, b, tol, f"{what}: parts {parts[:3]}.. chunk {chunk} vs one call")
 
 
-def test_long_caches_take_the_tensor_core_attention_with_ragged_lengths():
-    """Caches of more than 4096 positions run their cache segment on the tcgen05 attention kernel (keys streamed by
-    TMA, scores and the output accumulator in TMEM); the tree segment stays on the split-KV kernel and the parts are
-    merged. Two sequences with different lengths, one of them with an empty self-attention prefix (key ranges of
-    zero blocks), lengths that are not multiples of the 64-position block."""
-    p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=1031, lsa_hq=2, lsa_hkv=2,
-                     lsa_mlp=128, sa_hq=4, sa_hkv=1, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=448, ctx=5000, batch=2,
-                     tree_topk=4, tree_depth=3, tree_keep=9, head_dim=128)
+@pytest.mark.parametrize("case", ["ragged", "wide_tree"])
+def test_long_caches_take_the_tensor_core_attention_with_ragged_lengths(case):
+    """Caches of 2048 positions and more run on the tcgen05 attention kernel (keys and values streamed by TMA in blocks
+    of 128 positions, queries, scores, probabilities and the output accumulator in tensor memory), the tree segment
+    as one more CTA of the same grid; the parts are merged by the split-KV kernel's merge.
+    "ragged": two sequences with different lengths, one of them with an empty self-attention prefix (key ranges of
+    zero blocks), lengths that are not multiples of the block, a last block whose second half is empty.
+    "wide_tree": 16 x 8 = 128 query rows per kv head (every tensor-memory lane in use), a tree of 145 slots (two tree
+    blocks, the second one ragged), lengths at and just above the 2048-position threshold."""
+    if case == "ragged":
+        p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=1031, lsa_hq=2, lsa_hkv=2,
+                         lsa_mlp=128, sa_hq=4, sa_hkv=1, sa_mlp=64, ca_hq=4, ca_hkv=2, ca_mlp=448, ctx=5000, batch=2,
+                         tree_topk=4, tree_depth=3, tree_keep=9, head_dim=128)
+        lens_ca, lens_sa = [5000, 4101], [4990, 0]
+    else:
+        p = synth.scaled(synth.PRESETS["c5"], d_model=256, n_stack=2, d_stack=128, vocab=1031, lsa_hq=2, lsa_hkv=2,
+                         lsa_mlp=128, sa_hq=8, sa_hkv=1, sa_mlp=64, ca_hq=8, ca_hkv=2, ca_mlp=192, ctx=2100, batch=2,
+                         tree_topk=16, tree_depth=10, tree_keep=60, head_dim=128)
+        lens_ca, lens_sa = [2100, 2048], [2049, 2090]
     w = synth.make_weights(p)
-    g = H.make_gpu(p, w, max_ctx=5056)
+    g = H.make_gpu(p, w, max_ctx=p.ctx + 56)
     exact, dec = H.make_oracles(p, w)
     caK, caV = synth.make_cache(p, "ca")
     saK, saV = synth.make_cache(p, "sa")
     g.fill_cache("ca", caK.cuda(), caV.cuda())
     g.fill_cache("sa", saK.cuda(), saV.cuda())
-    lens_ca, lens_sa = [5000, 4101], [4990, 0]
     g.moa_state_set_len("ca", lens_ca)
     g.moa_state_set_len("sa", lens_sa)
     root = synth.make_root(p)
@@ -470,4 +480,4 @@ def test_long_caches_take_the_tensor_core_attention_with_ragged_lengths():
         g.moa_tree_expand(torch.from_numpy(f_ids).cuda(), torch.from_numpy(f_lp).cuda())
     torch.cuda.synchronize()
     assert g.moa_state_status() == 0
-    print(f"[long caches, tensor-core attention] worst hidden {worst:.2e}")
+    print(f"[long caches, tensor-core attention, {case}] worst hidden {worst:.2e}")
