@@ -69,7 +69,7 @@ def assert_rows_close(got, want, tol, what=""):
 def tie_window(p: synth.Preset, z) -> float:
     """How close two of the oracle's log-probabilities must be for either order to count as correct.
 
-    fp32 path: 1e-3, as the task states. bf16 forwards of up to 256 rows: 1e-3 plus 2e-3 * max|z| -- weights,
+    fp32 path: 1e-3. bf16 forwards of up to 256 rows: 1e-3 plus 2e-3 * max|z| -- weights,
     cache entries and tree keys / values are stored in 16 bits whatever the arithmetic, which leaves the logits
     about 1e-3 * max|z| away from the fp64 oracle's (measured: worst 1.1e-3 on configs 2 and 4, 1.7e-3 on the
     reduced shapes). Larger bf16
@@ -88,7 +88,7 @@ def check_topk(gpu_ids, gpu_lp, z, tol, window=1e-3, what="", literal=None):
     Each reported log-probability must match the oracle's for that token within tol * max|z|; the j-th pick
     must be within `window` of the oracle's j-th best log-probability (either of two near-tied tokens is
     accepted); ids are distinct. Returns True when the id list equals the oracle's exactly. With `literal` (a
-    list) given, appends whether the row also passes the window the task states literally (1e-3)."""
+    list) given, appends whether the row also passes the plain 1e-3 window (no logit-scaled term)."""
     z = np.asarray(z, np.float64)
     lse = z.max() + np.log(np.exp(z - z.max()).sum())
     logp = z - lse

@@ -27,7 +27,7 @@ assert g.lib.moa_trace_begin is not None
 # a whole cycle against the oracle with every check armed: the status word must stay clear
 stats = run_cycle(p, g, H.make_oracles(p, w), synth.make_h_stack(p, p.lsa_tokens * 2), synth.make_tokens(p, p.ctx), synth.make_root(p))
 assert stats["rows"] == 2 * (1 + 2 * 5) and g.moa_state_status() == 0
-# a token id outside the vocabulary: the normal build clamps it silently, this build also reports it
+# a token id outside the vocabulary: the normal library clamps it silently, the checking variant also reports it
 g.moa_tree_begin(synth.make_root(p).cuda())
 g.moa_state_set_len("sa", [0, 0])
 bad = torch.tensor([3, p.vocab + 5, 7, 1], dtype=torch.int32).cuda()

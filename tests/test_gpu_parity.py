@@ -1,6 +1,6 @@
 """Parity of the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
 
-Tolerances (stated by the benchmark spec): hidden states and log-probabilities within
+Tolerances: hidden states and log-probabilities within
 max-abs 1e-4 (fp32 path) / 2e-2 (bf16 path) of the row's max |value|; token ids and tree structure
 bit-exact except where the oracle's competing log-probabilities differ by less than the tie window
 (1e-3 on the fp32 path; helpers.tie_window derives the bf16 ones). bf16 forwards of up to 256 rows (every draft
