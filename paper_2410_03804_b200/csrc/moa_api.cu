@@ -31,7 +31,7 @@ struct NvtxRange {
 static thread_local char g_cuda_err[256] = "";
 static thread_local long long g_launches = 0;
 
-enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256, TC_MIN_KEYS = 2048 };
+enum { PROF_MAX = 512, WMAP_MAX = 64, PREFILL_ROWS = 256, TC_MIN_KEYS = 2048, RN_ROWS_PER_CTA_FROM = 64 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -275,6 +275,15 @@ static inline int lo_rows_of(size_t elt, int R) {
   return R <= 128 ? npad_for(R) : LO_ROW_WIDE;
 }
 
+// Launch shape of rope_store_kernel for R rows of n_heads heads: eight threads per head; with few rows blocks of 64
+// threads (8 heads each) spread a row over several CTAs, with many rows blocks of 256 threads (32 heads each).
+static inline void rope_shape(const moa_ctx* ctx, int R, int n_heads, dim3* grid, dim3* block) {
+  (void)ctx;
+  const int per_block = R <= 32 ? 8 : 32;
+  *grid = dim3(R, (n_heads + per_block - 1) / per_block);
+  *block = dim3(per_block * 8);
+}
+
 static bool fast_shape(const moa_ctx* ctx, int K, int nseg, const void* const* W) {
   if (!ctx->fast || K % WS_BK != 0) return false;
   for (int i = 0; i < nseg; ++i)
@@ -474,7 +483,8 @@ template <typename T>
 static moa_status residual_norm(cudaStream_t s, const moa_ctx* ctx, char* ws, const Workspace& p, int R, int K,
                                 const LinOut* lo, const void* gain, void* hidden_out) {
   if (R <= 0) return MOA_OK;
-  if (K % (RN_CLUSTER * 8) == 0 && K / RN_CLUSTER <= 256 * 8 * (RN_MAX_PER_THREAD / 4)) {
+  // few rows: a cluster of 8 CTAs per row (a row alone cannot fill the machine); many rows: one CTA per row
+  if (R < RN_ROWS_PER_CTA_FROM && K % (RN_CLUSTER * 8) == 0 && K / RN_CLUSTER <= 256 * 8 * (RN_MAX_PER_THREAD / 4)) {
     launch_pdl(residual_norm_cluster_kernel<T>, dim3(dim3(RN_CLUSTER, R)), dim3(256), 0, s, 
         (float*)(ws + p.xres), lo ? lo->part : nullptr, lo ? lo->splits : 0, lo ? lo->plane : 0, K, (const T*)gain,
         ctx->c.rms_eps, (T*)(ws + p.xn), (T*)hidden_out, lo_rows_of(sizeof(T), R));
@@ -599,7 +609,9 @@ static moa_status sa_append_t(moa_ctx* ctx, moa_state* st, const int* tok, const
     rr.max_ctx = c.max_ctx;
     rr.split = split;
     rr.row0 = t0;
-    launch_pdl(rope_store_kernel<T>, dim3(dim3(R, 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
+    dim3 rgrid, rblock;
+    rope_shape(ctx, R, 2 * c.sa_hkv, &rgrid, &rblock);
+    launch_pdl(rope_store_kernel<T>, rgrid, rblock, 0, s, lo.part, lo.splits, lo.plane, 2 * nkv, 0, 0, nkv, 0, c.sa_hkv, dh,
                                            c.sa_rope_theta, st->sa_len, rr, (T*)nullptr, (float*)nullptr, (T*)st->sa_k, (T*)st->sa_v, (int*)status_word);
     MOA_CHECK_LAUNCH();
   }
@@ -715,7 +727,9 @@ static moa_status drafter_prefill_t(moa_ctx* ctx, moa_state* st, const int* tok,
       rr.max_ctx = c.max_ctx;
       rr.split = one;
       rr.row0 = r0;
-      launch_pdl(rope_store_kernel<T>, dim3(dim3(R, c.sa_hq + 2 * c.sa_hkv)), dim3(64), 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq,
+      dim3 rgrid, rblock;
+      rope_shape(ctx, R, c.sa_hq + 2 * c.sa_hkv, &rgrid, &rblock);
+      launch_pdl(rope_store_kernel<T>, rgrid, rblock, 0, s, lo.part, lo.splits, lo.plane, nq + 2 * nkv, 0, nq,
                  nq + nkv, c.sa_hq, c.sa_hkv, dh, c.sa_rope_theta, st->sa_len, rr, narrow, q32, (T*)st->sa_k, (T*)st->sa_v, (int*)status_word);
       MOA_CHECK_LAUNCH();
       // row i of the chunk sits at position base + r0 + i and sees positions 0 .. base + r0 + i
@@ -795,7 +809,9 @@ static moa_status tree_attn_layer(moa_ctx* ctx, moa_state* st, cudaStream_t s, c
   rr.step = step;
   rr.B = B;
   rr.slots = L.NS;
-  launch_pdl(rope_store_kernel<T>, dim3(dim3(R, a.hq + 2 * a.hkv)), dim3(64), 0, s, lo->part, lo->splits, lo->plane, nq + 2 * nkv, 0, nq,
+  dim3 rgrid, rblock;
+  rope_shape(ctx, R, a.hq + 2 * a.hkv, &rgrid, &rblock);
+  launch_pdl(rope_store_kernel<T>, rgrid, rblock, 0, s, lo->part, lo->splits, lo->plane, nq + 2 * nkv, 0, nq,
              nq + nkv, a.hq, a.hkv, dh, a.theta, st->sa_len, rr, narrow, q32, (T*)a.tk, (T*)a.tv, (int*)status_word);
   MOA_CHECK_LAUNCH();
   MOA_TRY(attention<T>(ctx, s, ws, p, dh, narrow, q32, 1, 0, nq, R, a.hq, a.hkv, (const T*)a.ck, (const T*)a.cv, c.max_ctx, nkv,

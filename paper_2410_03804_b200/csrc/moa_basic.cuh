@@ -342,7 +342,7 @@ struct RopeRows {
 };
 
 template <typename T>
-__global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, size_t plane, int ld, int q_off, int k_off,
+__global__ void __launch_bounds__(256) rope_store_kernel(const float* __restrict__ qkv, int splits, size_t plane, int ld, int q_off, int k_off,
                                   int v_off,
                                   int hq, int hkv, int dh, float theta, const int* __restrict__ pos_base,
                                   RopeRows rr, T* __restrict__ qdst, float* __restrict__ qdst32, T* __restrict__ kdst,
@@ -388,35 +388,53 @@ __global__ void rope_store_kernel(const float* __restrict__ qkv, int splits, siz
   }
   __syncthreads();
   const float* row0 = qkv + (size_t)r * ld;
-  auto row = [&](int c) { return load1_planes(row0 + c, splits, plane); };   // planes added in a fixed order
-  // blockIdx.y walks the heads: query heads (when qdst is given), then key heads, then value heads
-  int h = blockIdx.y;
+  // Heads: query heads (when qdst is given), then key heads, then value heads. Eight threads share a head, each with
+  // 8 consecutive elements of both halves (16-byte loads of every split plane, planes added in a fixed order); the
+  // block's blockDim.x / 8 groups take heads blockIdx.y * groups + g, then every gridDim.y * groups-th one.
   const int nqh = qdst ? hq : 0;
-  if (h < nqh) {
-    for (int j = threadIdx.x; j < half; j += blockDim.x) {
-      const float x1 = row(q_off + h * dh + j), x2 = row(q_off + h * dh + half + j);
-      if (qdst32) {                    // rotated queries kept in fp32 (the attention kernel splits them)
-        qdst32[(size_t)r * hq * dh + h * dh + j] = x1 * cs[j] - x2 * sn[j];
-        qdst32[(size_t)r * hq * dh + h * dh + half + j] = x2 * cs[j] + x1 * sn[j];
-      } else {
-        qdst[(size_t)r * hq * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
-        qdst[(size_t)r * hq * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+  const int n_heads = nqh + 2 * hkv;
+  const int groups = blockDim.x >> 3, slot = threadIdx.x >> 3, j0 = threadIdx.x & 7;
+  for (int hh = blockIdx.y * groups + slot; hh < n_heads; hh += gridDim.y * groups) {
+    int h = hh;
+    const bool is_q = h < nqh;
+    if (!is_q) h -= nqh;
+    if (!is_q && !store_kv) continue;
+    if (is_q || h < hkv) {                               // rotated: element i pairs with i + dh/2
+      const int off = (is_q ? q_off : k_off) + h * dh;
+      for (int i = j0; i < (half >> 3); i += 8) {
+        float a[8], b2[8], o1[8], o2[8];
+        load8_planes(row0 + off + i * 8, splits, plane, a);
+        load8_planes(row0 + off + half + i * 8, splits, plane, b2);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float c = cs[i * 8 + e], sv = sn[i * 8 + e];
+          o1[e] = a[e] * c - b2[e] * sv;
+          o2[e] = b2[e] * c + a[e] * sv;
+        }
+        if (is_q) {
+          const size_t at = (size_t)r * hq * dh + h * dh + i * 8;
+          if (qdst32) {                  // rotated queries kept in fp32 (the attention kernel splits them)
+            store8<float>(qdst32 + at, o1);
+            store8<float>(qdst32 + at + half, o2);
+          } else {
+            store8<T>(qdst + at, o1);
+            store8<T>(qdst + at + half, o2);
+          }
+        } else {
+          const size_t at = dst * hkv * dh + h * dh + i * 8;
+          store8<T>(kdst + at, o1);
+          store8<T>(kdst + at + half, o2);
+        }
       }
+      continue;
     }
-    return;
-  }
-  h -= nqh;
-  if (!store_kv) return;
-  if (h < hkv) {
-    for (int j = threadIdx.x; j < half; j += blockDim.x) {
-      const float x1 = row(k_off + h * dh + j), x2 = row(k_off + h * dh + half + j);
-      kdst[dst * hkv * dh + h * dh + j] = from_f<T>(x1 * cs[j] - x2 * sn[j]);
-      kdst[dst * hkv * dh + h * dh + half + j] = from_f<T>(x2 * cs[j] + x1 * sn[j]);
+    h -= hkv;
+    for (int i = j0; i < (dh >> 3); i += 8) {
+      float v8[8];
+      load8_planes(row0 + v_off + h * dh + i * 8, splits, plane, v8);
+      store8<T>(vdst + dst * hkv * dh + h * dh + i * 8, v8);
     }
-    return;
   }
-  h -= hkv;
-  for (int j = threadIdx.x; j < dh; j += blockDim.x) vdst[dst * hkv * dh + h * dh + j] = from_f<T>(row(v_off + h * dh + j));
 }
 
 // Cross-attention cache append: fp32 [n, hkv*dh] k and v rows -> T cache rows at (seq, ca_len[seq] + i).
